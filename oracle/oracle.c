@@ -1,0 +1,436 @@
+/*
+ * CPU oracle for HAG aggregation -- TEST INFRASTRUCTURE, not part of the product.
+ *
+ * Plain, slow, single-threaded C.  Only tests, the smoke check and the
+ * benchmark's CPU-baseline leg may call it; the CUDA library never does and
+ * shares no code with it.
+ *
+ * What each function follows in the paper (arxiv 1906.03707):
+ *   o1_direct_forward   Algorithm 1 line 4 with the GCN row of Table 1:
+ *                       a_v = sum over u in N(v) of h_u   (mean: divided by |N(v)|)
+ *   o2_direct_backward  equivalence clause (2) of Section 3.2 ("the same
+ *                       gradients"): gx_u = sum over v with u in N(v) of s_v g_v
+ *   o4_hag_forward      Algorithm 2 lines 3-8, evaluated over a given HAG
+ *   o4_hag_backward     the adjoint of Algorithm 2 over the transposed HAG
+ *   o3b_greedy          Algorithm 3, set-Aggregate branch, with the pair-count
+ *                       heap the complexity appendix sketches
+ *   o_count_pair / o_max_pair_recount   the Redundancy function of Algorithm 3
+ *                       evaluated from its definition
+ *
+ * All floating point is fp64.  Graph layout: CSR of in-neighbours, row v lists
+ * the sources u of v, int64 row pointers, int32 sorted duplicate-free columns.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <math.h>
+
+/* ------------------------------------------------------------------------- */
+/* O1: direct forward.  rows == NULL: all n rows, out is n x d.  Otherwise out
+ * is n_rows x d, row i holding the result for node rows[i].  abs_out (may be
+ * NULL) receives sum |x_u| (mean: divided by |N(v)|), the tolerance scale.   */
+void o1_direct_forward(int64_t n, const int64_t *row_ptr, const int32_t *col, int64_t d,
+                       const double *x, int mean, const int64_t *rows, int64_t n_rows,
+                       double *out, double *abs_out)
+{
+    int64_t count = rows ? n_rows : n;
+    for (int64_t i = 0; i < count; ++i) {
+        int64_t v = rows ? rows[i] : i;
+        double *o = out + i * d;
+        double *ao = abs_out ? abs_out + i * d : NULL;
+        for (int64_t k = 0; k < d; ++k) o[k] = 0.0;
+        if (ao) for (int64_t k = 0; k < d; ++k) ao[k] = 0.0;
+        for (int64_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) {
+            const double *xu = x + (int64_t)col[e] * d;
+            for (int64_t k = 0; k < d; ++k) o[k] += xu[k];
+            if (ao) for (int64_t k = 0; k < d; ++k) ao[k] += fabs(xu[k]);
+        }
+        int64_t deg = row_ptr[v + 1] - row_ptr[v];
+        if (mean && deg > 0) {
+            for (int64_t k = 0; k < d; ++k) o[k] /= (double)deg;
+            if (ao) for (int64_t k = 0; k < d; ++k) ao[k] /= (double)deg;
+        }
+    }
+}
+
+/* O2: direct backward.  slot == NULL: gx is n x d and every source row is
+ * produced.  Otherwise slot[u] is -1 (skip) or the row of gx that receives
+ * node u's gradient (gx then has as many rows as there are slots).          */
+void o2_direct_backward(int64_t n, const int64_t *row_ptr, const int32_t *col, int64_t d,
+                        const double *g, int mean, const int64_t *slot, int64_t n_slots,
+                        double *gx, double *abs_gx)
+{
+    int64_t out_rows = slot ? n_slots : n;
+    memset(gx, 0, sizeof(double) * (size_t)(out_rows * d));
+    if (abs_gx) memset(abs_gx, 0, sizeof(double) * (size_t)(out_rows * d));
+    for (int64_t v = 0; v < n; ++v) {
+        int64_t deg = row_ptr[v + 1] - row_ptr[v];
+        double s = (mean && deg > 0) ? 1.0 / (double)deg : 1.0;
+        const double *gv = g + v * d;
+        for (int64_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) {
+            int64_t u = col[e];
+            int64_t r = slot ? slot[u] : u;
+            if (r < 0) continue;
+            double *o = gx + r * d;
+            for (int64_t k = 0; k < d; ++k) o[k] += s * gv[k];
+            if (abs_gx) {
+                double *ao = abs_gx + r * d;
+                for (int64_t k = 0; k < d; ++k) ao[k] += fabs(s * gv[k]);
+            }
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* O4: Algorithm 2 over a HAG in canonical layout.
+ *   ids 0..n-1 graph nodes, n..n+num_agg-1 aggregation nodes in an order in
+ *   which every aggregation node comes after both of its inputs;
+ *   agg_in[2j], agg_in[2j+1]: the two inputs of aggregation node n+j;
+ *   res_ptr/res_idx: the remaining in-neighbours of every graph node;
+ *   in_degree[v] = |N(v)| in the input graph (mean divides by it).
+ * scratch: (n + num_agg) x d doubles, the a-hat buffer of Algorithm 2.        */
+void o4_hag_forward(int64_t n, int64_t num_agg, const int32_t *agg_in,
+                    const int64_t *res_ptr, const int32_t *res_idx, const int32_t *in_degree,
+                    int64_t d, const double *x, int mean, double *scratch, double *out)
+{
+    double *ahat = scratch;
+    memcpy(ahat, x, sizeof(double) * (size_t)(n * d));                 /* lines 3-4 */
+    for (int64_t j = 0; j < num_agg; ++j) {                            /* lines 5-6 */
+        const double *p = ahat + (int64_t)agg_in[2 * j] * d;
+        const double *q = ahat + (int64_t)agg_in[2 * j + 1] * d;
+        double *w = ahat + (n + j) * d;
+        for (int64_t k = 0; k < d; ++k) w[k] = p[k] + q[k];
+    }
+    for (int64_t v = 0; v < n; ++v) {                                  /* lines 7-8 */
+        double *o = out + v * d;
+        for (int64_t k = 0; k < d; ++k) o[k] = 0.0;
+        for (int64_t e = res_ptr[v]; e < res_ptr[v + 1]; ++e) {
+            const double *a = ahat + (int64_t)res_idx[e] * d;
+            for (int64_t k = 0; k < d; ++k) o[k] += a[k];
+        }
+        if (mean && in_degree[v] > 0)
+            for (int64_t k = 0; k < d; ++k) o[k] /= (double)in_degree[v];
+    }
+}
+
+/* Adjoint of the above over the transposed HAG: t_ptr has n+num_agg+1
+ * entries, row s lists the destinations of source s; a destination < n is the
+ * OUTPUT row of that graph node, a destination >= n an aggregation node.
+ * Aggregation nodes are visited in reverse canonical order, then the graph
+ * nodes as sources.  scratch: num_agg x d doubles.                           */
+void o4_hag_backward(int64_t n, int64_t num_agg, const int64_t *t_ptr, const int32_t *t_idx,
+                     const int32_t *in_degree, int64_t d, const double *g, int mean,
+                     double *scratch, double *gx)
+{
+    double *ghat = scratch;
+    for (int64_t s = n + num_agg - 1; s >= 0; --s) {
+        double *o = (s >= n) ? ghat + (s - n) * d : gx + s * d;
+        for (int64_t k = 0; k < d; ++k) o[k] = 0.0;
+        for (int64_t e = t_ptr[s]; e < t_ptr[s + 1]; ++e) {
+            int64_t dst = t_idx[e];
+            if (dst < n) {
+                double sc = (mean && in_degree[dst] > 0) ? 1.0 / (double)in_degree[dst] : 1.0;
+                const double *gv = g + dst * d;
+                for (int64_t k = 0; k < d; ++k) o[k] += sc * gv[k];
+            } else {
+                const double *gh = ghat + (dst - n) * d;
+                for (int64_t k = 0; k < d; ++k) o[k] += gh[k];
+            }
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Redundancy(v1, v2) from its definition: the number of graph-node rows of the
+ * current edge set that contain both.  cur_ptr/cur_len/cur_idx: row u occupies
+ * cur_idx[cur_ptr[u] .. cur_ptr[u]+cur_len[u]), sorted.                       */
+static int row_has(const int32_t *row, int32_t len, int32_t key)
+{
+    int32_t lo = 0, hi = len;
+    while (lo < hi) {
+        int32_t mid = lo + (hi - lo) / 2;
+        if (row[mid] < key) lo = mid + 1; else hi = mid;
+    }
+    return lo < len && row[lo] == key;
+}
+
+int64_t o_count_pair(int64_t n, const int64_t *cur_ptr, const int32_t *cur_len, const int32_t *cur_idx,
+                     int32_t v1, int32_t v2)
+{
+    int64_t r = 0;
+    for (int64_t u = 0; u < n; ++u) {
+        const int32_t *row = cur_idx + cur_ptr[u];
+        if (row_has(row, cur_len[u], v1) && row_has(row, cur_len[u], v2)) ++r;
+    }
+    return r;
+}
+
+/* Full recount for one node a: over every row that holds a, count every other
+ * member; returns the largest count, *best_partner = the smallest id attaining
+ * it.  counts: zeroed scratch of n_ids int32, left zeroed on return.          */
+int64_t o_max_pair_recount(int64_t n, const int64_t *cur_ptr, const int32_t *cur_len, const int32_t *cur_idx,
+                           int64_t n_ids, int32_t a, int32_t *counts, int32_t *best_partner)
+{
+    int64_t best = 0;
+    int32_t arg = -1;
+    for (int64_t u = 0; u < n; ++u) {
+        const int32_t *row = cur_idx + cur_ptr[u];
+        if (!row_has(row, cur_len[u], a)) continue;
+        for (int32_t i = 0; i < cur_len[u]; ++i) if (row[i] != a) counts[row[i]]++;
+    }
+    for (int64_t y = 0; y < n_ids; ++y) {
+        if (counts[y] > best) { best = counts[y]; arg = (int32_t)y; }
+    }
+    for (int64_t u = 0; u < n; ++u) {
+        const int32_t *row = cur_idx + cur_ptr[u];
+        if (!row_has(row, cur_len[u], a)) continue;
+        for (int32_t i = 0; i < cur_len[u]; ++i) counts[row[i]] = 0;
+    }
+    *best_partner = arg;
+    return best;
+}
+
+/* ------------------------------------------------------------------------- */
+/* O3b: Algorithm 3 (set Aggregate) with an explicit map pair -> redundancy and
+ * a max-heap over (redundancy, pair), as the complexity appendix describes.
+ * The heap is lazy: an entry is valid only while the map still shows its
+ * count; counts of existing pairs only ever fall and a new pair gets its
+ * count once, so every live (pair, count >= 2) has exactly one valid entry.
+ * Tie-break: highest redundancy, then the smallest v1, then the smallest v2
+ * (v1 < v2, aggregation nodes numbered n, n+1, ... in creation order).       */
+
+typedef struct { uint64_t *keys; int32_t *vals; uint64_t mask; uint64_t used; } pairmap;
+#define PM_EMPTY UINT64_MAX
+
+static uint64_t pm_hash(uint64_t k) {
+    k ^= k >> 33; k *= 0xff51afd7ed558ccdULL; k ^= k >> 33; k *= 0xc4ceb9fe1a85ec53ULL; k ^= k >> 33;
+    return k;
+}
+static int pm_init(pairmap *m, uint64_t cap_pow2) {
+    m->keys = (uint64_t *)malloc(sizeof(uint64_t) * cap_pow2);
+    m->vals = (int32_t *)malloc(sizeof(int32_t) * cap_pow2);
+    if (!m->keys || !m->vals) return -1;
+    memset(m->keys, 0xff, sizeof(uint64_t) * cap_pow2);
+    m->mask = cap_pow2 - 1; m->used = 0;
+    return 0;
+}
+static void pm_free(pairmap *m) { free(m->keys); free(m->vals); }
+static int32_t *pm_slot(pairmap *m, uint64_t key);
+static int pm_grow(pairmap *m) {
+    pairmap bigger;
+    if (pm_init(&bigger, (m->mask + 1) * 2)) return -1;
+    for (uint64_t i = 0; i <= m->mask; ++i)
+        if (m->keys[i] != PM_EMPTY) *pm_slot(&bigger, m->keys[i]) = m->vals[i];
+    pm_free(m);
+    *m = bigger;
+    return 0;
+}
+/* pointer to the count of `key`, inserted with 0 if absent (NULL: out of memory) */
+static int32_t *pm_slot(pairmap *m, uint64_t key) {
+    if ((m->used + 1) * 10 > (m->mask + 1) * 6) { if (pm_grow(m)) return NULL; }
+    uint64_t i = pm_hash(key) & m->mask;
+    while (m->keys[i] != PM_EMPTY && m->keys[i] != key) i = (i + 1) & m->mask;
+    if (m->keys[i] == PM_EMPTY) { m->keys[i] = key; m->vals[i] = 0; m->used++; }
+    return &m->vals[i];
+}
+static uint64_t pair_key(int32_t a, int32_t b) {
+    if (a > b) { int32_t t = a; a = b; b = t; }
+    return ((uint64_t)(uint32_t)a << 32) | (uint32_t)b;
+}
+
+typedef struct { int32_t cnt, a, b; } hent;
+/* 1 if x must come out of the heap before y */
+static int h_before(const hent *x, const hent *y) {
+    if (x->cnt != y->cnt) return x->cnt > y->cnt;
+    if (x->a != y->a) return x->a < y->a;
+    return x->b < y->b;
+}
+typedef struct { hent *e; int64_t n, cap; } heap;
+static int h_push(heap *h, hent v) {
+    if (h->n == h->cap) {
+        int64_t nc = h->cap ? h->cap * 2 : 1024;
+        hent *ne = (hent *)realloc(h->e, sizeof(hent) * (size_t)nc);
+        if (!ne) return -1;
+        h->e = ne; h->cap = nc;
+    }
+    int64_t i = h->n++;
+    while (i > 0) {
+        int64_t p = (i - 1) / 2;
+        if (!h_before(&v, &h->e[p])) break;
+        h->e[i] = h->e[p]; i = p;
+    }
+    h->e[i] = v;
+    return 0;
+}
+static hent h_pop(heap *h) {
+    hent top = h->e[0];
+    hent last = h->e[--h->n];
+    int64_t i = 0;
+    for (;;) {
+        int64_t l = 2 * i + 1, r = l + 1, c;
+        if (l >= h->n) break;
+        c = (r < h->n && h_before(&h->e[r], &h->e[l])) ? r : l;
+        if (!h_before(&h->e[c], &last)) break;
+        h->e[i] = h->e[c]; i = c;
+    }
+    if (h->n > 0) h->e[i] = last;
+    return top;
+}
+
+typedef struct { int32_t *v; int32_t len; } ilist;
+
+/* Returns the number of aggregation nodes created (<= capacity), or a negative
+ * number when memory runs out.
+ *   trace_v1/v2/r: capacity entries each, the merged pair (creation ids,
+ *                  v1 < v2) and its redundancy, in creation order;
+ *   cur_len[n], cur_idx[E]: on return row u's remaining in-neighbours (creation
+ *                  ids, ascending) are cur_idx[row_ptr[u] .. row_ptr[u]+cur_len[u]).
+ *   final_max_redundancy: the largest redundancy left when the loop stopped.  */
+int64_t o3b_greedy(int64_t n, const int64_t *row_ptr, const int32_t *col, int64_t capacity,
+                   int32_t *trace_v1, int32_t *trace_v2, int32_t *trace_r,
+                   int32_t *cur_len, int32_t *cur_idx, int32_t *final_max_redundancy)
+{
+    int64_t E = row_ptr[n];
+    int64_t n_ids = n + capacity;
+    int64_t num_agg = 0, rc = 0;
+    pairmap map; heap hp = {0, 0, 0};
+    ilist *out = (ilist *)calloc((size_t)n_ids, sizeof(ilist));
+    int32_t *out_store = (int32_t *)malloc(sizeof(int32_t) * (size_t)(E > 0 ? E : 1));
+    int32_t *delta = (int32_t *)calloc((size_t)n_ids, sizeof(int32_t));
+    int32_t *touched = (int32_t *)malloc(sizeof(int32_t) * (size_t)n_ids);
+    int32_t *users = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n > 0 ? n : 1));
+    uint64_t cap0 = 1024;
+    *final_max_redundancy = 0;
+    if (!out || !out_store || !delta || !touched || !users || pm_init(&map, cap0)) return -1;
+
+    memcpy(cur_idx, col, sizeof(int32_t) * (size_t)E);
+    for (int64_t u = 0; u < n; ++u) cur_len[u] = (int32_t)(row_ptr[u + 1] - row_ptr[u]);
+
+    /* out(s): the graph nodes whose row holds s (ascending because u ascends) */
+    {
+        int64_t *fill = (int64_t *)calloc((size_t)n + 1, sizeof(int64_t));
+        if (!fill) return -1;
+        for (int64_t e = 0; e < E; ++e) fill[col[e] + 1]++;
+        for (int64_t s = 0; s < n; ++s) fill[s + 1] += fill[s];
+        for (int64_t s = 0; s < n; ++s) { out[s].v = out_store + fill[s]; out[s].len = 0; }
+        for (int64_t u = 0; u < n; ++u)
+            for (int64_t e = row_ptr[u]; e < row_ptr[u + 1]; ++e) { ilist *l = &out[col[e]]; l->v[l->len++] = (int32_t)u; }
+        free(fill);
+    }
+
+    /* initial redundancy of every pair that shares at least one row */
+    for (int64_t u = 0; u < n; ++u) {
+        const int32_t *row = col + row_ptr[u];
+        int32_t len = cur_len[u];
+        for (int32_t i = 0; i < len; ++i)
+            for (int32_t j = i + 1; j < len; ++j) {
+                int32_t *c = pm_slot(&map, pair_key(row[i], row[j]));
+                if (!c) { rc = -1; goto done; }
+                (*c)++;
+            }
+    }
+    for (uint64_t i = 0; i <= map.mask; ++i)
+        if (map.keys[i] != PM_EMPTY && map.vals[i] >= 2) {
+            hent h = { map.vals[i], (int32_t)(map.keys[i] >> 32), (int32_t)(map.keys[i] & 0xffffffffu) };
+            if (h_push(&hp, h)) { rc = -1; goto done; }
+        }
+
+    while (num_agg < capacity) {
+        /* argmax of Redundancy over all pairs */
+        hent top; int found = 0;
+        while (hp.n > 0) {
+            top = h_pop(&hp);
+            int32_t *c = pm_slot(&map, pair_key(top.a, top.b));
+            if (!c) { rc = -1; goto done; }
+            if (*c == top.cnt) { found = 1; break; }
+        }
+        if (!found || top.cnt <= 1) break;                     /* "if Redundancy > 1" */
+        int32_t v1 = top.a, v2 = top.b, w = (int32_t)(n + num_agg);
+
+        /* R = { u : (v1,u) and (v2,u) are edges } */
+        int32_t nu = 0;
+        {
+            ilist *A = &out[v1], *B = &out[v2];
+            int32_t i = 0, j = 0;
+            while (i < A->len && j < B->len) {
+                if (A->v[i] < B->v[j]) ++i; else if (A->v[i] > B->v[j]) ++j;
+                else { users[nu++] = A->v[i]; ++i; ++j; }
+            }
+        }
+        if (nu != top.cnt) { rc = -2; goto done; }              /* map and rows disagree */
+        trace_v1[num_agg] = v1; trace_v2[num_agg] = v2; trace_r[num_agg] = nu;
+
+        /* how often every other member y shares a row of R with the pair */
+        int32_t nt = 0;
+        for (int32_t k = 0; k < nu; ++k) {
+            int32_t u = users[k];
+            int32_t *row = cur_idx + row_ptr[u];
+            for (int32_t i = 0; i < cur_len[u]; ++i) {
+                int32_t y = row[i];
+                if (y == v1 || y == v2) continue;
+                if (delta[y]++ == 0) touched[nt++] = y;
+            }
+        }
+        for (int32_t t = 0; t < nt; ++t) {
+            int32_t y = touched[t], dl = delta[y];
+            delta[y] = 0;
+            int32_t ends[2] = { v1, v2 };
+            for (int q = 0; q < 2; ++q) {
+                int32_t *c = pm_slot(&map, pair_key(ends[q], y));
+                if (!c) { rc = -1; goto done; }
+                *c -= dl;
+                if (*c >= 2) {
+                    hent h = { *c, ends[q] < y ? ends[q] : y, ends[q] < y ? y : ends[q] };
+                    if (h_push(&hp, h)) { rc = -1; goto done; }
+                }
+            }
+            int32_t *c = pm_slot(&map, pair_key(y, w));
+            if (!c) { rc = -1; goto done; }
+            *c = dl;
+            if (dl >= 2) { hent h = { dl, y, w }; if (h_push(&hp, h)) { rc = -1; goto done; } }
+        }
+        { int32_t *c = pm_slot(&map, pair_key(v1, v2)); if (!c) { rc = -1; goto done; } *c -= nu; }
+
+        /* E-hat <- E-hat - (v1,u) - (v2,u) + (w,u) for u in R; + (v1,w) + (v2,w) */
+        for (int32_t k = 0; k < nu; ++k) {
+            int32_t u = users[k];
+            int32_t *row = cur_idx + row_ptr[u];
+            int32_t len = cur_len[u], o = 0;
+            for (int32_t i = 0; i < len; ++i) if (row[i] != v1 && row[i] != v2) row[o++] = row[i];
+            row[o++] = w;                                       /* w exceeds every older id */
+            cur_len[u] = o;
+        }
+        {
+            int32_t ends[2] = { v1, v2 };
+            for (int q = 0; q < 2; ++q) {
+                ilist *L = &out[ends[q]];
+                int32_t o = 0, k = 0;
+                for (int32_t i = 0; i < L->len; ++i) {
+                    while (k < nu && users[k] < L->v[i]) ++k;
+                    if (k < nu && users[k] == L->v[i]) continue;
+                    L->v[o++] = L->v[i];
+                }
+                L->len = o;
+            }
+            out[w].v = (int32_t *)malloc(sizeof(int32_t) * (size_t)nu);
+            if (!out[w].v) { rc = -1; goto done; }
+            memcpy(out[w].v, users, sizeof(int32_t) * (size_t)nu);
+            out[w].len = nu;
+        }
+        ++num_agg;
+    }
+    /* what is left: the best still-valid entry, if any */
+    while (hp.n > 0) {
+        hent top = h_pop(&hp);
+        int32_t *c = pm_slot(&map, pair_key(top.a, top.b));
+        if (c && *c == top.cnt) { *final_max_redundancy = top.cnt; break; }
+    }
+    if (*final_max_redundancy == 0 && map.used > 0) {
+        for (uint64_t i = 0; i <= map.mask; ++i)
+            if (map.keys[i] != PM_EMPTY && map.vals[i] > *final_max_redundancy) *final_max_redundancy = map.vals[i];
+    }
+done:
+    for (int64_t s = n; s < n_ids; ++s) free(out[s].v);
+    free(out); free(out_store); free(delta); free(touched); free(users); free(hp.e); pm_free(&map);
+    return rc < 0 ? rc : num_agg;
+}
