@@ -1,0 +1,180 @@
+/*
+ * hag.h -- C ABI of the B200 HAG aggregation library.
+ *
+ * Sum / mean neighbourhood aggregation of a GNN layer, forward and backward,
+ * evaluated over a Hierarchically Aggregated computation Graph (HAG) as defined
+ * in "Redundancy-Free Computation Graphs for Graph Neural Networks"
+ * (arxiv 1906.03707).  The three operations the paper implements
+ * (Section 5.1: graph_to_hag, hag_aggregate, hag_aggregate_grad) map to
+ * hag_build, hag_aggregate_fwd and hag_aggregate_bwd; csr_aggregate_* evaluate
+ * the plain GNN-graph (the special case V_A = {} of Section 3.1) with the same
+ * kernels, as the comparison path.
+ *
+ * Conventions
+ *   ids        graph nodes 0..N-1; aggregation nodes N..N+|V_A|-1, sorted by level
+ *              (level = longest path from a graph node; every aggregation node
+ *              comes after both of its inputs).
+ *   graphs     CSR of IN-neighbours on the HOST: row v lists the sources u that v
+ *              aggregates (the edge (u,v) of Section 3.1), int64 row_ptr[N+1],
+ *              int32 col_idx[E], every row strictly ascending (no duplicates).
+ *              Self-loops are ordinary edges.
+ *   features   x, out, grad_out, grad_x are DEVICE pointers to N x D row-major
+ *              contiguous matrices of the given dtype, 16-byte aligned, with
+ *              D * sizeof(dtype) a multiple of 16.
+ *   workspace  DEVICE pointer to hag_workspace_bytes() bytes, 16-byte aligned; holds
+ *              the fp32 rows of the aggregation nodes (a-hat of Algorithm 2, or their
+ *              gradients).  It carries nothing between calls and may be shared by
+ *              all layers and by forward and backward (Algorithm 2's caption).
+ *   streams    cuda_stream is a cudaStream_t passed as void* (NULL = default
+ *              stream).  Calls only enqueue work; they never synchronise.
+ *   errors     every function returns a hag_status; nothing throws, aborts or
+ *              traps.  Argument checks are synchronous.  A failing kernel surfaces
+ *              at the caller's next synchronisation, as usual for CUDA.
+ *   threads    a handle may be used from one thread at a time.
+ *   results    no floating-point atomics anywhere: the same inputs give the same
+ *              bits on every run.
+ */
+#ifndef HAG_B200_H
+#define HAG_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hag hag_t; /* opaque: owns the structure arrays on host and device */
+
+typedef enum {
+    HAG_OK = 0,
+    HAG_ERR_NULL = 1,        /* a required pointer is NULL                                  */
+    HAG_ERR_ARG = 2,         /* a scalar argument is out of range                           */
+    HAG_ERR_GRAPH = 3,       /* malformed CSR (unsorted / duplicate / out-of-range columns) */
+    HAG_ERR_OOM_HOST = 4,
+    HAG_ERR_OOM_DEVICE = 5,
+    HAG_ERR_CUDA = 6,        /* a CUDA runtime call failed (incl. no device)                */
+    HAG_ERR_DTYPE = 7,
+    HAG_ERR_ALIGN = 8,       /* pointer or row size not 16-byte aligned                     */
+    HAG_ERR_WORKSPACE = 9,   /* workspace missing although the HAG has aggregation nodes    */
+    HAG_ERR_TIMEOUT = 10,    /* reserved: a bounded device-side wait gave up                */
+    HAG_ERR_NOT_ON_DEVICE = 11 /* hag_to_device has not been called                         */
+} hag_status;
+
+typedef enum { HAG_SUM = 0, HAG_MEAN = 1 } hag_reduce;
+typedef enum { HAG_F32 = 0, HAG_BF16 = 1 } hag_dtype;
+
+/* Counters of one built HAG.  "aggregations" are binary aggregations as counted
+ * by the cost function of Section 4.1: sum over nodes of (in-edges - 1). */
+typedef struct hag_info {
+    int32_t n;                      /* |V|                                                    */
+    int32_t capacity;               /* the limit that was asked for                           */
+    int32_t num_agg;                /* |V_A| (<= capacity: the search stops at redundancy 1)   */
+    int32_t num_levels;             /* depth of the hierarchy                                 */
+    int64_t e;                      /* |E| of the input graph (directed)                      */
+    int64_t e_hat;                  /* |E-hat| = 2 |V_A| + residual edges                     */
+    int64_t aggregations_gnn;       /* sum_v max(|N(v)| - 1, 0)                               */
+    int64_t aggregations_hag;       /* the same sum over V and V_A of the HAG                 */
+    int64_t aggregations_hag_closed;/* |E-hat| - |V| - |V_A| (equal when no row is empty)     */
+    int64_t saved;                  /* sum_i (r_i - 1) = f of the Theorem 4 proof             */
+    int32_t first_redundancy;       /* r of the first merge (0 if none)                       */
+    int32_t last_redundancy;        /* r of the last merge                                    */
+    int32_t max_in_degree;          /* longest row of the input graph                         */
+    int32_t max_res_degree;         /* longest residual row                                   */
+    int32_t max_out_degree;         /* longest row of the transposed HAG                      */
+    int32_t device;                 /* CUDA device holding the arrays, -1 if host only        */
+    double build_seconds;           /* host time spent in the search and layout               */
+} hag_info;
+
+/* Borrowed HOST views of the canonical arrays; valid until hag_destroy. */
+typedef struct hag_arrays {
+    int32_t n, num_agg, num_levels;
+    const int64_t *level_ptr;  /* [num_levels+1] level l (1-based) = ids n+level_ptr[l-1] .. n+level_ptr[l]-1 */
+    const int32_t *agg_in;     /* [2*num_agg] inputs (lo < hi) of aggregation node n+j                 */
+    const int64_t *res_ptr;    /* [n+1]                                                                */
+    const int32_t *res_idx;    /* residual in-neighbours of every graph node, ascending                */
+    const int64_t *t_ptr;      /* [n+num_agg+1] transposed HAG, by source                              */
+    const int32_t *t_idx;      /* destinations ascending; d < n: output row d; d >= n: aggregation node */
+    const int32_t *in_degree;  /* [n] |N(v)| of the input graph                                        */
+    const int32_t *trace;      /* [3*num_agg] merges in creation order: v1 < v2 (creation ids), r      */
+    const int64_t *csr_t_ptr;  /* [n+1] transposed input graph                                          */
+    const int32_t *csr_t_idx;
+} hag_arrays;
+
+/* Algorithm 3, set-Aggregate branch (the paper's graph_to_hag): starting from the
+ * GNN-graph, repeatedly merge the pair of nodes (graph or aggregation nodes) that
+ * the most graph nodes aggregate together into a new aggregation node, until
+ * `capacity` nodes exist or no pair is shared by more than one node.  Ties go to
+ * the lexicographically smallest pair (v1 < v2; aggregation nodes numbered N, N+1,
+ * ... as created).  Then lays the result out for the device (levels, level-sorted
+ * ids, input pairs, residual CSR, transposed HAG, transposed input graph).
+ * Host only; the input arrays are read during the call and not kept.
+ * Errors: HAG_ERR_NULL; HAG_ERR_ARG (n < 0, capacity < 0, n + capacity or |E| >=
+ * 2^31); HAG_ERR_GRAPH; HAG_ERR_OOM_HOST.  On error *out is NULL. */
+hag_status hag_build(int32_t n, const int64_t *row_ptr, const int32_t *col_idx, int32_t capacity, hag_t **out);
+
+/* Frees host and device arrays.  NULL is allowed. */
+hag_status hag_destroy(hag_t *h);
+
+/* Counters of Section 4.1 / Section 5.3 for this HAG. */
+hag_status hag_get_info(const hag_t *h, hag_info *out);
+
+/* Borrowed host pointers to the canonical arrays (for checking and export). */
+hag_status hag_export(const hag_t *h, hag_arrays *out);
+
+/* Copies the structure arrays to CUDA device `device` (idempotent for the same
+ * device; HAG_ERR_ARG if already on another one).  Synchronous.  Allocates with
+ * cudaMalloc; HAG_ERR_OOM_DEVICE / HAG_ERR_CUDA on failure. */
+hag_status hag_to_device(hag_t *h, int device);
+
+/* Bytes of workspace the aggregate calls need for feature width D:
+ * |V_A| * D * 4 (fp32 rows whatever the dtype); 0 when the HAG has no
+ * aggregation node or on bad arguments. */
+size_t hag_workspace_bytes(const hag_t *h, int32_t D);
+
+/* Algorithm 2 (the paper's hag_aggregate), one layer:
+ *   a-hat_w = a-hat_in0(w) + a-hat_in1(w)  for aggregation nodes, level by level;
+ *   out_v   = sum over the residual in-neighbours of v of a-hat  (x_u for graph nodes),
+ *   times 1/|N(v)| for HAG_MEAN (|N(v)| = in-degree in the input graph; an empty
+ *   neighbourhood gives a zero row).
+ * x and out are N x D of `dtype`, must not overlap; accumulation is fp32.
+ * Enqueues 1 + (number of level launches) kernels on the stream.
+ * Errors: NULL, ARG (D <= 0), DTYPE, ALIGN, WORKSPACE, NOT_ON_DEVICE, CUDA. */
+hag_status hag_aggregate_fwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D,
+                             const void *x, void *out, void *workspace, void *cuda_stream);
+
+/* Gradient of the above (the paper's hag_aggregate_grad; Section 3.2 requires the
+ * same gradients as the GNN-graph): grad_x = A^T (s * grad_out), s_v = 1 or
+ * 1/|N(v)|, computed without atomics by gathering over the transposed HAG --
+ * aggregation nodes from the last level to the first, then the input rows. */
+hag_status hag_aggregate_bwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D,
+                             const void *grad_out, void *grad_x, void *workspace, void *cuda_stream);
+
+/* The GNN-graph itself (Algorithm 1 line 4; V_A = {} in Section 3.1): the same
+ * gather kernel over the input CSR held by the handle, and over its transpose for
+ * the gradient.  No workspace. */
+hag_status csr_aggregate_fwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D,
+                             const void *x, void *out, void *cuda_stream);
+hag_status csr_aggregate_bwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D,
+                             const void *grad_out, void *grad_x, void *cuda_stream);
+
+/* Host-buffer variants for callers that keep features in host memory: x_host and
+ * out_host are HOST pointers to N x D matrices (pinned memory makes the copies
+ * asynchronous).  The call copies the input to device staging buffers owned by
+ * the handle (grown on demand with cudaMalloc), runs the aggregation on
+ * cuda_stream and copies the result back; it returns after enqueuing, so the
+ * caller synchronises the stream before reading out_host.  `backward` != 0 runs
+ * hag_aggregate_bwd instead of hag_aggregate_fwd; `use_hag` == 0 runs the
+ * csr_aggregate_* path. */
+hag_status hag_aggregate_host(hag_t *h, int backward, int use_hag, hag_reduce reduce, hag_dtype dtype, int32_t D,
+                              const void *in_host, void *out_host, void *cuda_stream);
+
+/* Number of kernels the last aggregate call on this handle enqueued. */
+int32_t hag_last_launch_count(const hag_t *h);
+
+const char *hag_status_str(hag_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HAG_B200_H */

@@ -1,0 +1,263 @@
+"""Python binding of the B200 HAG aggregation library.
+
+Thin argument marshalling over the C ABI declared in ``include/hag.h``: every
+step of the aggregation runs in the library's CUDA kernels.  PyTorch supplies
+device memory and streams only.  There is no CPU fallback: if the shared
+library is missing the first call raises.
+
+    h = Hag.build(row_ptr, col_idx, capacity)   # Algorithm 3 (host)
+    h.to_device(0)
+    out = h.aggregate_fwd(x, reduce="mean")     # Algorithm 2
+    gx = h.aggregate_bwd(grad_out, reduce="mean")
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libhag_b200.so")
+
+HAG_SUM, HAG_MEAN = 0, 1
+HAG_F32, HAG_BF16 = 0, 1
+
+EXPORTED_SYMBOLS = [
+    "hag_build", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes",
+    "hag_aggregate_fwd", "hag_aggregate_bwd", "csr_aggregate_fwd", "csr_aggregate_bwd",
+    "hag_aggregate_host", "hag_last_launch_count", "hag_status_str",
+]
+
+
+class HagError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        super().__init__(f"{what}: {status_str(status)} (status {status})")
+        self.status = status
+
+
+class HagInfo(ctypes.Structure):
+    _fields_ = [
+        ("n", ctypes.c_int32), ("capacity", ctypes.c_int32), ("num_agg", ctypes.c_int32),
+        ("num_levels", ctypes.c_int32), ("e", ctypes.c_int64), ("e_hat", ctypes.c_int64),
+        ("aggregations_gnn", ctypes.c_int64), ("aggregations_hag", ctypes.c_int64),
+        ("aggregations_hag_closed", ctypes.c_int64), ("saved", ctypes.c_int64),
+        ("first_redundancy", ctypes.c_int32), ("last_redundancy", ctypes.c_int32),
+        ("max_in_degree", ctypes.c_int32), ("max_res_degree", ctypes.c_int32),
+        ("max_out_degree", ctypes.c_int32), ("device", ctypes.c_int32),
+        ("build_seconds", ctypes.c_double),
+    ]
+
+    def as_dict(self) -> dict:
+        return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class HagArrays(ctypes.Structure):
+    _fields_ = [("n", ctypes.c_int32), ("num_agg", ctypes.c_int32), ("num_levels", ctypes.c_int32)] + [
+        (k, ctypes.c_void_p) for k in ("level_ptr", "agg_in", "res_ptr", "res_idx", "t_ptr", "t_idx", "in_degree",
+                                       "trace", "csr_t_ptr", "csr_t_idx")]
+
+
+_lib = None
+
+
+def load_library():
+    """Load the shared library (raises if it has not been built)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_1906_03707_b200.build` "
+                          "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32 = ctypes.c_void_p, ctypes.c_int32
+    lib.hag_build.argtypes = [i32, vp, vp, i32, ctypes.POINTER(vp)]
+    lib.hag_build.restype = ctypes.c_int
+    lib.hag_destroy.argtypes = [vp]
+    lib.hag_destroy.restype = ctypes.c_int
+    lib.hag_get_info.argtypes = [vp, ctypes.POINTER(HagInfo)]
+    lib.hag_get_info.restype = ctypes.c_int
+    lib.hag_export.argtypes = [vp, ctypes.POINTER(HagArrays)]
+    lib.hag_export.restype = ctypes.c_int
+    lib.hag_to_device.argtypes = [vp, ctypes.c_int]
+    lib.hag_to_device.restype = ctypes.c_int
+    lib.hag_workspace_bytes.argtypes = [vp, i32]
+    lib.hag_workspace_bytes.restype = ctypes.c_size_t
+    for name in ("hag_aggregate_fwd", "hag_aggregate_bwd"):
+        f = getattr(lib, name)
+        f.argtypes = [vp, ctypes.c_int, ctypes.c_int, i32, vp, vp, vp, vp]
+        f.restype = ctypes.c_int
+    for name in ("csr_aggregate_fwd", "csr_aggregate_bwd"):
+        f = getattr(lib, name)
+        f.argtypes = [vp, ctypes.c_int, ctypes.c_int, i32, vp, vp, vp]
+        f.restype = ctypes.c_int
+    lib.hag_aggregate_host.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, i32, vp, vp, vp]
+    lib.hag_aggregate_host.restype = ctypes.c_int
+    lib.hag_last_launch_count.argtypes = [vp]
+    lib.hag_last_launch_count.restype = i32
+    lib.hag_status_str.argtypes = [ctypes.c_int]
+    lib.hag_status_str.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def status_str(status: int) -> str:
+    return load_library().hag_status_str(int(status)).decode()
+
+
+def _check(status: int, what: str):
+    if status != 0:
+        raise HagError(status, what)
+
+
+def _reduce_code(reduce) -> int:
+    if reduce in ("sum", HAG_SUM):
+        return HAG_SUM
+    if reduce in ("mean", HAG_MEAN):
+        return HAG_MEAN
+    raise ValueError(f"reduce must be 'sum' or 'mean', got {reduce!r}")
+
+
+def _view(ptr, count, dtype):
+    if count == 0 or not ptr:
+        return np.zeros(0, dtype=dtype)
+    ctype = {np.int32: ctypes.c_int32, np.int64: ctypes.c_int64}[dtype]
+    return np.ctypeslib.as_array(ctypes.cast(ptr, ctypes.POINTER(ctype)), shape=(count,)).copy()
+
+
+class Hag:
+    """A built HAG: owns the library handle."""
+
+    def __init__(self, handle):
+        self._h = handle
+        self._ws = None
+
+    # -- construction ------------------------------------------------------- #
+    @classmethod
+    def build(cls, row_ptr, col_idx, capacity: int) -> "Hag":
+        """``hag_build``: CSR of in-neighbours on the host (int64 row_ptr, int32 col_idx)."""
+        lib = load_library()
+        rp = np.ascontiguousarray(row_ptr, dtype=np.int64)
+        ci = np.ascontiguousarray(col_idx, dtype=np.int32)
+        handle = ctypes.c_void_p()
+        n = rp.shape[0] - 1
+        st = lib.hag_build(n, rp.ctypes.data, ci.ctypes.data if ci.size else None, int(capacity), ctypes.byref(handle))
+        _check(st, "hag_build")
+        return cls(handle)
+
+    def close(self):
+        if self._h:
+            load_library().hag_destroy(self._h)
+            self._h = None
+            self._ws = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- inspection --------------------------------------------------------- #
+    def info(self) -> dict:
+        out = HagInfo()
+        _check(load_library().hag_get_info(self._h, ctypes.byref(out)), "hag_get_info")
+        return out.as_dict()
+
+    def arrays(self) -> dict:
+        """Copies of the canonical host arrays (``hag_export``)."""
+        a = HagArrays()
+        _check(load_library().hag_export(self._h, ctypes.byref(a)), "hag_export")
+        n, k, lv = a.n, a.num_agg, a.num_levels
+        res_ptr = _view(a.res_ptr, n + 1, np.int64)
+        t_ptr = _view(a.t_ptr, n + k + 1, np.int64)
+        csr_t_ptr = _view(a.csr_t_ptr, n + 1, np.int64)
+        return dict(
+            n=n, num_agg=k, num_levels=lv,
+            level_ptr=_view(a.level_ptr, lv + 1, np.int64),
+            agg_in=_view(a.agg_in, 2 * k, np.int32),
+            res_ptr=res_ptr, res_idx=_view(a.res_idx, int(res_ptr[-1]) if n >= 0 and res_ptr.size else 0, np.int32),
+            t_ptr=t_ptr, t_idx=_view(a.t_idx, int(t_ptr[-1]) if t_ptr.size else 0, np.int32),
+            in_degree=_view(a.in_degree, n, np.int32),
+            trace=_view(a.trace, 3 * k, np.int32).reshape(-1, 3),
+            csr_t_ptr=csr_t_ptr, csr_t_idx=_view(a.csr_t_idx, int(csr_t_ptr[-1]) if csr_t_ptr.size else 0, np.int32),
+        )
+
+    def workspace_bytes(self, d: int) -> int:
+        return int(load_library().hag_workspace_bytes(self._h, int(d)))
+
+    @property
+    def last_launch_count(self) -> int:
+        return int(load_library().hag_last_launch_count(self._h))
+
+    # -- device ------------------------------------------------------------- #
+    def to_device(self, device: int = 0) -> "Hag":
+        _check(load_library().hag_to_device(self._h, int(device)), "hag_to_device")
+        self._device = int(device)
+        return self
+
+    def _workspace(self, d: int, device):
+        import torch
+        need = self.workspace_bytes(d)
+        if need == 0:
+            return None
+        if self._ws is None or self._ws.numel() * 4 < need or self._ws.device != device:
+            self._ws = torch.empty(need // 4, dtype=torch.float32, device=device)
+        return self._ws
+
+    @staticmethod
+    def _dtype_code(t) -> int:
+        import torch
+        if t.dtype == torch.float32:
+            return HAG_F32
+        if t.dtype == torch.bfloat16:
+            return HAG_BF16
+        raise TypeError(f"features must be float32 or bfloat16, got {t.dtype}")
+
+    def _run(self, name, use_hag, inp, reduce, out, workspace):
+        import torch
+        if not inp.is_cuda or inp.dim() != 2 or not inp.is_contiguous():
+            raise ValueError("features must be a contiguous 2-D CUDA tensor")
+        if out is None:
+            out = torch.empty_like(inp)
+        elif out.shape != inp.shape or out.dtype != inp.dtype or not out.is_contiguous() or out.device != inp.device:
+            raise ValueError("out must match the input's shape, dtype and device")
+        d = inp.shape[1]
+        stream = torch.cuda.current_stream(inp.device).cuda_stream
+        lib = load_library()
+        code = self._dtype_code(inp)
+        if use_hag:
+            ws = workspace if workspace is not None else self._workspace(d, inp.device)
+            st = getattr(lib, name)(self._h, _reduce_code(reduce), code, d, inp.data_ptr(), out.data_ptr(),
+                                    ws.data_ptr() if ws is not None else None, stream)
+        else:
+            st = getattr(lib, name)(self._h, _reduce_code(reduce), code, d, inp.data_ptr(), out.data_ptr(), stream)
+        _check(st, name)
+        return out
+
+    def aggregate_fwd(self, x, reduce="sum", out=None, workspace=None):
+        """``hag_aggregate_fwd`` on the current stream."""
+        return self._run("hag_aggregate_fwd", True, x, reduce, out, workspace)
+
+    def aggregate_bwd(self, grad_out, reduce="sum", out=None, workspace=None):
+        """``hag_aggregate_bwd`` on the current stream."""
+        return self._run("hag_aggregate_bwd", True, grad_out, reduce, out, workspace)
+
+    def csr_fwd(self, x, reduce="sum", out=None):
+        """``csr_aggregate_fwd``: the plain GNN-graph, same kernel."""
+        return self._run("csr_aggregate_fwd", False, x, reduce, out, None)
+
+    def csr_bwd(self, grad_out, reduce="sum", out=None):
+        """``csr_aggregate_bwd``."""
+        return self._run("csr_aggregate_bwd", False, grad_out, reduce, out, None)
+
+    def aggregate_host(self, inp, out, reduce="sum", backward=False, use_hag=True, stream=None):
+        """``hag_aggregate_host``: host tensors in and out (pinned for async copies);
+        enqueues copy-in, aggregation and copy-out on the stream; the caller synchronises."""
+        import torch
+        if inp.is_cuda or out.is_cuda or inp.shape != out.shape or inp.dtype != out.dtype:
+            raise ValueError("aggregate_host takes matching host tensors")
+        s = torch.cuda.current_stream().cuda_stream if stream is None else stream
+        st = load_library().hag_aggregate_host(self._h, int(backward), int(use_hag), _reduce_code(reduce),
+                                               self._dtype_code(inp), inp.shape[1], inp.data_ptr(), out.data_ptr(), s)
+        _check(st, "hag_aggregate_host")
+        return out

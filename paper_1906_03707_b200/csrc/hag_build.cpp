@@ -1,0 +1,401 @@
+// hag_build: the HAG search of Algorithm 3 (set Aggregate) and the device layout.
+//
+// The search is exact: every iteration merges the pair with the largest
+// Redundancy (number of graph nodes aggregating both), ties to the smallest
+// (v1, v2).  Instead of a count per pair (billions at the larger shapes) it
+// keeps, per node x, key[x] >= max_b Redundancy(x, b) together with a partner
+// and a "dirty" flag:
+//   * a merge of (v1, v2) with users U changes only pairs that contain v1 or v2
+//     (they lose |U n out(y)|) and creates pairs (y, w) with count |U n out(y)|,
+//     which never exceeds the old count of (y, v1).  So no key ever has to rise,
+//     a node whose recorded partner is neither v1 nor v2 keeps an exact key, and
+//     the new node's key is known exactly from the same pass;
+//   * nodes whose partner was merged away are only marked dirty; their key stays
+//     a valid upper bound and is recounted when it reaches the top of the queue.
+// The queue is ordered by (key descending, id ascending); a clean top is the
+// arg-max with the required tie-break (its partner is the smallest id attaining
+// the count, and is larger than the node itself, otherwise the partner would
+// have been on top).  Memory is O(|E|).
+#include <algorithm>
+#include <chrono>
+#include <cstring>
+#include <new>
+#include <queue>
+
+#include "hag_internal.h"
+
+namespace {
+
+struct Searcher {
+    int32_t n;
+    int64_t cap;
+    const int64_t *row_ptr;
+    std::vector<int32_t> &rows;      // row u: rows[row_ptr[u] .. row_ptr[u] + row_len[u])
+    std::vector<int32_t> &row_len;
+    std::vector<int32_t> out_store;  // users of the graph nodes, grouped by source
+    std::vector<int32_t *> out_ptr;  // per id
+    std::vector<int32_t> out_len;
+    std::vector<std::vector<int32_t>> out_new;  // storage for aggregation nodes' user lists
+    std::vector<int32_t> key, partner;
+    std::vector<uint8_t> dirty;
+    std::vector<int32_t> cnt, touched, users;
+    std::priority_queue<uint64_t> pq;
+
+    Searcher(int32_t n_, int64_t cap_, const int64_t *rp, std::vector<int32_t> &r, std::vector<int32_t> &rl)
+        : n(n_), cap(cap_), row_ptr(rp), rows(r), row_len(rl) {}
+
+    static uint64_t enc(int32_t k, int32_t id) { return (uint64_t(uint32_t(k)) << 32) | uint32_t(0x7fffffff - id); }
+
+    // exact max_b Redundancy(x, b) and the smallest b attaining it
+    void recount(int32_t x, int32_t &best, int32_t &arg) {
+        touched.clear();
+        const int32_t *ou = out_ptr[x];
+        for (int32_t i = 0, m = out_len[x]; i < m; ++i) {
+            const int32_t u = ou[i];
+            const int32_t *row = rows.data() + row_ptr[u];
+            for (int32_t j = 0, l = row_len[u]; j < l; ++j) {
+                const int32_t y = row[j];
+                if (cnt[y]++ == 0) touched.push_back(y);
+            }
+        }
+        best = 0;
+        arg = -1;
+        for (int32_t y : touched) {
+            const int32_t c = cnt[y];
+            cnt[y] = 0;
+            if (y == x) continue;
+            if (c > best || (c == best && y < arg)) { best = c; arg = y; }
+        }
+    }
+
+    hag_status run(std::vector<int32_t> &trace) {
+        const int64_t n_ids = int64_t(n) + cap;
+        const int64_t e = row_ptr[n];
+        out_ptr.assign(n_ids, nullptr);
+        out_len.assign(n_ids, 0);
+        key.assign(n_ids, 0);
+        partner.assign(n_ids, -1);
+        dirty.assign(n_ids, 0);
+        cnt.assign(n_ids, 0);
+        out_new.resize(cap);
+        out_store.resize(e > 0 ? e : 1);
+        users.reserve(1024);
+        {   // users of every graph node as a source: transpose of the rows
+            std::vector<int64_t> off(n + 1, 0);
+            for (int64_t i = 0; i < e; ++i) off[rows[i] + 1]++;
+            for (int32_t s = 0; s < n; ++s) off[s + 1] += off[s];
+            for (int32_t s = 0; s < n; ++s) out_ptr[s] = out_store.data() + off[s];
+            for (int32_t u = 0; u < n; ++u)
+                for (int64_t i = row_ptr[u]; i < row_ptr[u + 1]; ++i) {
+                    const int32_t s = rows[i];
+                    out_ptr[s][out_len[s]++] = u;
+                }
+        }
+        // a pair cannot be shared by more rows than either member has users
+        for (int32_t s = 0; s < n; ++s) {
+            key[s] = out_len[s];
+            dirty[s] = 1;
+            if (key[s] >= 2) pq.push(enc(key[s], s));
+        }
+        int64_t num = 0;
+        while (num < cap && !pq.empty()) {
+            const uint64_t top = pq.top();
+            pq.pop();
+            const int32_t k = int32_t(top >> 32);
+            const int32_t x = int32_t(0x7fffffff - uint32_t(top & 0xffffffffu));
+            if (k != key[x]) continue;              // superseded entry
+            if (k < 2) break;
+            if (dirty[x]) {
+                int32_t m, p;
+                recount(x, m, p);
+                key[x] = m;
+                partner[x] = p;
+                dirty[x] = 0;
+                if (m >= 2) pq.push(enc(m, x));
+                continue;
+            }
+            const int32_t p = partner[x];
+            if (p <= x) return HAG_ERR_ARG;         // cannot happen (see header comment)
+            // users of the pair
+            users.clear();
+            {
+                const int32_t *a = out_ptr[x], *b = out_ptr[p];
+                int32_t i = 0, j = 0;
+                const int32_t la = out_len[x], lb = out_len[p];
+                while (i < la && j < lb) {
+                    if (a[i] < b[j]) ++i;
+                    else if (a[i] > b[j]) ++j;
+                    else { users.push_back(a[i]); ++i; ++j; }
+                }
+            }
+            if (int32_t(users.size()) != k) return HAG_ERR_ARG;  // internal inconsistency
+            const int32_t w = int32_t(n + num);
+            trace.push_back(x);
+            trace.push_back(p);
+            trace.push_back(k);
+            // rewrite the users' rows; count what else they hold (= the new node's pair counts)
+            touched.clear();
+            for (int32_t u : users) {
+                int32_t *row = rows.data() + row_ptr[u];
+                const int32_t l = row_len[u];
+                int32_t o = 0;
+                for (int32_t j = 0; j < l; ++j) {
+                    const int32_t y = row[j];
+                    if (y == x || y == p) continue;
+                    row[o++] = y;
+                    if (cnt[y]++ == 0) touched.push_back(y);
+                }
+                row[o++] = w;                       // larger than every existing id: row stays sorted
+                row_len[u] = o;
+            }
+            int32_t wbest = 0, warg = -1;
+            for (int32_t y : touched) {
+                const int32_t c = cnt[y];
+                cnt[y] = 0;
+                if (c > wbest || (c == wbest && y < warg)) { wbest = c; warg = y; }
+                if (!dirty[y] && (partner[y] == x || partner[y] == p)) dirty[y] = 1;
+            }
+            // user lists: x and p lose U, w gets it
+            for (int32_t s : {x, p}) {
+                int32_t *l = out_ptr[s];
+                const int32_t len = out_len[s];
+                int32_t o = 0;
+                size_t q = 0;
+                for (int32_t i = 0; i < len; ++i) {
+                    while (q < users.size() && users[q] < l[i]) ++q;
+                    if (q < users.size() && users[q] == l[i]) continue;
+                    l[o++] = l[i];
+                }
+                out_len[s] = o;
+                dirty[s] = 1;                        // every pair with x or p changed
+                const int32_t bound = std::min(key[s], o);
+                // x's entry was popped; p still has one unless its bound moved
+                if ((s == x || bound != key[s]) && bound >= 2) pq.push(enc(bound, s));
+                key[s] = bound;
+            }
+            out_new[num] = users;
+            out_ptr[w] = out_new[num].data();
+            out_len[w] = int32_t(users.size());
+            key[w] = wbest;
+            partner[w] = warg;
+            dirty[w] = 0;
+            if (wbest >= 2) pq.push(enc(wbest, w));
+            ++num;
+        }
+        return HAG_OK;
+    }
+};
+
+}  // namespace
+
+hag_status hag_search(hag *h, std::vector<int32_t> &rows_store, std::vector<int32_t> &rows_len) {
+    try {
+        rows_store = h->csr_idx;
+        rows_len.resize(h->n);
+        for (int32_t u = 0; u < h->n; ++u) rows_len[u] = int32_t(h->csr_ptr[u + 1] - h->csr_ptr[u]);
+        h->trace.clear();
+        if (h->capacity == 0 || h->n == 0) return HAG_OK;
+        Searcher s(h->n, h->capacity, h->csr_ptr.data(), rows_store, rows_len);
+        hag_status st = s.run(h->trace);
+        if (st != HAG_OK) return st;
+    } catch (const std::bad_alloc &) {
+        return HAG_ERR_OOM_HOST;
+    }
+    h->num_agg = int32_t(h->trace.size() / 3);
+    return HAG_OK;
+}
+
+hag_status hag_layout(hag *h, const std::vector<int32_t> &rows_store, const std::vector<int32_t> &rows_len) {
+    try {
+        const int32_t n = h->n, k = h->num_agg;
+        // level = 1 + the larger level of the two inputs (graph nodes are level 0)
+        std::vector<int32_t> level(size_t(n) + k, 0);
+        int32_t max_level = 0;
+        for (int32_t j = 0; j < k; ++j) {
+            const int32_t l = 1 + std::max(level[h->trace[3 * j]], level[h->trace[3 * j + 1]]);
+            level[n + j] = l;
+            max_level = std::max(max_level, l);
+        }
+        h->num_levels = max_level;
+        h->level_ptr.assign(size_t(max_level) + 1, 0);
+        for (int32_t j = 0; j < k; ++j) h->level_ptr[level[n + j]]++;
+        // level_ptr[l] currently holds the size of level l (l >= 1); make it a running end
+        for (int32_t l = 1; l <= max_level; ++l) h->level_ptr[l] += h->level_ptr[l - 1];
+        // stable placement by (level, creation index)
+        std::vector<int64_t> next(size_t(max_level) + 1, 0);
+        for (int32_t l = 1; l <= max_level; ++l) next[l] = h->level_ptr[l - 1];
+        std::vector<int32_t> canon(size_t(n) + k);
+        for (int32_t v = 0; v < n; ++v) canon[v] = v;
+        for (int32_t j = 0; j < k; ++j) canon[n + j] = int32_t(n + next[level[n + j]]++);
+        h->agg_in.assign(size_t(2) * k, 0);
+        for (int32_t j = 0; j < k; ++j) {
+            const int32_t a = canon[h->trace[3 * j]], b = canon[h->trace[3 * j + 1]];
+            const int32_t pos = canon[n + j] - n;
+            h->agg_in[2 * pos] = std::min(a, b);
+            h->agg_in[2 * pos + 1] = std::max(a, b);
+        }
+        // residual CSR in canonical ids, every row ascending
+        h->res_ptr.assign(size_t(n) + 1, 0);
+        for (int32_t v = 0; v < n; ++v) h->res_ptr[v + 1] = h->res_ptr[v] + rows_len[v];
+        h->e_res = h->res_ptr[n];
+        h->res_idx.resize(h->e_res);
+        int32_t max_res = 0;
+        for (int32_t v = 0; v < n; ++v) {
+            const int32_t *src = rows_store.data() + h->csr_ptr[v];
+            int32_t *dst = h->res_idx.data() + h->res_ptr[v];
+            for (int32_t j = 0; j < rows_len[v]; ++j) dst[j] = canon[src[j]];
+            std::sort(dst, dst + rows_len[v]);
+            max_res = std::max(max_res, rows_len[v]);
+        }
+        h->e_hat = h->e_res + 2 * int64_t(k);
+        // transposed HAG by counting sort; destinations come out ascending because
+        // graph-node rows are visited first in id order, then aggregation nodes in id order
+        const size_t n_src = size_t(n) + k;
+        h->t_ptr.assign(n_src + 1, 0);
+        for (int64_t i = 0; i < h->e_res; ++i) h->t_ptr[h->res_idx[i] + 1]++;
+        for (int64_t i = 0; i < 2 * int64_t(k); ++i) h->t_ptr[h->agg_in[i] + 1]++;
+        int64_t max_out = 0;
+        for (size_t s = 0; s < n_src; ++s) {
+            max_out = std::max(max_out, h->t_ptr[s + 1]);
+            h->t_ptr[s + 1] += h->t_ptr[s];
+        }
+        h->t_idx.resize(h->e_hat);
+        {
+            std::vector<int64_t> fill(h->t_ptr.begin(), h->t_ptr.end() - 1);
+            for (int32_t v = 0; v < n; ++v)
+                for (int64_t i = h->res_ptr[v]; i < h->res_ptr[v + 1]; ++i) h->t_idx[fill[h->res_idx[i]]++] = v;
+            for (int32_t j = 0; j < k; ++j) {
+                h->t_idx[fill[h->agg_in[2 * j]]++] = n + j;
+                h->t_idx[fill[h->agg_in[2 * j + 1]]++] = n + j;
+            }
+        }
+        // transposed input graph, same method
+        h->csr_t_ptr.assign(size_t(n) + 1, 0);
+        for (int64_t i = 0; i < h->e; ++i) h->csr_t_ptr[h->csr_idx[i] + 1]++;
+        for (int32_t s = 0; s < n; ++s) h->csr_t_ptr[s + 1] += h->csr_t_ptr[s];
+        h->csr_t_idx.resize(h->e);
+        {
+            std::vector<int64_t> fill(h->csr_t_ptr.begin(), h->csr_t_ptr.end() - 1);
+            for (int32_t v = 0; v < n; ++v)
+                for (int64_t i = h->csr_ptr[v]; i < h->csr_ptr[v + 1]; ++i) h->csr_t_idx[fill[h->csr_idx[i]]++] = v;
+        }
+        // counters of the cost function
+        hag_info &f = h->info;
+        f = hag_info{};
+        f.n = n;
+        f.capacity = h->capacity;
+        f.num_agg = k;
+        f.num_levels = max_level;
+        f.e = h->e;
+        f.e_hat = h->e_hat;
+        int32_t max_in = 0;
+        for (int32_t v = 0; v < n; ++v) {
+            const int32_t deg = h->in_degree[v];
+            max_in = std::max(max_in, deg);
+            f.aggregations_gnn += std::max(deg - 1, 0);
+            f.aggregations_hag += std::max(rows_len[v] - 1, 0);
+        }
+        f.aggregations_hag += k;  // two in-edges each: one binary aggregation
+        f.aggregations_hag_closed = h->e_hat - n - k;
+        for (int32_t j = 0; j < k; ++j) f.saved += h->trace[3 * j + 2] - 1;
+        f.first_redundancy = k ? h->trace[2] : 0;
+        f.last_redundancy = k ? h->trace[3 * (k - 1) + 2] : 0;
+        f.max_in_degree = max_in;
+        f.max_res_degree = max_res;
+        f.max_out_degree = int32_t(max_out);
+        f.device = -1;
+    } catch (const std::bad_alloc &) {
+        return HAG_ERR_OOM_HOST;
+    }
+    return HAG_OK;
+}
+
+extern "C" hag_status hag_build(int32_t n, const int64_t *row_ptr, const int32_t *col_idx, int32_t capacity, hag_t **out) {
+    if (!out) return HAG_ERR_NULL;
+    *out = nullptr;
+    if (!row_ptr || (!col_idx && n > 0 && row_ptr[n] > 0)) return HAG_ERR_NULL;
+    if (n < 0 || capacity < 0) return HAG_ERR_ARG;
+    if (int64_t(n) + int64_t(capacity) >= (int64_t(1) << 31)) return HAG_ERR_ARG;
+    // validate the CSR before anything reads through it
+    if (row_ptr[0] != 0) return HAG_ERR_GRAPH;
+    for (int32_t v = 0; v < n; ++v)
+        if (row_ptr[v + 1] < row_ptr[v]) return HAG_ERR_GRAPH;
+    const int64_t e = row_ptr[n];
+    if (e >= (int64_t(1) << 31)) return HAG_ERR_ARG;
+    for (int32_t v = 0; v < n; ++v) {
+        int64_t prev = -1;
+        for (int64_t i = row_ptr[v]; i < row_ptr[v + 1]; ++i) {
+            const int64_t c = col_idx[i];
+            if (c < 0 || c >= n || c <= prev) return HAG_ERR_GRAPH;
+            prev = c;
+        }
+    }
+    const auto t0 = std::chrono::steady_clock::now();
+    hag *h = new (std::nothrow) hag();
+    if (!h) return HAG_ERR_OOM_HOST;
+    hag_status st = HAG_OK;
+    try {
+        h->n = n;
+        h->capacity = capacity;
+        h->e = e;
+        h->csr_ptr.assign(row_ptr, row_ptr + n + 1);
+        h->csr_idx.assign(col_idx, col_idx + e);
+        h->in_degree.resize(n);
+        for (int32_t v = 0; v < n; ++v) h->in_degree[v] = int32_t(row_ptr[v + 1] - row_ptr[v]);
+        std::vector<int32_t> rows_store, rows_len;
+        st = hag_search(h, rows_store, rows_len);
+        if (st == HAG_OK) st = hag_layout(h, rows_store, rows_len);
+    } catch (const std::bad_alloc &) {
+        st = HAG_ERR_OOM_HOST;
+    }
+    if (st != HAG_OK) {
+        delete h;
+        return st;
+    }
+    h->info.build_seconds = std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count();
+    *out = h;
+    return HAG_OK;
+}
+
+extern "C" hag_status hag_get_info(const hag_t *h, hag_info *out) {
+    if (!h || !out) return HAG_ERR_NULL;
+    *out = h->info;
+    out->device = h->device;
+    return HAG_OK;
+}
+
+extern "C" hag_status hag_export(const hag_t *h, hag_arrays *out) {
+    if (!h || !out) return HAG_ERR_NULL;
+    out->n = h->n;
+    out->num_agg = h->num_agg;
+    out->num_levels = h->num_levels;
+    out->level_ptr = h->level_ptr.data();
+    out->agg_in = h->agg_in.data();
+    out->res_ptr = h->res_ptr.data();
+    out->res_idx = h->res_idx.data();
+    out->t_ptr = h->t_ptr.data();
+    out->t_idx = h->t_idx.data();
+    out->in_degree = h->in_degree.data();
+    out->trace = h->trace.data();
+    out->csr_t_ptr = h->csr_t_ptr.data();
+    out->csr_t_idx = h->csr_t_idx.data();
+    return HAG_OK;
+}
+
+extern "C" const char *hag_status_str(hag_status s) {
+    switch (s) {
+        case HAG_OK: return "ok";
+        case HAG_ERR_NULL: return "null pointer";
+        case HAG_ERR_ARG: return "argument out of range";
+        case HAG_ERR_GRAPH: return "malformed graph (rows must be strictly ascending, ids in range)";
+        case HAG_ERR_OOM_HOST: return "out of host memory";
+        case HAG_ERR_OOM_DEVICE: return "out of device memory";
+        case HAG_ERR_CUDA: return "CUDA runtime error";
+        case HAG_ERR_DTYPE: return "unsupported dtype";
+        case HAG_ERR_ALIGN: return "pointer or row size not 16-byte aligned";
+        case HAG_ERR_WORKSPACE: return "workspace required but missing";
+        case HAG_ERR_TIMEOUT: return "device-side wait timed out";
+        case HAG_ERR_NOT_ON_DEVICE: return "structure not on a device (call hag_to_device)";
+    }
+    return "unknown status";
+}

@@ -1,0 +1,339 @@
+// Device side of the C ABI: upload of the structure arrays and the launch
+// sequences of the forward / backward aggregation (Algorithm 2 and its adjoint).
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdint>
+#include <limits>
+#include <new>
+#include <vector>
+
+#include "hag_internal.h"
+#include "hag_kernels.cuh"
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+template <typename V>
+hag_status upload_i32(int32_t **dst, const V *src, size_t count) {
+    std::vector<int32_t> tmp;
+    try {
+        tmp.resize(std::max<size_t>(count, 1));
+    } catch (const std::bad_alloc &) {
+        return HAG_ERR_OOM_HOST;
+    }
+    for (size_t i = 0; i < count; ++i) tmp[i] = int32_t(src[i]);
+    cudaError_t err = cudaMalloc(reinterpret_cast<void **>(dst), tmp.size() * sizeof(int32_t));
+    if (err == cudaErrorMemoryAllocation) { cudaGetLastError(); return HAG_ERR_OOM_DEVICE; }
+    if (err != cudaSuccess) { cudaGetLastError(); return HAG_ERR_CUDA; }
+    if (cudaMemcpy(*dst, tmp.data(), tmp.size() * sizeof(int32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaGetLastError();
+        return HAG_ERR_CUDA;
+    }
+    return HAG_OK;
+}
+
+void free_device(hag *h) {
+    hag_device_arrays &d = h->d;
+    void *ptrs[] = {d.agg_in, d.res_ptr, d.res_idx, d.t_ptr, d.t_idx, d.csr_ptr, d.csr_idx, d.csr_t_ptr,
+                    d.csr_t_idx, d.inv_degree, d.stage_in, d.stage_out, d.stage_ws};
+    for (void *p : ptrs)
+        if (p) cudaFree(p);
+    d = hag_device_arrays{};
+}
+
+int lanes_per_row(int n_chunks) {
+    int l = 4;
+    while (l < 32 && l < n_chunks) l *= 2;
+    return l;
+}
+
+template <typename T>
+cudaError_t launch_gather(const hagk::GatherArgs &a, int n_chunks, cudaStream_t s) {
+    if (a.row_count <= 0) return cudaSuccess;
+    const int lpr = lanes_per_row(n_chunks);
+    const int rows_per_cta = hagk::kWarps * (32 / lpr);
+    const unsigned grid = unsigned((a.row_count + rows_per_cta - 1) / rows_per_cta);
+    switch (lpr) {
+        case 4: hagk::gather_sum_kernel<T, 4><<<grid, hagk::kThreads, 0, s>>>(a); break;
+        case 8: hagk::gather_sum_kernel<T, 8><<<grid, hagk::kThreads, 0, s>>>(a); break;
+        case 16: hagk::gather_sum_kernel<T, 16><<<grid, hagk::kThreads, 0, s>>>(a); break;
+        default: hagk::gather_sum_kernel<T, 32><<<grid, hagk::kThreads, 0, s>>>(a); break;
+    }
+    return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t launch_pairs(const hagk::PairArgs &p, int n_chunks, cudaStream_t s) {
+    if (p.count <= 0) return cudaSuccess;
+    const int lpr = lanes_per_row(n_chunks);
+    const int rows_per_cta = hagk::kWarps * (32 / lpr);
+    const unsigned grid = unsigned((p.count + rows_per_cta - 1) / rows_per_cta);
+    switch (lpr) {
+        case 4: hagk::pair_sum_kernel<T, 4><<<grid, hagk::kThreads, 0, s>>>(p); break;
+        case 8: hagk::pair_sum_kernel<T, 8><<<grid, hagk::kThreads, 0, s>>>(p); break;
+        case 16: hagk::pair_sum_kernel<T, 16><<<grid, hagk::kThreads, 0, s>>>(p); break;
+        default: hagk::pair_sum_kernel<T, 32><<<grid, hagk::kThreads, 0, s>>>(p); break;
+    }
+    return cudaGetLastError();
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+hag_status check_call(const hag *h, hag_dtype dtype, int32_t D, const void *in, const void *out) {
+    if (!h || !in || !out) return HAG_ERR_NULL;
+    if (dtype != HAG_F32 && dtype != HAG_BF16) return HAG_ERR_DTYPE;
+    if (D <= 0) return HAG_ERR_ARG;
+    const size_t elem = dtype == HAG_F32 ? 4 : 2;
+    if ((size_t(D) * elem) % 16 != 0 || !aligned16(in) || !aligned16(out)) return HAG_ERR_ALIGN;
+    if (h->device < 0) return HAG_ERR_NOT_ON_DEVICE;
+    if (in == out) return HAG_ERR_ARG;
+    return HAG_OK;
+}
+
+// Forward over the HAG: level launches (Algorithm 2 lines 5-6), then the gather (lines 7-8).
+template <typename T>
+hag_status fwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, const void *x, void *out, void *ws,
+                    cudaStream_t s, int32_t *launches) {
+    const int n_chunks = D / hagk::Chunk<T>::kElems;
+    const hag_device_arrays &d = h->d;
+    *launches = 0;
+    hagk::GatherArgs a{};
+    a.row_begin = 0;
+    a.row_count = h->n;
+    a.prim = x;
+    a.dst_scale = (reduce == HAG_MEAN) ? d.inv_degree : nullptr;
+    a.out = out;
+    a.D = D;
+    if (use_hag && h->num_agg > 0) {
+        for (int32_t l = 1; l <= h->num_levels; ++l) {
+            hagk::PairArgs p{};
+            p.agg_in = d.agg_in;
+            p.first = int32_t(h->level_ptr[l - 1]);
+            p.count = int32_t(h->level_ptr[l] - h->level_ptr[l - 1]);
+            p.x = x;
+            p.ahat = static_cast<float *>(ws);
+            p.n = h->n;
+            p.D = D;
+            if (launch_pairs<T>(p, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+            ++*launches;
+        }
+        a.row_ptr = d.res_ptr;
+        a.idx = d.res_idx;
+        a.sec = static_cast<const float *>(ws);
+        a.n_prim = h->n;
+    } else if (use_hag) {
+        a.row_ptr = d.res_ptr;
+        a.idx = d.res_idx;
+        a.n_prim = std::numeric_limits<int32_t>::max();
+    } else {
+        a.row_ptr = d.csr_ptr;
+        a.idx = d.csr_idx;
+        a.n_prim = std::numeric_limits<int32_t>::max();
+    }
+    if (launch_gather<T>(a, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+    if (h->n > 0) ++*launches;
+    return HAG_OK;
+}
+
+// Backward: gather over the transposed structure.  Aggregation nodes from the
+// last level to the first (their gradient rows live in the workspace), then the
+// graph nodes as sources.  A destination id < n stands for the output row of
+// that graph node (scaled by 1/|N| for mean), an id >= n for an aggregation node.
+template <typename T>
+hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, const void *g, void *gx, void *ws,
+                    cudaStream_t s, int32_t *launches) {
+    const int n_chunks = D / hagk::Chunk<T>::kElems;
+    const hag_device_arrays &d = h->d;
+    *launches = 0;
+    hagk::GatherArgs a{};
+    a.prim = g;
+    a.src_scale = (reduce == HAG_MEAN) ? d.inv_degree : nullptr;
+    a.D = D;
+    if (use_hag && h->num_agg > 0) {
+        a.row_ptr = d.t_ptr;
+        a.idx = d.t_idx;
+        a.sec = static_cast<const float *>(ws);
+        a.n_prim = h->n;
+        for (int32_t l = h->num_levels; l >= 1; --l) {
+            hagk::GatherArgs lv = a;
+            lv.row_begin = h->n + int32_t(h->level_ptr[l - 1]);
+            lv.row_count = int32_t(h->level_ptr[l] - h->level_ptr[l - 1]);
+            lv.out = ws;
+            lv.out_row_offset = h->n;
+            lv.out_is_f32 = 1;
+            if (launch_gather<T>(lv, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+            ++*launches;
+        }
+    } else if (use_hag) {
+        a.row_ptr = d.t_ptr;
+        a.idx = d.t_idx;
+        a.n_prim = std::numeric_limits<int32_t>::max();
+    } else {
+        a.row_ptr = d.csr_t_ptr;
+        a.idx = d.csr_t_idx;
+        a.n_prim = std::numeric_limits<int32_t>::max();
+    }
+    a.row_begin = 0;
+    a.row_count = h->n;
+    a.out = gx;
+    if (launch_gather<T>(a, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+    if (h->n > 0) ++*launches;
+    return HAG_OK;
+}
+
+hag_status run(const hag *h, bool backward, bool use_hag, hag_reduce reduce, hag_dtype dtype, int32_t D, const void *in,
+               void *out, void *ws, void *stream) {
+    hag_status st = check_call(h, dtype, D, in, out);
+    if (st != HAG_OK) return st;
+    if (reduce != HAG_SUM && reduce != HAG_MEAN) return HAG_ERR_ARG;
+    if (use_hag && h->num_agg > 0) {
+        if (!ws) return HAG_ERR_WORKSPACE;
+        if (!aligned16(ws)) return HAG_ERR_ALIGN;
+    }
+    DeviceGuard guard(h->device);
+    if (!guard.ok) { cudaGetLastError(); return HAG_ERR_CUDA; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int32_t launches = 0;
+    if (dtype == HAG_F32)
+        st = backward ? bwd_impl<float>(h, use_hag, reduce, D, in, out, ws, s, &launches)
+                      : fwd_impl<float>(h, use_hag, reduce, D, in, out, ws, s, &launches);
+    else
+        st = backward ? bwd_impl<__nv_bfloat16>(h, use_hag, reduce, D, in, out, ws, s, &launches)
+                      : fwd_impl<__nv_bfloat16>(h, use_hag, reduce, D, in, out, ws, s, &launches);
+    const_cast<hag *>(h)->last_launches = launches;
+    return st;
+}
+
+hag_status grow(void **buf, size_t *have, size_t need) {
+    if (*have >= need) return HAG_OK;
+    if (*buf) cudaFree(*buf);
+    *buf = nullptr;
+    *have = 0;
+    cudaError_t err = cudaMalloc(buf, need);
+    if (err == cudaErrorMemoryAllocation) { cudaGetLastError(); return HAG_ERR_OOM_DEVICE; }
+    if (err != cudaSuccess) { cudaGetLastError(); return HAG_ERR_CUDA; }
+    *have = need;
+    return HAG_OK;
+}
+
+}  // namespace
+
+extern "C" hag_status hag_destroy(hag_t *h) {
+    if (!h) return HAG_OK;
+    if (h->device >= 0) {
+        DeviceGuard guard(h->device);
+        if (guard.ok) free_device(h);
+    }
+    delete h;
+    return HAG_OK;
+}
+
+extern "C" hag_status hag_to_device(hag_t *h, int device) {
+    if (!h) return HAG_ERR_NULL;
+    if (device < 0) return HAG_ERR_ARG;
+    if (h->device == device) return HAG_OK;
+    if (h->device >= 0) return HAG_ERR_ARG;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess) { cudaGetLastError(); return HAG_ERR_CUDA; }
+    if (device >= count) return HAG_ERR_ARG;
+    DeviceGuard guard(device);
+    if (!guard.ok) { cudaGetLastError(); return HAG_ERR_CUDA; }
+    hag_device_arrays &d = h->d;
+    hag_status st = HAG_OK;
+    const size_t n = size_t(h->n), k = size_t(h->num_agg);
+    if (st == HAG_OK) st = upload_i32(&d.agg_in, h->agg_in.data(), 2 * k);
+    if (st == HAG_OK) st = upload_i32(&d.res_ptr, h->res_ptr.data(), n + 1);
+    if (st == HAG_OK) st = upload_i32(&d.res_idx, h->res_idx.data(), size_t(h->e_res));
+    if (st == HAG_OK) st = upload_i32(&d.t_ptr, h->t_ptr.data(), n + k + 1);
+    if (st == HAG_OK) st = upload_i32(&d.t_idx, h->t_idx.data(), size_t(h->e_hat));
+    if (st == HAG_OK) st = upload_i32(&d.csr_ptr, h->csr_ptr.data(), n + 1);
+    if (st == HAG_OK) st = upload_i32(&d.csr_idx, h->csr_idx.data(), size_t(h->e));
+    if (st == HAG_OK) st = upload_i32(&d.csr_t_ptr, h->csr_t_ptr.data(), n + 1);
+    if (st == HAG_OK) st = upload_i32(&d.csr_t_idx, h->csr_t_idx.data(), size_t(h->e));
+    if (st == HAG_OK) {
+        std::vector<float> inv(std::max<size_t>(n, 1), 1.0f);
+        for (size_t v = 0; v < n; ++v) inv[v] = h->in_degree[v] > 0 ? 1.0f / float(h->in_degree[v]) : 1.0f;
+        cudaError_t err = cudaMalloc(reinterpret_cast<void **>(&d.inv_degree), inv.size() * sizeof(float));
+        if (err != cudaSuccess) {
+            cudaGetLastError();
+            st = err == cudaErrorMemoryAllocation ? HAG_ERR_OOM_DEVICE : HAG_ERR_CUDA;
+        } else if (cudaMemcpy(d.inv_degree, inv.data(), inv.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaGetLastError();
+            st = HAG_ERR_CUDA;
+        }
+    }
+    if (st != HAG_OK) {
+        free_device(h);
+        return st;
+    }
+    h->device = device;
+    return HAG_OK;
+}
+
+extern "C" size_t hag_workspace_bytes(const hag_t *h, int32_t D) {
+    if (!h || D <= 0) return 0;
+    return size_t(h->num_agg) * size_t(D) * sizeof(float);
+}
+
+extern "C" hag_status hag_aggregate_fwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D, const void *x,
+                                        void *out, void *workspace, void *cuda_stream) {
+    return run(h, false, true, reduce, dtype, D, x, out, workspace, cuda_stream);
+}
+
+extern "C" hag_status hag_aggregate_bwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D,
+                                        const void *grad_out, void *grad_x, void *workspace, void *cuda_stream) {
+    return run(h, true, true, reduce, dtype, D, grad_out, grad_x, workspace, cuda_stream);
+}
+
+extern "C" hag_status csr_aggregate_fwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D, const void *x,
+                                        void *out, void *cuda_stream) {
+    return run(h, false, false, reduce, dtype, D, x, out, nullptr, cuda_stream);
+}
+
+extern "C" hag_status csr_aggregate_bwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D,
+                                        const void *grad_out, void *grad_x, void *cuda_stream) {
+    return run(h, true, false, reduce, dtype, D, grad_out, grad_x, nullptr, cuda_stream);
+}
+
+extern "C" hag_status hag_aggregate_host(hag_t *h, int backward, int use_hag, hag_reduce reduce, hag_dtype dtype,
+                                         int32_t D, const void *in_host, void *out_host, void *cuda_stream) {
+    if (!h || !in_host || !out_host) return HAG_ERR_NULL;
+    if (dtype != HAG_F32 && dtype != HAG_BF16) return HAG_ERR_DTYPE;
+    if (D <= 0) return HAG_ERR_ARG;
+    if (h->device < 0) return HAG_ERR_NOT_ON_DEVICE;
+    const size_t bytes = size_t(h->n) * size_t(D) * (dtype == HAG_F32 ? 4 : 2);
+    DeviceGuard guard(h->device);
+    if (!guard.ok) { cudaGetLastError(); return HAG_ERR_CUDA; }
+    hag_device_arrays &d = h->d;
+    hag_status st = grow(&d.stage_in, &d.stage_in_bytes, std::max<size_t>(bytes, 16));
+    if (st == HAG_OK) st = grow(&d.stage_out, &d.stage_out_bytes, std::max<size_t>(bytes, 16));
+    if (st == HAG_OK) st = grow(&d.stage_ws, &d.stage_ws_bytes, std::max<size_t>(hag_workspace_bytes(h, D), 16));
+    if (st != HAG_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (bytes && cudaMemcpyAsync(d.stage_in, in_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+        cudaGetLastError();
+        return HAG_ERR_CUDA;
+    }
+    st = run(h, backward != 0, use_hag != 0, reduce, dtype, D, d.stage_in, d.stage_out, d.stage_ws, cuda_stream);
+    if (st != HAG_OK) return st;
+    if (bytes && cudaMemcpyAsync(out_host, d.stage_out, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) {
+        cudaGetLastError();
+        return HAG_ERR_CUDA;
+    }
+    return HAG_OK;
+}
+
+extern "C" int32_t hag_last_launch_count(const hag_t *h) { return h ? h->last_launches : 0; }

@@ -1,0 +1,170 @@
+"""Host side of the library (no GPU): hag_build against the oracle, bit for bit;
+the C ABI's symbols; argument and graph validation."""
+import ctypes
+import json
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_1906_03707_b200 as hb
+from oracle import oracle as O
+from paper_1906_03707_b200 import synth
+from paper_1906_03707_b200.build import build as build_library
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _library():
+    build_library()
+    hb.load_library()
+
+
+def _same_structure(g, capacity, search=O.greedy_pairmap):
+    h = hb.Hag.build(g.row_ptr, g.col_idx, capacity)
+    arr = h.arrays()
+    res = search(g.row_ptr, g.col_idx, capacity)
+    ref = O.canonical_hag(g.row_ptr, res)
+    assert arr["trace"].tolist() == res.trace.tolist()
+    assert arr["num_agg"] == ref.num_agg and arr["num_levels"] == ref.num_levels
+    for key in ("level_ptr", "agg_in", "res_ptr", "res_idx", "t_ptr", "t_idx", "in_degree"):
+        got, want = arr[key], getattr(ref, key)
+        assert got.dtype == want.dtype and np.array_equal(got, want), key
+    t_ptr, t_idx = O.transposed_csr(g.row_ptr, g.col_idx)
+    assert np.array_equal(arr["csr_t_ptr"], t_ptr) and np.array_equal(arr["csr_t_idx"], t_idx)
+    info = h.info()
+    c = O.counters(g.row_ptr, ref)
+    assert info["n"] == g.n and info["e"] == c["e"] and info["e_hat"] == c["e_hat"]
+    assert info["num_agg"] == c["num_agg"] and info["num_levels"] == c["num_levels"]
+    assert info["aggregations_gnn"] == c["aggregations_gnn"]
+    assert info["aggregations_hag"] == c["aggregations_hag"]
+    assert info["aggregations_hag_closed"] == c["aggregations_hag_closed_form"]
+    assert info["saved"] == c["saved_f"]
+    assert info["device"] == -1
+    h.close()
+    return info
+
+
+def test_header_symbols_are_exported():
+    text = open(os.path.join(ROOT, "include", "hag.h")).read()
+    declared = set(re.findall(r"\b((?:hag|csr)_[a-z_]+)\s*\(", text))
+    assert declared == set(hb.EXPORTED_SYMBOLS)
+    lib = ctypes.CDLL(hb.LIB_PATH)
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+@pytest.mark.parametrize("name", ["k4_no_self_loops.json", "k4_self_loops.json", "renumbering_13.json"])
+def test_worked_examples(golden_dir, name):
+    gold = json.load(open(os.path.join(golden_dir, name)))
+    g = synth.csr_from_rows(gold["rows"])
+    h = hb.Hag.build(g.row_ptr, g.col_idx, gold["capacity"])
+    arr = h.arrays()
+    assert arr["trace"].tolist() == gold["trace"]
+    for key in ("level_ptr", "agg_in", "res_ptr", "res_idx", "t_ptr", "t_idx"):
+        if key in gold:
+            assert arr[key].tolist() == gold[key], key
+
+
+@pytest.mark.parametrize("seed", range(60))
+def test_every_merge_matches_brute_force(seed):
+    rng = np.random.default_rng(1000 + seed)
+    n = int(rng.integers(6, 36))
+    g = synth.random_digraph(500 + seed, n, float(rng.uniform(0.15, 0.6)), bool(seed % 2), bool((seed // 2) % 2))
+    for cap in (n // 4, 3 * n):
+        _same_structure(g, cap, search=O.greedy_bruteforce)
+
+
+@pytest.mark.parametrize("maker,cap_frac", [
+    (lambda: synth.workload(1).graph, 0.25),
+    (lambda: synth.config2_graph(seed=11, n=3000, n_comm=30), 0.25),
+    (lambda: synth.config2_graph(seed=11, n=3000, n_comm=30), 2.0),
+    (lambda: synth.config3_graph(seed=12, n=1800, n_comm=3, d_lo=10, d_hi=300), 0.25),
+    (lambda: synth.config4_graph(seed=13, n_graphs=20, graph_size=60), 0.25),
+    (lambda: synth.config5_graph(seed=14, n=4000, n_comm=12, s_lo=60, s_hi=900, d_lo=8, d_hi=150), 0.5),
+    (lambda: synth.clique_union_graph(seed=15, n=1500, n_groups=400, g_lo=3, g_hi=40), 0.25),
+    (lambda: synth.workload(1).graph, 0.0),
+])
+def test_structure_is_bit_exact_on_workload_shapes(maker, cap_frac):
+    g = maker()
+    info = _same_structure(g, int(g.n * cap_frac))
+    if cap_frac == 0.0:
+        assert info["num_agg"] == 0 and info["e_hat"] == info["e"]
+
+
+def test_stored_structure_hashes(golden_dir):
+    """Digests written by tests/golden/make_structure_hashes.py from the oracle alone."""
+    import hashlib
+    path = os.path.join(golden_dir, "structure_hashes.json")
+    if not os.path.exists(path):
+        pytest.skip("no stored digests")
+    stored = json.load(open(path))
+    checked = 0
+    for key, rec in stored["cases"].items():
+        if rec["host_seconds_hint"] > 30:
+            continue
+        w = synth.workload(rec["workload"], scale=rec["scale"])
+        h = hb.Hag.build(w.graph.row_ptr, w.graph.col_idx, rec["capacity"])
+        arr = h.arrays()
+        dig = hashlib.sha256()
+        for k in stored["array_order"]:
+            dig.update(np.ascontiguousarray(arr[k]).tobytes())
+        assert dig.hexdigest() == rec["sha256"], key
+        checked += 1
+    assert checked > 0
+
+
+def test_empty_and_degenerate_graphs():
+    # no nodes
+    h = hb.Hag.build(np.zeros(1, np.int64), np.zeros(0, np.int32), 4)
+    assert h.info()["n"] == 0 and h.info()["num_agg"] == 0
+    # nodes without edges
+    h = hb.Hag.build(np.zeros(6, np.int64), np.zeros(0, np.int32), 4)
+    arr = h.arrays()
+    assert arr["num_agg"] == 0 and arr["res_ptr"].tolist() == [0] * 6 and h.workspace_bytes(64) == 0
+    # capacity reached exactly, then workspace size
+    g = synth.csr_from_rows([list(range(8))] * 8)
+    h = hb.Hag.build(g.row_ptr, g.col_idx, 2)
+    assert h.info()["num_agg"] == 2 and h.workspace_bytes(64) == 2 * 64 * 4 and h.workspace_bytes(0) == 0
+
+
+def test_argument_and_graph_validation():
+    lib = hb.load_library()
+    rp = np.asarray([0, 2, 3], dtype=np.int64)
+    handle = ctypes.c_void_p()
+
+    def build(n, rp_, ci_, cap):
+        return lib.hag_build(n, rp_.ctypes.data if rp_ is not None else None,
+                             ci_.ctypes.data if ci_ is not None else None, cap, ctypes.byref(handle))
+
+    ok = np.asarray([0, 1, 0], dtype=np.int32)
+    assert build(2, rp, ok, 1) == 0
+    lib.hag_destroy(handle)
+    assert build(2, None, ok, 1) == 1                                           # NULL
+    assert lib.hag_build(2, rp.ctypes.data, ok.ctypes.data, 1, None) == 1       # NULL out
+    assert build(-1, rp, ok, 1) == 2 and build(2, rp, ok, -1) == 2              # ARG
+    assert build(2, rp, ok, 2 ** 31 - 2) == 2                                   # n + capacity overflow
+    assert build(2, rp, np.asarray([1, 0, 0], dtype=np.int32), 1) == 3          # unsorted row
+    assert build(2, rp, np.asarray([1, 1, 0], dtype=np.int32), 1) == 3          # duplicate
+    assert build(2, rp, np.asarray([0, 2, 0], dtype=np.int32), 1) == 3          # out of range
+    assert build(2, rp, np.asarray([0, -1, 0], dtype=np.int32), 1) == 3
+    assert build(2, np.asarray([0, 3, 2], dtype=np.int64), ok, 1) == 3          # decreasing row_ptr
+    assert build(2, np.asarray([1, 2, 3], dtype=np.int64), ok, 1) == 3          # row_ptr[0] != 0
+    assert handle.value is None
+    # calls on a host-only handle fail with a status, not a crash
+    h = hb.Hag.build(rp, ok, 1)
+    dummy = ctypes.c_void_p(4096)
+    assert lib.hag_aggregate_fwd(h._h, 0, 0, 64, dummy, ctypes.c_void_p(8192), None, None) == 11   # not on device
+    assert lib.hag_aggregate_fwd(h._h, 0, 0, 6, dummy, ctypes.c_void_p(8192), None, None) == 8     # row bytes % 16
+    assert lib.hag_aggregate_fwd(h._h, 0, 0, 64, ctypes.c_void_p(4100), ctypes.c_void_p(8192), None, None) == 8
+    assert lib.hag_aggregate_fwd(h._h, 0, 5, 64, dummy, ctypes.c_void_p(8192), None, None) == 7    # dtype
+    assert lib.hag_aggregate_fwd(h._h, 0, 0, 0, dummy, ctypes.c_void_p(8192), None, None) == 2     # D
+    assert lib.hag_aggregate_fwd(h._h, 0, 0, 64, None, ctypes.c_void_p(8192), None, None) == 1     # NULL
+    assert lib.hag_aggregate_fwd(None, 0, 0, 64, dummy, ctypes.c_void_p(8192), None, None) == 1
+    assert lib.hag_get_info(None, None) == 1 and lib.hag_export(h._h, None) == 1
+    assert lib.hag_to_device(h._h, -1) == 2
+    assert lib.hag_workspace_bytes(None, 4) == 0 and lib.hag_last_launch_count(None) == 0
+    assert hb.status_str(3).startswith("malformed") and hb.status_str(99) == "unknown status"
+    assert lib.hag_destroy(None) == 0
