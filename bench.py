@@ -1,0 +1,429 @@
+#!/usr/bin/env python
+"""Benchmark of the HAG aggregation hot path on B200.
+
+A step is one pass of the whole path over one synthetic workload: for every
+layer the forward aggregation over the HAG (level pair-sum kernels, then the
+gather over the residual rows) and then for every layer the backward aggregation
+(gathers over the transposed HAG, last level first).  Inputs are resident in
+HBM when the timed region starts; the L2 is flushed between timed steps (a
+256 MiB write) so every step starts cold.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 1..5]
+    python bench.py --impl reference       # the fp64 CPU oracle on the host cores
+
+Prints ONE JSON line.  With N > 1 (under torchrun) every rank runs the same
+workload on its own GPU (independent problems, no data-path collective): weak
+scaling, value = units of all ranks / max-over-ranks time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "HAG fwd+bwd aggregation GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+L2_FLUSH_BYTES = 256 << 20
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# --------------------------------------------------------------------------- #
+# clocks
+# --------------------------------------------------------------------------- #
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = sorted(sm)[len(sm) // 2:]          # upper half: samples taken under load
+        return {"sm_mhz": float(np.median(busy)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- #
+# bytes
+# --------------------------------------------------------------------------- #
+def algorithmic_bytes(n, d, dtype, arr, info):
+    """Rows read + rows written per pass, at their stored width.  Rows of the
+    aggregation nodes (a-hat / their gradients) are fp32 whatever the dtype."""
+    s = 4 if dtype == "f32" else 2
+    k = info["num_agg"]
+    res_sec = int((arr["res_idx"] >= n).sum())
+    agg_sec = int((arr["agg_in"] >= n).sum())
+    e_res = int(arr["res_idx"].shape[0])
+    reads_prim = (e_res - res_sec) + (2 * k - agg_sec)
+    reads_sec = res_sec + agg_sec
+    per_pass = d * (s * reads_prim + 4 * reads_sec + s * n + 4 * k)      # forward; backward moves the same rows
+    plain = d * s * (info["e"] + n)
+    fwd_gather = d * (s * (e_res - res_sec) + 4 * res_sec + s * n)       # the dominant launch
+    return dict(hag_pass=per_pass, plain_pass=plain, fwd_gather=fwd_gather)
+
+
+# --------------------------------------------------------------------------- #
+# CPU oracle legs
+# --------------------------------------------------------------------------- #
+def oracle_step_factory(w, budget_edges=3.0e7):
+    """One oracle 'step': direct fp64 forward + backward on a bounded sample of the
+    workload's rows.  Returns (fn, fraction_of_workload, description)."""
+    from oracle import oracle as O
+    from paper_1906_03707_b200 import synth
+    g = w.graph
+    x = synth.features(w.seed, g.n, w.d, w.feat_dist, w.dtype).astype(np.float64)
+    gr = synth.upstream_grad(w.seed, g.n, w.d, w.feat_dist, w.dtype).astype(np.float64)
+    work = g.e * w.d / 64.0
+    if work <= budget_edges:
+        rows, frac, what = None, 1.0, "all rows"
+    else:
+        frac = budget_edges / work
+        m = max(1, int(g.n * frac))
+        rows = np.sort(np.random.default_rng(0).choice(g.n, m, replace=False))
+        frac = m / g.n
+        what = f"{m} of {g.n} rows drawn uniformly (forward and backward each)"
+
+    def step():
+        for _ in range(w.layers):
+            O.direct_forward(g.row_ptr, g.col_idx, x, w.reduce, rows=rows)
+        for _ in range(w.layers):
+            O.direct_backward(g.row_ptr, g.col_idx, gr, w.reduce, rows=rows)
+
+    return step, frac, what
+
+
+def run_reference(args, w, bytes_per_step_fn):
+    """--impl reference: the oracle as it stands, timed on the host cores."""
+    step, frac, what = oracle_step_factory(w)
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    sec = (time.perf_counter() - t0) / max(args.steps, 1)
+    bytes_step = bytes_per_step_fn() * frac
+    value = bytes_step / sec / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "sample": what},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": what},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- #
+# main
+# --------------------------------------------------------------------------- #
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=2, help="1-5; 2 is the 50 000-node clustered power-law graph")
+    ap.add_argument("--scale", type=float, default=1.0)
+    ap.add_argument("--capacity-frac", type=float, default=0.25)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    from paper_1906_03707_b200 import synth
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        w = synth.workload(args.workload, scale=args.scale, capacity_frac=args.capacity_frac)
+        s = 4 if w.dtype == "f32" else 2
+
+        def plain_bytes():      # the oracle evaluates the GNN-graph directly
+            return 2 * w.layers * w.d * s * (w.graph.e + w.graph.n)
+
+        run_reference(args, w, plain_bytes)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_1906_03707_b200 as hb
+    from paper_1906_03707_b200.build import build as build_library
+
+    build_library()
+    hb.load_library()                       # raises if the CUDA library is missing: no fallback
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (use --impl reference for the CPU oracle)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = synth.workload(args.workload, scale=args.scale, capacity_frac=args.capacity_frac)
+    g = w.graph
+    t0 = time.perf_counter()
+    h = hb.Hag.build(g.row_ptr, g.col_idx, w.capacity).to_device(local_rank)
+    build_s = time.perf_counter() - t0
+    info = h.info()
+    arr = h.arrays()
+    nbytes = algorithmic_bytes(g.n, w.d, w.dtype, arr, info)
+    tdt = torch.float32 if w.dtype == "f32" else torch.bfloat16
+    x = torch.from_numpy(synth.features(w.seed, g.n, w.d, w.feat_dist, w.dtype)).to(dev).to(tdt)
+    gr = torch.from_numpy(synth.upstream_grad(w.seed, g.n, w.d, w.feat_dist, w.dtype)).to(dev).to(tdt)
+    bufs = [torch.empty_like(x) for _ in range(2 * w.layers)]
+    ws_bytes = h.workspace_bytes(w.d)
+    ws = torch.empty(max(ws_bytes // 4, 4), dtype=torch.float32, device=dev)
+    flush = torch.empty(L2_FLUSH_BYTES // 4, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def step(hag: bool):
+        launches = 0
+        cur = x
+        for l in range(w.layers):
+            if hag:
+                h.aggregate_fwd(cur, w.reduce, out=bufs[l], workspace=ws)
+            else:
+                h.csr_fwd(cur, w.reduce, out=bufs[l])
+            launches += h.last_launch_count
+            cur = bufs[l]
+        cur = gr
+        for l in range(w.layers):
+            o = bufs[w.layers + l]
+            if hag:
+                h.aggregate_bwd(cur, w.reduce, out=o, workspace=ws)
+            else:
+                h.csr_bwd(cur, w.reduce, out=o)
+            launches += h.last_launch_count
+            cur = o
+        return launches
+
+    def barrier():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+
+    def timed(hag: bool, steps: int, cold: bool):
+        """Sum of the per-step device times (events on the launching stream); the L2 flush sits between steps."""
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        stops = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        launches = 0
+        barrier()
+        for i in range(steps):
+            if cold:
+                flush.zero_()
+            starts[i].record(stream)
+            launches += step(hag)
+            stops[i].record(stream)
+        barrier()
+        ms = sum(a.elapsed_time(b) for a, b in zip(starts, stops))
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms / max(steps, 1), launches
+
+    for _ in range(args.warmup):
+        step(True)
+        step(False)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    hag_ms, launches = timed(True, args.steps, cold=True)
+    clocks = sampler.stop() if rank == 0 else {}
+    csr_ms, _ = timed(False, args.steps, cold=True)
+    hag_warm_ms, _ = timed(True, args.steps, cold=False)
+    csr_warm_ms, _ = timed(False, args.steps, cold=False)
+
+    # the dominant kernel, timed live with event pairs around every launch
+    h.profile(True)
+    kinds = {0: [], 1: [], 2: []}
+    fwd_gather, bwd_gather = [], []
+    for _ in range(args.steps):
+        flush.zero_()
+        h.aggregate_fwd(x, w.reduce, out=bufs[0], workspace=ws)
+        rec = h.profile_read()
+        for ms, kind, _, _ in rec:
+            kinds[kind].append(ms)
+        fwd_gather.append(rec[-1][0])
+        h.aggregate_bwd(gr, w.reduce, out=bufs[w.layers], workspace=ws)
+        rec = h.profile_read()
+        for ms, kind, _, _ in rec:
+            kinds[kind].append(ms)
+        bwd_gather.append(rec[-1][0])
+    h.profile(False)
+    peak, peak_kind = measured_peak()
+    fg_ms = float(np.mean(fwd_gather))
+    achieved = nbytes["fwd_gather"] / (fg_ms * 1e-3) / 1e9
+
+    # end to end through the host-buffer entry point: pinned host inputs and outputs
+    e2e = None
+    if not args.no_e2e:
+        xh = x.cpu().pin_memory()
+        gh = gr.cpu().pin_memory()
+        oh = [torch.empty_like(xh).pin_memory() for _ in range(2 * w.layers)]
+
+        def host_step():
+            cur = xh
+            for l in range(w.layers):
+                h.aggregate_host(cur, oh[l], w.reduce, backward=False, use_hag=True)
+                cur = oh[l]
+                if w.layers > 1:
+                    torch.cuda.synchronize(dev)      # the next layer reads this host buffer
+            cur = gh
+            for l in range(w.layers):
+                h.aggregate_host(cur, oh[w.layers + l], w.reduce, backward=True, use_hag=True)
+                cur = oh[w.layers + l]
+                if w.layers > 1:
+                    torch.cuda.synchronize(dev)
+
+        for _ in range(3):
+            host_step()
+        barrier()
+        t0 = time.perf_counter()
+        e0 = torch.cuda.Event(enable_timing=True)
+        e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            host_step()
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / max(args.steps, 1)
+        if world > 1:
+            t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        io = 2 * w.layers * x.numel() * x.element_size()
+        e2e = {"value": world * 2 * w.layers * nbytes["hag_pass"] / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
+               "h2d_bytes_per_step": io, "d2h_bytes_per_step": io, "ms_per_step": e2e_ms,
+               "api": "hag_aggregate_host (pinned host buffers in and out, copies inside the timed region)"}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        ostep, frac, what = oracle_step_factory(w)
+        ostep()
+        reps, t0 = 0, time.perf_counter()
+        while reps < 3 or time.perf_counter() - t0 < 10.0:
+            ostep()
+            reps += 1
+            if time.perf_counter() - t0 > 30.0:
+                break
+        sec = (time.perf_counter() - t0) / reps
+        s = 4 if w.dtype == "f32" else 2
+        plain_step = 2 * w.layers * w.d * s * (g.e + g.n)
+        cpu = {"value": plain_step * frac / sec / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+               "sample": f"{what}; {reps} repetitions; bytes counted as (|E|+N)*D*{s} per pass like the GPU's plain path",
+               "ms_per_step_full_workload": sec / frac * 1e3}
+
+    if rank == 0:
+        bytes_step = 2 * w.layers * nbytes["hag_pass"]
+        value = world * bytes_step / (hag_ms * 1e-3) / 1e9
+        plain_step = 2 * w.layers * nbytes["plain_pass"]
+        line = {
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": hag_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {
+                "workload": f"{w.name}: {g.name}, N={g.n}, E={info['e']}, D={w.d}, {w.dtype} storage, {w.reduce}, "
+                            f"|V_A|={info['num_agg']} (capacity {w.capacity}), {w.layers} layer(s), fwd+bwd",
+                "l2": "flushed between timed steps (256 MiB write outside the per-step events)",
+                "timing": "sum of per-step CUDA-event intervals on the launching stream, max over ranks",
+            },
+            "clocks": clocks,
+            "e2e": e2e,
+            "gpu_launches": launches,
+            "pct_of_hbm_nominal_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
+            "pct_of_hbm_measured": 100.0 * value / world / peak,
+            "plain_csr": {"ms_per_step": csr_ms, "gbps": world * plain_step / (csr_ms * 1e-3) / 1e9,
+                          "speedup_hag_vs_plain": csr_ms / hag_ms},
+            "warm_l2": {"hag_ms_per_step": hag_warm_ms, "plain_ms_per_step": csr_warm_ms,
+                        "hag_gbps": world * bytes_step / (hag_warm_ms * 1e-3) / 1e9},
+            "hag": {"num_agg": info["num_agg"], "levels": info["num_levels"], "e_hat": info["e_hat"],
+                    "aggregation_reduction": info["aggregations_gnn"] / max(info["aggregations_hag"], 1),
+                    "read_reduction": info["e"] / max(info["e_hat"], 1),
+                    "byte_reduction": nbytes["plain_pass"] / nbytes["hag_pass"],
+                    "build_seconds": build_s, "bytes_per_step": bytes_step},
+            "kernels_ms": {"level_pair_sum_total": float(np.sum(kinds[0])) / args.steps,
+                           "bwd_level_gather_total": float(np.sum(kinds[1])) / args.steps,
+                           "fwd_final_gather": fg_ms, "bwd_final_gather": float(np.mean(bwd_gather))},
+            "roofline": {"bound": "hbm", "kernel": "gather_sum_kernel (forward gather over the residual rows)",
+                         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_kind": f"{peak_kind} copy bandwidth", "traffic": None,
+                         "algorithmic_bytes_per_launch": nbytes["fwd_gather"], "ms_per_launch": fg_ms},
+            "cpu_baseline": cpu,
+        }
+        if w.dtype == "bf16":
+            line["dtype"] = "f32 accumulate, bf16 storage"
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -169,6 +169,18 @@ hag_status csr_aggregate_bwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype,
 hag_status hag_aggregate_host(hag_t *h, int backward, int use_hag, hag_reduce reduce, hag_dtype dtype, int32_t D,
                               const void *in_host, void *out_host, void *cuda_stream);
 
+/* Per-launch timing for measurement (no counterpart in the paper; it reports
+ * kernel time only).  While enabled, every kernel an aggregate call enqueues is
+ * bracketed by a pair of CUDA events on the caller's stream (created on first use
+ * with cudaEventCreate and kept by the handle).  hag_profile_read synchronises
+ * on the events of the LAST call and returns how many launches it made; for the
+ * first `max` of them it fills ms[i] (device time), kind[i] (0 = level pair-sum,
+ * 1 = gather over the aggregation nodes of one level (backward), 2 = gather over
+ * the graph nodes), rows[i] (rows written) and edges[i] (source rows read).
+ * Arrays may be NULL.  Returns -1 on error. */
+hag_status hag_profile_enable(hag_t *h, int enable);
+int32_t hag_profile_read(hag_t *h, int32_t max, float *ms, int32_t *kind, int64_t *rows, int64_t *edges);
+
 /* Number of kernels the last aggregate call on this handle enqueued. */
 int32_t hag_last_launch_count(const hag_t *h);
 

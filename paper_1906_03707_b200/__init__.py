@@ -26,7 +26,7 @@ HAG_F32, HAG_BF16 = 0, 1
 EXPORTED_SYMBOLS = [
     "hag_build", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes",
     "hag_aggregate_fwd", "hag_aggregate_bwd", "csr_aggregate_fwd", "csr_aggregate_bwd",
-    "hag_aggregate_host", "hag_last_launch_count", "hag_status_str",
+    "hag_aggregate_host", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
 ]
 
 
@@ -93,6 +93,10 @@ def load_library():
         f.restype = ctypes.c_int
     lib.hag_aggregate_host.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, i32, vp, vp, vp]
     lib.hag_aggregate_host.restype = ctypes.c_int
+    lib.hag_profile_enable.argtypes = [vp, ctypes.c_int]
+    lib.hag_profile_enable.restype = ctypes.c_int
+    lib.hag_profile_read.argtypes = [vp, i32, vp, vp, vp, vp]
+    lib.hag_profile_read.restype = i32
     lib.hag_last_launch_count.argtypes = [vp]
     lib.hag_last_launch_count.restype = i32
     lib.hag_status_str.argtypes = [ctypes.c_int]
@@ -188,6 +192,25 @@ class Hag:
     @property
     def last_launch_count(self) -> int:
         return int(load_library().hag_last_launch_count(self._h))
+
+    def profile(self, enable: bool):
+        """``hag_profile_enable``: bracket every launch with CUDA events."""
+        _check(load_library().hag_profile_enable(self._h, int(bool(enable))), "hag_profile_enable")
+
+    def profile_read(self):
+        """``hag_profile_read``: list of (ms, kind, rows, edges) for the launches of the last call."""
+        lib = load_library()
+        n = lib.hag_profile_read(self._h, 0, None, None, None, None)
+        if n < 0:
+            raise HagError(6, "hag_profile_read")
+        ms = np.zeros(max(n, 1), np.float32)
+        kind = np.zeros(max(n, 1), np.int32)
+        rows = np.zeros(max(n, 1), np.int64)
+        edges = np.zeros(max(n, 1), np.int64)
+        got = lib.hag_profile_read(self._h, n, ms.ctypes.data, kind.ctypes.data, rows.ctypes.data, edges.ctypes.data)
+        if got < 0:
+            raise HagError(6, "hag_profile_read")
+        return [(float(ms[i]), int(kind[i]), int(rows[i]), int(edges[i])) for i in range(n)]
 
     # -- device ------------------------------------------------------------- #
     def to_device(self, device: int = 0) -> "Hag":

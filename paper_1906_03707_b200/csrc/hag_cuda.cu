@@ -47,6 +47,8 @@ hag_status upload_i32(int32_t **dst, const V *src, size_t count) {
 
 void free_device(hag *h) {
     hag_device_arrays &d = h->d;
+    for (cudaEvent_t ev : h->events) cudaEventDestroy(ev);
+    h->events.clear();
     void *ptrs[] = {d.agg_in, d.res_ptr, d.res_idx, d.t_ptr, d.t_idx, d.csr_ptr, d.csr_idx, d.csr_t_ptr,
                     d.csr_t_idx, d.inv_degree, d.stage_in, d.stage_out, d.stage_ws};
     for (void *p : ptrs)
@@ -90,6 +92,36 @@ cudaError_t launch_pairs(const hagk::PairArgs &p, int n_chunks, cudaStream_t s) 
     return cudaGetLastError();
 }
 
+// Brackets each launch with an event pair when profiling is on; always counts launches.
+struct Recorder {
+    hag *h;
+    cudaStream_t s;
+    bool failed = false;
+    Recorder(const hag *h_, cudaStream_t s_) : h(const_cast<hag *>(h_)), s(s_) {
+        h->notes.clear();
+        h->last_launches = 0;
+    }
+    void begin(int32_t kind, int64_t rows, int64_t edges) {
+        if (h->profile) {
+            const size_t i = h->notes.size();
+            while (h->events.size() < 2 * (i + 1)) {
+                cudaEvent_t ev;
+                if (cudaEventCreate(&ev) != cudaSuccess) { cudaGetLastError(); failed = true; return; }
+                h->events.push_back(ev);
+            }
+            if (cudaEventRecord(h->events[2 * i], s) != cudaSuccess) { cudaGetLastError(); failed = true; }
+        }
+        h->notes.push_back({kind, rows, edges});
+    }
+    void end() {
+        if (h->profile && !failed) {
+            const size_t i = h->notes.size() - 1;
+            if (cudaEventRecord(h->events[2 * i + 1], s) != cudaSuccess) { cudaGetLastError(); failed = true; }
+        }
+        ++h->last_launches;
+    }
+};
+
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 hag_status check_call(const hag *h, hag_dtype dtype, int32_t D, const void *in, const void *out) {
@@ -106,10 +138,9 @@ hag_status check_call(const hag *h, hag_dtype dtype, int32_t D, const void *in, 
 // Forward over the HAG: level launches (Algorithm 2 lines 5-6), then the gather (lines 7-8).
 template <typename T>
 hag_status fwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, const void *x, void *out, void *ws,
-                    cudaStream_t s, int32_t *launches) {
+                    cudaStream_t s, Recorder &rec) {
     const int n_chunks = D / hagk::Chunk<T>::kElems;
     const hag_device_arrays &d = h->d;
-    *launches = 0;
     hagk::GatherArgs a{};
     a.row_begin = 0;
     a.row_count = h->n;
@@ -127,8 +158,10 @@ hag_status fwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
             p.ahat = static_cast<float *>(ws);
             p.n = h->n;
             p.D = D;
+            if (p.count <= 0) continue;
+            rec.begin(0, p.count, 2 * int64_t(p.count));
             if (launch_pairs<T>(p, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
-            ++*launches;
+            rec.end();
         }
         a.row_ptr = d.res_ptr;
         a.idx = d.res_idx;
@@ -143,8 +176,11 @@ hag_status fwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
         a.idx = d.csr_idx;
         a.n_prim = std::numeric_limits<int32_t>::max();
     }
-    if (launch_gather<T>(a, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
-    if (h->n > 0) ++*launches;
+    if (h->n > 0) {
+        rec.begin(2, h->n, (use_hag && h->num_agg > 0) ? h->e_res : (use_hag ? h->e_res : h->e));
+        if (launch_gather<T>(a, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+        rec.end();
+    }
     return HAG_OK;
 }
 
@@ -154,10 +190,9 @@ hag_status fwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
 // that graph node (scaled by 1/|N| for mean), an id >= n for an aggregation node.
 template <typename T>
 hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, const void *g, void *gx, void *ws,
-                    cudaStream_t s, int32_t *launches) {
+                    cudaStream_t s, Recorder &rec) {
     const int n_chunks = D / hagk::Chunk<T>::kElems;
     const hag_device_arrays &d = h->d;
-    *launches = 0;
     hagk::GatherArgs a{};
     a.prim = g;
     a.src_scale = (reduce == HAG_MEAN) ? d.inv_degree : nullptr;
@@ -174,8 +209,10 @@ hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
             lv.out = ws;
             lv.out_row_offset = h->n;
             lv.out_is_f32 = 1;
+            if (lv.row_count <= 0) continue;
+            rec.begin(1, lv.row_count, h->t_ptr[size_t(lv.row_begin) + lv.row_count] - h->t_ptr[lv.row_begin]);
             if (launch_gather<T>(lv, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
-            ++*launches;
+            rec.end();
         }
     } else if (use_hag) {
         a.row_ptr = d.t_ptr;
@@ -189,8 +226,11 @@ hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
     a.row_begin = 0;
     a.row_count = h->n;
     a.out = gx;
-    if (launch_gather<T>(a, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
-    if (h->n > 0) ++*launches;
+    if (h->n > 0) {
+        rec.begin(2, h->n, use_hag ? h->t_ptr[h->n] : h->e);
+        if (launch_gather<T>(a, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+        rec.end();
+    }
     return HAG_OK;
 }
 
@@ -206,14 +246,14 @@ hag_status run(const hag *h, bool backward, bool use_hag, hag_reduce reduce, hag
     DeviceGuard guard(h->device);
     if (!guard.ok) { cudaGetLastError(); return HAG_ERR_CUDA; }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    int32_t launches = 0;
+    Recorder rec(h, s);
     if (dtype == HAG_F32)
-        st = backward ? bwd_impl<float>(h, use_hag, reduce, D, in, out, ws, s, &launches)
-                      : fwd_impl<float>(h, use_hag, reduce, D, in, out, ws, s, &launches);
+        st = backward ? bwd_impl<float>(h, use_hag, reduce, D, in, out, ws, s, rec)
+                      : fwd_impl<float>(h, use_hag, reduce, D, in, out, ws, s, rec);
     else
-        st = backward ? bwd_impl<__nv_bfloat16>(h, use_hag, reduce, D, in, out, ws, s, &launches)
-                      : fwd_impl<__nv_bfloat16>(h, use_hag, reduce, D, in, out, ws, s, &launches);
-    const_cast<hag *>(h)->last_launches = launches;
+        st = backward ? bwd_impl<__nv_bfloat16>(h, use_hag, reduce, D, in, out, ws, s, rec)
+                      : fwd_impl<__nv_bfloat16>(h, use_hag, reduce, D, in, out, ws, s, rec);
+    if (st == HAG_OK && rec.failed) st = HAG_ERR_CUDA;
     return st;
 }
 
@@ -337,3 +377,28 @@ extern "C" hag_status hag_aggregate_host(hag_t *h, int backward, int use_hag, ha
 }
 
 extern "C" int32_t hag_last_launch_count(const hag_t *h) { return h ? h->last_launches : 0; }
+
+extern "C" hag_status hag_profile_enable(hag_t *h, int enable) {
+    if (!h) return HAG_ERR_NULL;
+    h->profile = enable != 0;
+    return HAG_OK;
+}
+
+extern "C" int32_t hag_profile_read(hag_t *h, int32_t max, float *ms, int32_t *kind, int64_t *rows, int64_t *edges) {
+    if (!h || h->device < 0) return -1;
+    const int32_t count = int32_t(h->notes.size());
+    if (!h->profile) return count;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) { cudaGetLastError(); return -1; }
+    for (int32_t i = 0; i < count && i < max; ++i) {
+        if (h->events.size() < size_t(2 * (i + 1))) return -1;
+        if (cudaEventSynchronize(h->events[2 * i + 1]) != cudaSuccess) { cudaGetLastError(); return -1; }
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, h->events[2 * i], h->events[2 * i + 1]) != cudaSuccess) { cudaGetLastError(); return -1; }
+        if (ms) ms[i] = t;
+        if (kind) kind[i] = h->notes[i].kind;
+        if (rows) rows[i] = h->notes[i].rows;
+        if (edges) edges[i] = h->notes[i].edges;
+    }
+    return count;
+}

@@ -4,6 +4,8 @@
 #include <cstdint>
 #include <vector>
 
+#include <cuda_runtime.h>
+
 #include "hag.h"
 
 struct hag_device_arrays {
@@ -45,6 +47,11 @@ struct hag {
     int device = -1;
     hag_device_arrays d;
     int32_t last_launches = 0;
+    // per-launch timing (hag_profile_*)
+    bool profile = false;
+    std::vector<cudaEvent_t> events;          // pairs: 2*i start, 2*i+1 stop
+    struct launch_note { int32_t kind; int64_t rows, edges; };
+    std::vector<launch_note> notes;           // launches of the last call
 };
 
 // hag_build.cpp: the search (Algorithm 3) in creation-id space.  Fills

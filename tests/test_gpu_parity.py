@@ -1,0 +1,250 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle
+element by element on the same seeded inputs.
+
+Tolerances (Sigma|terms| is the oracle's sum of absolute addends, scaled like the result):
+  fp32 features:  |gpu - oracle| <= 1e-5 * Sigma|terms| + 1e-6
+  bf16 features:  |gpu - oracle| <= 1e-2 * Sigma|terms| + 1e-6, and the tighter
+                  fp32 bound plus one bf16 output rounding, 2^-8 * |oracle|
+"""
+import numpy as np
+import pytest
+
+import paper_1906_03707_b200 as hb
+from oracle import oracle as O
+from paper_1906_03707_b200 import synth
+from paper_1906_03707_b200.build import build as build_library
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _library():
+    build_library()
+    hb.load_library()
+    assert torch.cuda.is_available(), "the parity tests need a CUDA device"
+
+
+def _dev(a, dtype):
+    t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    return t.to(torch.bfloat16) if dtype == "bf16" else t
+
+
+def _host(t):
+    return t.float().cpu().numpy().astype(np.float64)
+
+
+def _assert_close(got, want, scale, dtype, what):
+    err = np.abs(got - want)
+    if dtype == "f32":
+        bound = 1e-5 * scale + 1e-6
+    else:
+        bound = np.minimum(1e-2 * scale + 1e-6, 1e-5 * scale + 1e-6 + 2.0 ** -8 * np.abs(want))
+    bad = err > bound
+    assert not bad.any(), f"{what}: {int(bad.sum())} elements out of tolerance, worst excess {float((err - bound).max()):.3e}"
+
+
+def _check_all_paths(g, hag, x, gr, reduce, dtype, rows=None):
+    """Forward and backward, HAG and plain CSR, against the direct fp64 definition."""
+    xd, gd = _dev(x, dtype), _dev(gr, dtype)
+    a, t = O.direct_forward(g.row_ptr, g.col_idx, x.astype(np.float64), reduce, rows=rows)
+    gx, tg = O.direct_backward(g.row_ptr, g.col_idx, gr.astype(np.float64), reduce, rows=rows)
+    sel = slice(None) if rows is None else rows
+    for name, fwd, bwd in (("hag", hag.aggregate_fwd, hag.aggregate_bwd), ("csr", hag.csr_fwd, hag.csr_bwd)):
+        out = _host(fwd(xd, reduce))[sel]
+        _assert_close(out, a, t, dtype, f"{name} forward {reduce}")
+        gout = _host(bwd(gd, reduce))[sel]
+        _assert_close(gout, gx, tg, dtype, f"{name} backward {reduce}")
+
+
+CASES = {
+    "cfg1": lambda: synth.workload(1),
+    "cfg2-small": lambda: synth.workload(2, scale=0.1),
+    "cfg3-small": lambda: synth.workload(3, scale=0.04),
+    "cfg4-small": lambda: synth.workload(4, scale=0.01),
+    "cfg5-small": lambda: synth.workload(5, scale=0.02),
+}
+_built = {}
+
+
+def _case(name):
+    if name not in _built:
+        w = CASES[name]()
+        h = hb.Hag.build(w.graph.row_ptr, w.graph.col_idx, w.capacity).to_device(0)
+        _built[name] = (w, h)
+    return _built[name]
+
+
+@pytest.mark.parametrize("name", list(CASES))
+@pytest.mark.parametrize("reduce", ["sum", "mean"])
+def test_workload_shapes_match_oracle(name, reduce):
+    w, h = _case(name)
+    g = w.graph
+    x = synth.features(w.seed, g.n, w.d, w.feat_dist, w.dtype)
+    gr = synth.upstream_grad(w.seed, g.n, w.d, w.feat_dist, w.dtype)
+    assert h.info()["num_agg"] > 0
+    _check_all_paths(g, h, x, gr, reduce, w.dtype)
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2-small", "cfg4-small", "cfg5-small"])
+def test_structure_on_device_run_equals_oracle_structure(name):
+    w, h = _case(name)
+    g = w.graph
+    ref = O.canonical_hag(g.row_ptr, O.greedy_pairmap(g.row_ptr, g.col_idx, w.capacity))
+    arr = h.arrays()
+    for key in ("level_ptr", "agg_in", "res_ptr", "res_idx", "t_ptr", "t_idx", "in_degree"):
+        assert np.array_equal(arr[key], getattr(ref, key)), key
+    assert h.info()["device"] == 0
+
+
+@pytest.mark.parametrize("dtype,d", [("f32", 4), ("f32", 8), ("f32", 20), ("f32", 64), ("f32", 100), ("f32", 128),
+                                      ("f32", 256), ("f32", 516), ("bf16", 8), ("bf16", 24), ("bf16", 256),
+                                      ("bf16", 264), ("bf16", 1024)])
+def test_feature_widths(dtype, d):
+    w, h = _case("cfg2-small")
+    g = w.graph
+    x = synth.features(7, g.n, d, "normal", dtype)
+    gr = synth.upstream_grad(7, g.n, d, "normal", dtype)
+    _check_all_paths(g, h, x, gr, "mean", dtype)
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2-small", "cfg3-small", "cfg5-small"])
+def test_integer_features_are_bit_exact_for_sum(name):
+    # every fp32 partial sum of small integers is exact, so any summation order must give the oracle's bits
+    w, h = _case(name)
+    g = w.graph
+    for dtype in ("f32", "bf16"):
+        x = synth.features(9, g.n, 32, "int", dtype)
+        a, _ = O.direct_forward(g.row_ptr, g.col_idx, x.astype(np.float64), "sum")
+        gx, _ = O.direct_backward(g.row_ptr, g.col_idx, x.astype(np.float64), "sum")
+        xd = _dev(x, dtype)
+        if dtype == "bf16" and max(np.abs(a).max(), np.abs(gx).max()) > 256:
+            continue  # bf16 output cannot hold the integers exactly
+        for fwd, bwd in ((h.aggregate_fwd, h.aggregate_bwd), (h.csr_fwd, h.csr_bwd)):
+            assert np.array_equal(_host(fwd(xd, "sum")), a)
+            assert np.array_equal(_host(bwd(xd, "sum")), gx)
+
+
+def test_capacity_zero_is_the_plain_path_bit_for_bit():
+    g = synth.workload(2, scale=0.05).graph
+    h = hb.Hag.build(g.row_ptr, g.col_idx, 0).to_device(0)
+    assert h.info()["num_agg"] == 0 and h.workspace_bytes(64) == 0
+    x = _dev(synth.features(3, g.n, 64, "normal"), "f32")
+    for reduce in ("sum", "mean"):
+        assert torch.equal(h.aggregate_fwd(x, reduce), h.csr_fwd(x, reduce))
+        assert torch.equal(h.aggregate_bwd(x, reduce), h.csr_bwd(x, reduce))
+    assert h.last_launch_count == 1
+
+
+def test_runs_are_reproducible_bit_for_bit():
+    w, h = _case("cfg2-small")
+    x = _dev(synth.features(4, w.graph.n, 64, "normal"), "f32")
+    a1, b1 = h.aggregate_fwd(x, "mean"), h.aggregate_bwd(x, "mean")
+    for _ in range(3):
+        assert torch.equal(h.aggregate_fwd(x, "mean"), a1) and torch.equal(h.aggregate_bwd(x, "mean"), b1)
+
+
+def test_adjoint_identity_on_device_outputs():
+    w, h = _case("cfg2-small")
+    n = w.graph.n
+    x = synth.features(5, n, 32, "normal")
+    gr = synth.upstream_grad(5, n, 32, "normal")
+    for reduce in ("sum", "mean"):
+        fx = _host(h.aggregate_fwd(_dev(x, "f32"), reduce))
+        bg = _host(h.aggregate_bwd(_dev(gr, "f32"), reduce))
+        lhs, rhs = float((fx * gr).sum()), float((x.astype(np.float64) * bg).sum())
+        scale = float(np.abs(fx * gr).sum())
+        assert abs(lhs - rhs) <= 1e-5 * scale
+
+
+def test_two_stacked_layers_share_handle_and_workspace():
+    # parity per call: the oracle is fed the device's input of that call
+    w, h = _case("cfg3-small")
+    g = w.graph
+    x = synth.features(w.seed, g.n, w.d, "normal")
+    ws = torch.empty(h.workspace_bytes(w.d) // 4, dtype=torch.float32, device="cuda")
+    y1 = h.aggregate_fwd(_dev(x, "f32"), "sum", workspace=ws)
+    y2 = h.aggregate_fwd(y1, "sum", workspace=ws)
+    g1 = h.aggregate_bwd(y2, "sum", workspace=ws)
+    g0 = h.aggregate_bwd(g1, "sum", workspace=ws)
+    for inp, out, fn in ((x, y1, O.direct_forward), (_host(y1), y2, O.direct_forward),
+                         (_host(y2), g1, O.direct_backward), (_host(g1), g0, O.direct_backward)):
+        want, t = fn(g.row_ptr, g.col_idx, np.asarray(inp, dtype=np.float64), "sum")
+        _assert_close(_host(out), want, t, "f32", fn.__name__)
+
+
+def test_rows_without_neighbours_and_hubs():
+    # star: node 0 aggregates everyone (long row), most nodes aggregate nothing (empty rows)
+    n = 3000
+    rows = [list(range(1, n))] + [[] for _ in range(n - 1)]
+    rows[5] = [0, 1, 2]
+    rows[6] = [0, 1, 2]
+    g = synth.csr_from_rows(rows)
+    h = hb.Hag.build(g.row_ptr, g.col_idx, n // 4).to_device(0)
+    x = synth.features(6, n, 64, "uniform")
+    gr = synth.upstream_grad(6, n, 64, "uniform")
+    for reduce in ("sum", "mean"):
+        _check_all_paths(g, h, x, gr, reduce, "f32")
+    out = h.aggregate_fwd(_dev(x, "f32"), "mean")
+    assert not out[1:5].any()
+
+
+def test_empty_graph_launches_nothing():
+    h = hb.Hag.build(np.zeros(1, np.int64), np.zeros(0, np.int32), 4).to_device(0)
+    x = torch.empty((0, 64), device="cuda")
+    lib = hb.load_library()
+    # zero rows: pointers may be anything valid and aligned
+    buf = torch.zeros(64, device="cuda")
+    out = torch.zeros(64, device="cuda")
+    st = lib.hag_aggregate_fwd(h._h, 0, 0, 64, buf.data_ptr(), out.data_ptr(), None, None)
+    assert st == 0 and h.last_launch_count == 0 and x.numel() == 0
+
+
+def test_host_buffer_entry_point_matches_device_path():
+    w, h = _case("cfg2-small")
+    n = w.graph.n
+    x = torch.from_numpy(synth.features(8, n, 64, "normal")).pin_memory()
+    out = torch.empty_like(x).pin_memory()
+    for backward in (False, True):
+        for use_hag in (True, False):
+            h.aggregate_host(x, out, "mean", backward=backward, use_hag=use_hag)
+            torch.cuda.synchronize()
+            fn = {(False, True): h.aggregate_fwd, (True, True): h.aggregate_bwd,
+                  (False, False): h.csr_fwd, (True, False): h.csr_bwd}[(backward, use_hag)]
+            assert torch.equal(out.cuda(), fn(x.cuda(), "mean"))
+
+
+def test_device_call_errors_are_statuses():
+    w, h = _case("cfg1")
+    lib = hb.load_library()
+    x = torch.zeros((w.graph.n, 16), device="cuda")
+    out = torch.zeros_like(x)
+    assert lib.hag_aggregate_fwd(h._h, 0, 0, 16, x.data_ptr(), out.data_ptr(), None, None) == 9       # workspace missing
+    assert lib.hag_aggregate_fwd(h._h, 0, 0, 16, x.data_ptr(), x.data_ptr(), None, None) == 2         # out aliases x
+    assert lib.hag_aggregate_fwd(h._h, 7, 0, 16, x.data_ptr(), out.data_ptr(), out.data_ptr(), None) == 2  # reduce
+    assert lib.hag_to_device(h._h, 0) == 0                                                            # idempotent
+    assert lib.hag_to_device(h._h, 10_000) == 2
+
+
+@pytest.mark.parametrize("index", [2, 4])
+def test_full_size_workloads_sampled_rows(index):
+    """The benchmark's launch configuration at full size; the oracle computes sampled rows one by one."""
+    w = synth.workload(index)
+    g = w.graph
+    h = hb.Hag.build(g.row_ptr, g.col_idx, w.capacity).to_device(0)
+    info = h.info()
+    assert info["num_agg"] == w.capacity
+    x = synth.features(w.seed, g.n, w.d, w.feat_dist, w.dtype)
+    gr = synth.upstream_grad(w.seed, g.n, w.d, w.feat_dist, w.dtype)
+    rng = np.random.default_rng(0)
+    deg = np.diff(g.row_ptr)
+    rows = np.unique(np.concatenate([rng.choice(g.n, 4000, replace=False), np.argsort(deg)[-50:], np.argsort(deg)[:50],
+                                     [0, g.n - 1]]))
+    _check_all_paths(g, h, x, gr, w.reduce, w.dtype, rows=rows)
+    # the HAG itself: Theorem 2 via exact integer features on every row
+    xi = synth.features(1, g.n, 16, "int")
+    a, _ = O.direct_forward(g.row_ptr, g.col_idx, xi.astype(np.float64), "sum")
+    assert np.array_equal(_host(h.aggregate_fwd(_dev(xi, "f32"), "sum")), a)
+    gx, _ = O.direct_backward(g.row_ptr, g.col_idx, xi.astype(np.float64), "sum")
+    assert np.array_equal(_host(h.aggregate_bwd(_dev(xi, "f32"), "sum")), gx)
+    h.close()
