@@ -58,7 +58,8 @@ typedef enum {
     HAG_ERR_ALIGN = 8,       /* pointer or row size not 16-byte aligned                     */
     HAG_ERR_WORKSPACE = 9,   /* workspace missing although the HAG has aggregation nodes    */
     HAG_ERR_TIMEOUT = 10,    /* reserved: a bounded device-side wait gave up                */
-    HAG_ERR_NOT_ON_DEVICE = 11 /* hag_to_device has not been called                         */
+    HAG_ERR_NOT_ON_DEVICE = 11,/* hag_to_device has not been called                         */
+    HAG_ERR_TOO_LARGE = 12     /* the problem needs more than the built-in scratch array holds */
 } hag_status;
 
 typedef enum { HAG_SUM = 0, HAG_MEAN = 1 } hag_reduce;
@@ -180,6 +181,36 @@ hag_status hag_aggregate_host(hag_t *h, int backward, int use_hag, hag_reduce re
  * Arrays may be NULL.  Returns -1 on error. */
 hag_status hag_profile_enable(hag_t *h, int enable);
 int32_t hag_profile_read(hag_t *h, int32_t max, float *ms, int32_t *kind, int64_t *rows, int64_t *edges);
+
+/* hag_aggregate_fwd for callers that must not allocate device memory (the paper
+ * has no counterpart: its operators take their buffers from the framework).
+ *
+ * Some hosts cannot hand this library a workspace and cannot let it call
+ * cudaMalloc either: a serving process whose device memory is one arena sized at
+ * start-up and owned by another component, or a latency-bound loop in which the
+ * device-wide synchronisation that cudaMalloc/cudaFree imply would stall every
+ * other stream.  For them the rows of the aggregation nodes live in an array that
+ * is part of the library image itself: HAG_STATIC_SCRATCH_BYTES of device memory,
+ * reserved on every GPU that loads the library until the process exits.
+ *
+ * Same arguments, results and errors as hag_aggregate_fwd, without `workspace`.
+ * Bit-identical output to hag_aggregate_fwd.  Additionally:
+ *   - HAG_ERR_TOO_LARGE when hag_workspace_bytes(h, D) exceeds
+ *     HAG_STATIC_SCRATCH_BYTES (nothing is launched);
+ *   - the call itself allocates nothing: no cudaMalloc, cudaFree, event or stream
+ *     creation, and no host heap use;
+ *   - the first call on each device looks up the array's device address (a
+ *     one-off query, made with that device current).  Make that first call
+ *     during start-up, before any stream capture begins;
+ *   - there is ONE array per device, shared by every handle and every call, and
+ *     it still holds the previous call's rows.  The forward pass writes every
+ *     aggregation-node row before it reads it, so nothing needs clearing; but
+ *     two calls that can run at the same time on one device (different streams,
+ *     or different threads) race on the array and corrupt each other's result.
+ *     Keep such calls on one stream or order them with events. */
+#define HAG_STATIC_SCRATCH_BYTES (16u << 20)
+hag_status hag_aggregate_fwd_static(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D,
+                                    const void *x, void *out, void *cuda_stream);
 
 /* Number of kernels the last aggregate call on this handle enqueued. */
 int32_t hag_last_launch_count(const hag_t *h);

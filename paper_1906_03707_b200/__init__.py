@@ -26,7 +26,7 @@ HAG_F32, HAG_BF16 = 0, 1
 EXPORTED_SYMBOLS = [
     "hag_build", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes",
     "hag_aggregate_fwd", "hag_aggregate_bwd", "csr_aggregate_fwd", "csr_aggregate_bwd",
-    "hag_aggregate_host", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
+    "hag_aggregate_host", "hag_aggregate_fwd_static", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
 ]
 
 
@@ -93,6 +93,8 @@ def load_library():
         f.restype = ctypes.c_int
     lib.hag_aggregate_host.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, i32, vp, vp, vp]
     lib.hag_aggregate_host.restype = ctypes.c_int
+    lib.hag_aggregate_fwd_static.argtypes = [vp, ctypes.c_int, ctypes.c_int, i32, vp, vp, vp]
+    lib.hag_aggregate_fwd_static.restype = ctypes.c_int
     lib.hag_profile_enable.argtypes = [vp, ctypes.c_int]
     lib.hag_profile_enable.restype = ctypes.c_int
     lib.hag_profile_read.argtypes = [vp, i32, vp, vp, vp, vp]
@@ -264,6 +266,20 @@ class Hag:
     def aggregate_bwd(self, grad_out, reduce="sum", out=None, workspace=None):
         """``hag_aggregate_bwd`` on the current stream."""
         return self._run("hag_aggregate_bwd", True, grad_out, reduce, out, workspace)
+
+    def aggregate_fwd_static(self, x, out, reduce="sum"):
+        """``hag_aggregate_fwd_static``: the forward pass for hosts that may not allocate
+        device memory.  The caller supplies ``out``; the aggregation-node rows go to the
+        scratch array built into the library (one per GPU, shared by all calls, so
+        keep calls on one stream).  This wrapper allocates nothing either."""
+        import torch
+        if out.shape != x.shape or out.dtype != x.dtype or not (x.is_contiguous() and out.is_contiguous()):
+            raise ValueError("out must match x")
+        stream = torch.cuda.current_stream(x.device).cuda_stream
+        st = load_library().hag_aggregate_fwd_static(self._h, _reduce_code(reduce), self._dtype_code(x), x.shape[1],
+                                                     x.data_ptr(), out.data_ptr(), stream)
+        _check(st, "hag_aggregate_fwd_static")
+        return out
 
     def csr_fwd(self, x, reduce="sum", out=None):
         """``csr_aggregate_fwd``: the plain GNN-graph, same kernel."""

@@ -396,6 +396,7 @@ extern "C" const char *hag_status_str(hag_status s) {
         case HAG_ERR_WORKSPACE: return "workspace required but missing";
         case HAG_ERR_TIMEOUT: return "device-side wait timed out";
         case HAG_ERR_NOT_ON_DEVICE: return "structure not on a device (call hag_to_device)";
+        case HAG_ERR_TOO_LARGE: return "aggregation-node rows exceed the built-in scratch array (HAG_STATIC_SCRATCH_BYTES)";
     }
     return "unknown status";
 }

@@ -402,3 +402,83 @@ extern "C" int32_t hag_profile_read(hag_t *h, int32_t max, float *ms, int32_t *k
     }
     return count;
 }
+
+// --------------------------------------------------------------------------- //
+// Forward pass without any allocation: the aggregation-node rows live in an
+// array inside the library image.  Kept apart from the code above on purpose:
+// it shares only the launch helpers.
+// --------------------------------------------------------------------------- //
+namespace {
+
+// Device memory reserved on every GPU that loads this library, until exit.
+static __device__ __align__(256) unsigned char g_static_scratch[HAG_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxStaticDevices = 64;
+// Device address of g_static_scratch per device ordinal.  In host code the name
+// g_static_scratch is only a handle for the runtime, never an address a kernel
+// may be given; the address comes from cudaGetSymbolAddress, once per device.
+void *g_static_scratch_addr[kMaxStaticDevices] = {};
+
+// Caller has made `device` current.
+hag_status static_scratch_address(int device, void **out) {
+    if (device < 0 || device >= kMaxStaticDevices) return HAG_ERR_ARG;
+    void *p = __atomic_load_n(&g_static_scratch_addr[device], __ATOMIC_ACQUIRE);
+    if (!p) {
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return HAG_ERR_CUDA;
+        }
+        __atomic_store_n(&g_static_scratch_addr[device], p, __ATOMIC_RELEASE);  // same value from any thread
+    }
+    *out = p;
+    return HAG_OK;
+}
+
+template <typename T>
+hag_status fwd_static_impl(const hag *h, hag_reduce reduce, int32_t D, const void *x, void *out, float *scratch,
+                           cudaStream_t s) {
+    const int n_chunks = D / hagk::Chunk<T>::kElems;
+    const hag_device_arrays &d = h->d;
+    for (int32_t l = 1; l <= h->num_levels; ++l) {
+        hagk::PairArgs p{};
+        p.agg_in = d.agg_in;
+        p.first = int32_t(h->level_ptr[l - 1]);
+        p.count = int32_t(h->level_ptr[l] - h->level_ptr[l - 1]);
+        p.x = x;
+        p.ahat = scratch;
+        p.n = h->n;
+        p.D = D;
+        if (launch_pairs<T>(p, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+    }
+    hagk::GatherArgs a{};
+    a.row_ptr = d.res_ptr;
+    a.idx = d.res_idx;
+    a.row_begin = 0;
+    a.row_count = h->n;
+    a.prim = x;
+    a.sec = scratch;
+    a.n_prim = h->num_agg > 0 ? h->n : std::numeric_limits<int32_t>::max();
+    a.dst_scale = (reduce == HAG_MEAN) ? d.inv_degree : nullptr;
+    a.out = out;
+    a.D = D;
+    if (launch_gather<T>(a, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+    return HAG_OK;
+}
+
+}  // namespace
+
+extern "C" hag_status hag_aggregate_fwd_static(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D,
+                                               const void *x, void *out, void *cuda_stream) {
+    hag_status st = check_call(h, dtype, D, x, out);
+    if (st != HAG_OK) return st;
+    if (reduce != HAG_SUM && reduce != HAG_MEAN) return HAG_ERR_ARG;
+    if (size_t(h->num_agg) * size_t(D) * sizeof(float) > size_t(HAG_STATIC_SCRATCH_BYTES)) return HAG_ERR_TOO_LARGE;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) { cudaGetLastError(); return HAG_ERR_CUDA; }
+    void *scratch = nullptr;
+    st = static_scratch_address(h->device, &scratch);
+    if (st != HAG_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (dtype == HAG_F32) return fwd_static_impl<float>(h, reduce, D, x, out, static_cast<float *>(scratch), s);
+    return fwd_static_impl<__nv_bfloat16>(h, reduce, D, x, out, static_cast<float *>(scratch), s);
+}
