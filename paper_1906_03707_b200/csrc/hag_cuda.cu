@@ -4,6 +4,7 @@
 
 #include <algorithm>
 #include <cstdint>
+#include <cstdlib>
 #include <limits>
 #include <new>
 #include <vector>
@@ -62,19 +63,56 @@ int lanes_per_row(int n_chunks) {
     return l;
 }
 
+// Every kernel is launched with programmatic stream serialisation (see hag_kernels.cuh).
+template <typename Args>
+cudaError_t launch_pdl(void (*kernel)(Args), unsigned grid, const Args &args, cudaStream_t s) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(hagk::kThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args);
+}
+
+int g_tune = 0;
+int tune_variant() { return g_tune; }
+
+template <typename T, int LPR, bool SS>
+cudaError_t launch_gather_lpr(const hagk::GatherArgs &a, cudaStream_t s) {
+    const unsigned grid = unsigned((a.row_count + hagk::kWarps - 1) / hagk::kWarps);
+    if constexpr (sizeof(T) == 4) {
+        switch (tune_variant()) {
+            case 1: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 8, SS, 6>, grid, a, s);
+            case 2: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 16, SS, 4>, grid, a, s);
+            case 3: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 12>, grid, a, s);
+            default: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 8, SS, 8>, grid, a, s);
+        }
+    } else {
+        switch (tune_variant()) {
+            case 1: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 8, SS, 4>, grid, a, s);
+            case 2: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 6>, grid, a, s);
+            case 3: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 12>, grid, a, s);
+            default: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 8>, grid, a, s);
+        }
+    }
+}
+
 template <typename T>
 cudaError_t launch_gather(const hagk::GatherArgs &a, int n_chunks, cudaStream_t s) {
     if (a.row_count <= 0) return cudaSuccess;
     const int lpr = lanes_per_row(n_chunks);
-    const int rows_per_cta = hagk::kWarps * (32 / lpr);
-    const unsigned grid = unsigned((a.row_count + rows_per_cta - 1) / rows_per_cta);
+    const bool ss = a.src_scale != nullptr;
     switch (lpr) {
-        case 4: hagk::gather_sum_kernel<T, 4><<<grid, hagk::kThreads, 0, s>>>(a); break;
-        case 8: hagk::gather_sum_kernel<T, 8><<<grid, hagk::kThreads, 0, s>>>(a); break;
-        case 16: hagk::gather_sum_kernel<T, 16><<<grid, hagk::kThreads, 0, s>>>(a); break;
-        default: hagk::gather_sum_kernel<T, 32><<<grid, hagk::kThreads, 0, s>>>(a); break;
+        case 4: return ss ? launch_gather_lpr<T, 4, true>(a, s) : launch_gather_lpr<T, 4, false>(a, s);
+        case 8: return ss ? launch_gather_lpr<T, 8, true>(a, s) : launch_gather_lpr<T, 8, false>(a, s);
+        case 16: return ss ? launch_gather_lpr<T, 16, true>(a, s) : launch_gather_lpr<T, 16, false>(a, s);
+        default: return ss ? launch_gather_lpr<T, 32, true>(a, s) : launch_gather_lpr<T, 32, false>(a, s);
     }
-    return cudaGetLastError();
 }
 
 template <typename T>
@@ -84,12 +122,11 @@ cudaError_t launch_pairs(const hagk::PairArgs &p, int n_chunks, cudaStream_t s) 
     const int rows_per_cta = hagk::kWarps * (32 / lpr);
     const unsigned grid = unsigned((p.count + rows_per_cta - 1) / rows_per_cta);
     switch (lpr) {
-        case 4: hagk::pair_sum_kernel<T, 4><<<grid, hagk::kThreads, 0, s>>>(p); break;
-        case 8: hagk::pair_sum_kernel<T, 8><<<grid, hagk::kThreads, 0, s>>>(p); break;
-        case 16: hagk::pair_sum_kernel<T, 16><<<grid, hagk::kThreads, 0, s>>>(p); break;
-        default: hagk::pair_sum_kernel<T, 32><<<grid, hagk::kThreads, 0, s>>>(p); break;
+        case 4: return launch_pdl(hagk::pair_sum_kernel<T, 4>, grid, p, s);
+        case 8: return launch_pdl(hagk::pair_sum_kernel<T, 8>, grid, p, s);
+        case 16: return launch_pdl(hagk::pair_sum_kernel<T, 16>, grid, p, s);
+        default: return launch_pdl(hagk::pair_sum_kernel<T, 32>, grid, p, s);
     }
-    return cudaGetLastError();
 }
 
 // Brackets each launch with an event pair when profiling is on; always counts launches.
@@ -482,3 +519,5 @@ extern "C" hag_status hag_aggregate_fwd_static(const hag_t *h, hag_reduce reduce
     if (dtype == HAG_F32) return fwd_static_impl<float>(h, reduce, D, x, out, static_cast<float *>(scratch), s);
     return fwd_static_impl<__nv_bfloat16>(h, reduce, D, x, out, static_cast<float *>(scratch), s);
 }
+
+extern "C" void hag_debug_set_tune(int v) { g_tune = v; }

@@ -2,18 +2,26 @@
 //
 // Everything here is a row gather-sum bounded by memory traffic, so the design
 // is about wide coalesced loads and enough of them in flight:
-//   * a group of LPR lanes (4..32, a power of two) owns one output row; lane i
-//     owns the 16-byte chunk i of the row (4 fp32 or 8 bf16 features), so one
-//     load instruction of the group reads one contiguous feature row;
-//   * neighbour ids are read coalesced, LPR at a time, and handed round with
-//     shuffles; UNROLL row loads are issued back to back before any add, and
-//     the next batch of ids is fetched before the current one is consumed;
-//   * sums are fp32 in NACC independent accumulators combined at the end in a
-//     fixed order: no atomics, same bits every run;
+//   * one warp owns one output row.  A row of D features is n_chunks 16-byte
+//     chunks (4 fp32 or 8 bf16 features); LPR = the power of two >= n_chunks
+//     (capped at 32) lanes cover one source row with ONE load instruction, and
+//     the 32/LPR lane groups ("slices") of the warp take alternate neighbours,
+//     so narrow rows still keep all 32 lanes loading distinct data;
+//   * neighbour ids are read coalesced, 32 at a time, and handed round with
+//     shuffles; the next batch of ids is fetched before the current one is used;
+//   * UNROLL row loads per lane are issued back to back, then summed as a
+//     balanced tree and added to ONE fp32 accumulator: the rounding error grows
+//     like n/UNROLL + log2(UNROLL) ulps, as with UNROLL independent partial sums,
+//     at a quarter of the registers (more resident warps);
+//   * slices are combined with butterfly shuffles in a fixed order; no atomics,
+//     one writer per output row: same bits every run;
 //   * a source id below n_prim reads the primary table (the layer input, fp32
 //     or bf16); an id at or above it reads the fp32 rows of the aggregation
 //     nodes.  One kernel therefore serves Algorithm 2's final loop, the plain
-//     GNN-graph, and every step of the backward pass over the transposed HAG.
+//     GNN-graph, and every step of the backward pass over the transposed HAG;
+//   * every kernel is launched with programmatic stream serialisation: it lets
+//     its successor start launching at once and waits for its predecessor's
+//     memory only after it has fetched its own (static) row pointers and ids.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -21,7 +29,7 @@
 
 namespace hagk {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 128;
 constexpr int kWarps = kThreads / 32;
 
 struct GatherArgs {
@@ -43,6 +51,10 @@ struct GatherArgs {
 template <typename T> struct Chunk;
 template <> struct Chunk<float> { static constexpr int kElems = 4; };
 template <> struct Chunk<__nv_bfloat16> { static constexpr int kElems = 8; };
+
+// Programmatic dependent launch (PTX griddepcontrol).
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 __device__ __forceinline__ float4 ld_f4(const void *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
 __device__ __forceinline__ uint4 ld_u4(const void *p) { return __ldg(reinterpret_cast<const uint4 *>(p)); }
@@ -66,120 +78,156 @@ __device__ __forceinline__ uint4 f32x8_to_bf16(const float *f) {
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-// One source row chunk -> kElems floats.
+// Per-lane view of the two source tables: byte pointers already offset to the
+// lane's chunk, so a row address is one multiply-add.
 template <typename T>
-__device__ __forceinline__ void load_chunk(const GatherArgs &a, int32_t id, int chunk, float *v) {
-    constexpr int E = Chunk<T>::kElems;
-    if constexpr (E == 4) {
-        const float *p = (id < a.n_prim) ? reinterpret_cast<const float *>(a.prim) + size_t(id) * a.D
-                                         : a.sec + size_t(id - a.n_prim) * a.D;
-        const float4 q = ld_f4(p + chunk * 4);
-        v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
-    } else {
-        if (id < a.n_prim) {
-            const __nv_bfloat16 *p = reinterpret_cast<const __nv_bfloat16 *>(a.prim) + size_t(id) * a.D;
-            bf16x8_to_f32(ld_u4(p + chunk * 8), v);
+struct Tables {
+    const char *prim;   // primary base + chunk offset
+    const char *sec;    // secondary base + chunk offset - n_prim * sec_row_bytes
+    int32_t n_prim;
+    uint32_t prim_row_bytes, sec_row_bytes;
+    __device__ __forceinline__ Tables(const void *p, const float *s, int32_t n, int32_t D, int chunk) {
+        constexpr int E = Chunk<T>::kElems;
+        n_prim = n;
+        prim_row_bytes = uint32_t(D) * sizeof(T);
+        sec_row_bytes = uint32_t(D) * 4u;
+        prim = reinterpret_cast<const char *>(p) + size_t(chunk) * 16;
+        // never dereferenced for ids < n_prim, so the wrapped offset is harmless when s is null
+        sec = reinterpret_cast<const char *>(s) + size_t(chunk) * (E * 4) - size_t(n) * sec_row_bytes;
+    }
+    // One source row chunk -> kElems floats.
+    __device__ __forceinline__ void load(int32_t id, float *v) const {
+        constexpr int E = Chunk<T>::kElems;
+        if constexpr (E == 4) {
+            const bool is_prim = id < n_prim;
+            const char *base = is_prim ? prim : sec;
+            const float4 q = ld_f4(base + size_t(uint32_t(id)) * prim_row_bytes);   // both tables have 4 D bytes per row
+            v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
         } else {
-            const float *p = a.sec + size_t(id - a.n_prim) * a.D + chunk * 8;
-            const float4 q0 = ld_f4(p), q1 = ld_f4(p + 4);
-            v[0] = q0.x; v[1] = q0.y; v[2] = q0.z; v[3] = q0.w;
-            v[4] = q1.x; v[5] = q1.y; v[6] = q1.z; v[7] = q1.w;
+            if (id < n_prim) {
+                bf16x8_to_f32(ld_u4(prim + size_t(uint32_t(id)) * prim_row_bytes), v);
+            } else {
+                const char *p = sec + size_t(uint32_t(id)) * sec_row_bytes;
+                const float4 q0 = ld_f4(p), q1 = ld_f4(p + 16);
+                v[0] = q0.x; v[1] = q0.y; v[2] = q0.z; v[3] = q0.w;
+                v[4] = q1.x; v[5] = q1.y; v[6] = q1.z; v[7] = q1.w;
+            }
         }
     }
-}
+};
 
 template <typename T>
-__device__ __forceinline__ void store_chunk(const GatherArgs &a, int32_t out_row, int chunk, const float *v) {
+__device__ __forceinline__ void store_chunk(void *out, int out_is_f32, int32_t D, int32_t out_row, int chunk, const float *v) {
     constexpr int E = Chunk<T>::kElems;
-    if (a.out_is_f32) {
-        float *p = reinterpret_cast<float *>(a.out) + size_t(out_row) * a.D + chunk * E;
+    if (out_is_f32) {
+        float *p = reinterpret_cast<float *>(out) + size_t(out_row) * D + chunk * E;
 #pragma unroll
         for (int i = 0; i < E; i += 4) *reinterpret_cast<float4 *>(p + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
     } else if constexpr (E == 4) {
-        float *p = reinterpret_cast<float *>(a.out) + size_t(out_row) * a.D + chunk * 4;
+        float *p = reinterpret_cast<float *>(out) + size_t(out_row) * D + chunk * 4;
         __stcs(reinterpret_cast<float4 *>(p), make_float4(v[0], v[1], v[2], v[3]));
     } else {
-        __nv_bfloat16 *p = reinterpret_cast<__nv_bfloat16 *>(a.out) + size_t(out_row) * a.D + chunk * 8;
+        __nv_bfloat16 *p = reinterpret_cast<__nv_bfloat16 *>(out) + size_t(out_row) * D + chunk * 8;
         __stcs(reinterpret_cast<uint4 *>(p), f32x8_to_bf16(v));
     }
 }
 
-// out[row] = (dst_scale[row]) * sum_{e in row} (src_scale[id_e]) * table[id_e]
-template <typename T, int LPR>
-__global__ void __launch_bounds__(kThreads) gather_sum_kernel(const GatherArgs a) {
+// Gather-sum of one row by one warp; used by the grid kernel and by the fused
+// small-level kernel.  Returns with the result stored.
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE>
+__device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int lane, bool first_row_of_kernel) {
     constexpr int E = Chunk<T>::kElems;
-    constexpr int UNROLL = (LPR >= 8) ? 8 : LPR;
-    constexpr int NACC = (E == 4) ? 8 : 4;      // independent partial sums (keeps fp32 error ~ n/NACC ulps)
-    constexpr int NA = (NACC < UNROLL) ? NACC : UNROLL;
-    constexpr int GROUPS = 32 / LPR;
-    const int lane = threadIdx.x & 31;
-    const int warp = threadIdx.x >> 5;
-    const int sub = lane / LPR;
+    constexpr int G = 32 / LPR;                 // slices per warp
+    constexpr int PER_BATCH = LPR;              // neighbours each slice takes from a batch of 32 ids
+    constexpr int U = (UNROLL < PER_BATCH) ? UNROLL : PER_BATCH;
+    const int slice = lane / LPR;
     const int gl = lane % LPR;
-    const unsigned mask = (LPR == 32) ? 0xffffffffu : (((1u << LPR) - 1u) << (sub * LPR));
-    const int r_local = (blockIdx.x * kWarps + warp) * GROUPS + sub;
-    if (r_local >= a.row_count) return;
-    const int32_t row = a.row_begin + r_local;
     const int32_t b = __ldg(a.row_ptr + row), e = __ldg(a.row_ptr + row + 1);
     const int n_chunks = a.D / E;
     const float dscale = a.dst_scale ? __ldg(a.dst_scale + row) : 1.0f;
+    int32_t first = (b + lane < e) ? __ldg(a.idx + b + lane) : -1;
+    // the factor of each source travels with its id: fetched a batch ahead, handed round by shuffle
+    float first_s = 1.0f;
+    if constexpr (SRC_SCALE) first_s = (first >= 0 && first < a.n_prim) ? __ldg(a.src_scale + first) : 1.0f;
+    if (first_row_of_kernel) pdl_wait();        // structure arrays are static; features may come from the previous kernel
 
     for (int c0 = 0; c0 < n_chunks; c0 += LPR) {
         const int chunk = c0 + gl;
         const bool live = chunk < n_chunks;
-        float acc[NA][E];
+        const Tables<T> tab(a.prim, a.sec, a.n_prim, a.D, live ? chunk : 0);
+        float acc[E];
 #pragma unroll
-        for (int i = 0; i < NA; ++i)
-#pragma unroll
-            for (int j = 0; j < E; ++j) acc[i][j] = 0.0f;
+        for (int j = 0; j < E; ++j) acc[j] = 0.0f;
 
-        int32_t mine = (b + gl < e) ? __ldg(a.idx + b + gl) : -1;
-        for (int32_t base = b; base < e; base += LPR) {
+        int32_t mine = first;
+        float mine_s = first_s;
+        if (c0 != 0) {
+            mine = (b + lane < e) ? __ldg(a.idx + b + lane) : -1;
+            if constexpr (SRC_SCALE) mine_s = (mine >= 0 && mine < a.n_prim) ? __ldg(a.src_scale + mine) : 1.0f;
+        }
+        for (int32_t base = b; base < e; base += 32) {
             const int32_t cur = mine;
-            const int32_t nb = base + LPR;
-            mine = (nb + gl < e) ? __ldg(a.idx + nb + gl) : -1;     // next batch of ids, in flight early
-            const int cnt = min(LPR, e - base);
+            const float cur_s = mine_s;
+            const int32_t nb = base + 32;
+            mine = (nb + lane < e) ? __ldg(a.idx + nb + lane) : -1;      // next batch of ids, in flight early
+            if constexpr (SRC_SCALE) mine_s = (mine >= 0 && mine < a.n_prim) ? __ldg(a.src_scale + mine) : 1.0f;
+            const int cnt = min(32, e - base);
 #pragma unroll
-            for (int k = 0; k < LPR; k += UNROLL) {
-                if (k < cnt) {
-                    float v[UNROLL][E];
-                    float s[UNROLL];
+            for (int k = 0; k < PER_BATCH; k += U) {
+                if (k * G < cnt) {
+                    float v[U][E];
 #pragma unroll
-                    for (int u = 0; u < UNROLL; ++u) {
-                        const int32_t id = __shfl_sync(mask, cur, k + u, LPR);
-                        s[u] = 1.0f;
+                    for (int u = 0; u < U; ++u) {
+                        const int src_lane = (k + u) * G + slice;
+                        const int32_t id = __shfl_sync(0xffffffffu, cur, src_lane);
                         if (id >= 0 && live) {
-                            load_chunk<T>(a, id, chunk, v[u]);
-                            if (a.src_scale && id < a.n_prim) s[u] = __ldg(a.src_scale + id);
+                            tab.load(id, v[u]);
                         } else {
 #pragma unroll
                             for (int j = 0; j < E; ++j) v[u][j] = 0.0f;
                         }
                     }
+                    if constexpr (SRC_SCALE) {
 #pragma unroll
-                    for (int u = 0; u < UNROLL; ++u)
+                        for (int u = 0; u < U; ++u) {
+                            const float sc = __shfl_sync(0xffffffffu, cur_s, (k + u) * G + slice);
 #pragma unroll
-                        for (int j = 0; j < E; ++j) acc[u % NA][j] = fmaf(v[u][j], s[u], acc[u % NA][j]);
+                            for (int j = 0; j < E; ++j) v[u][j] *= sc;
+                        }
+                    }
+                    // balanced tree over the U loaded rows, then one add into the accumulator
+#pragma unroll
+                    for (int w = U / 2; w >= 1; w /= 2)
+#pragma unroll
+                        for (int u = 0; u < w; ++u)
+#pragma unroll
+                            for (int j = 0; j < E; ++j) v[u][j] += v[u + w][j];
+#pragma unroll
+                    for (int j = 0; j < E; ++j) acc[j] += v[0][j];
                 }
             }
         }
-        if (live) {
-            float r[E];
+        // combine the slices (fixed butterfly), then slice 0 stores
 #pragma unroll
-            for (int j = 0; j < E; ++j) {
-                // fixed pairwise combine of the partial sums
-                float t[NA];
+        for (int off = LPR; off < 32; off <<= 1)
 #pragma unroll
-                for (int i = 0; i < NA; ++i) t[i] = acc[i][j];
+            for (int j = 0; j < E; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], off);
+        if (live && slice == 0) {
 #pragma unroll
-                for (int w = NA / 2; w >= 1; w /= 2)
-#pragma unroll
-                    for (int i = 0; i < w; ++i) t[i] += t[i + w];
-                r[j] = t[0] * dscale;
-            }
-            store_chunk<T>(a, row - a.out_row_offset, chunk, r);
+            for (int j = 0; j < E; ++j) acc[j] *= dscale;
+            store_chunk<T>(a.out, a.out_is_f32, a.D, row - a.out_row_offset, chunk, acc);
         }
     }
+}
+
+// out[row] = (dst_scale[row]) * sum_{e in row} (src_scale[id_e]) * table[id_e]
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS>
+__global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_kernel(const GatherArgs a) {
+    pdl_launch_dependents();
+    const int lane = threadIdx.x & 31;
+    const int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (r_local >= a.row_count) return;
+    gather_row<T, LPR, UNROLL, SRC_SCALE>(a, a.row_begin + r_local, lane, true);
 }
 
 // Level kernel of Algorithm 2 (lines 5-6): every aggregation node of one level is
@@ -195,32 +243,31 @@ struct PairArgs {
 };
 
 template <typename T, int LPR>
-__global__ void __launch_bounds__(kThreads) pair_sum_kernel(const PairArgs p) {
+__device__ __forceinline__ void pair_row(const PairArgs &p, int32_t j, int gl, bool first_of_kernel) {
     constexpr int E = Chunk<T>::kElems;
-    constexpr int GROUPS = 32 / LPR;
-    const int lane = threadIdx.x & 31;
-    const int warp = threadIdx.x >> 5;
-    const int sub = lane / LPR;
-    const int gl = lane % LPR;
-    const int j_local = (blockIdx.x * kWarps + warp) * GROUPS + sub;
-    if (j_local >= p.count) return;
-    const int32_t j = p.first + j_local;
     const int2 in = __ldg(reinterpret_cast<const int2 *>(p.agg_in) + j);
-    GatherArgs a{};
-    a.prim = p.x;
-    a.sec = p.ahat;
-    a.n_prim = p.n;
-    a.D = p.D;
+    if (first_of_kernel) pdl_wait();
     const int n_chunks = p.D / E;
     for (int chunk = gl; chunk < n_chunks; chunk += LPR) {
+        const Tables<T> tab(p.x, p.ahat, p.n, p.D, chunk);
         float u[E], v[E];
-        load_chunk<T>(a, in.x, chunk, u);
-        load_chunk<T>(a, in.y, chunk, v);
+        tab.load(in.x, u);
+        tab.load(in.y, v);
         float *o = p.ahat + size_t(j) * p.D + chunk * E;
 #pragma unroll
         for (int i = 0; i < E; i += 4)
             *reinterpret_cast<float4 *>(o + i) = make_float4(u[i] + v[i], u[i + 1] + v[i + 1], u[i + 2] + v[i + 2], u[i + 3] + v[i + 3]);
     }
+}
+
+template <typename T, int LPR>
+__global__ void __launch_bounds__(kThreads) pair_sum_kernel(const PairArgs p) {
+    pdl_launch_dependents();
+    constexpr int GROUPS = 32 / LPR;
+    const int lane = threadIdx.x & 31;
+    const int j_local = (blockIdx.x * kWarps + (threadIdx.x >> 5)) * GROUPS + lane / LPR;
+    if (j_local >= p.count) return;
+    pair_row<T, LPR>(p, p.first + j_local, lane % LPR, true);
 }
 
 }  // namespace hagk
