@@ -100,6 +100,13 @@ typedef struct hag_arrays {
     const int32_t *trace;      /* [3*num_agg] merges in creation order: v1 < v2 (creation ids), r      */
     const int64_t *csr_t_ptr;  /* [n+1] transposed input graph                                          */
     const int32_t *csr_t_idx;
+    /* Deep levels evaluated in one launch each way (see hag_build): */
+    int32_t fwd_cut;           /* levels 1..fwd_cut run level by level; deeper nodes from their expansion  */
+    int32_t bwd_cut;           /* same for the backward pass                                              */
+    const int64_t *ftail_ptr;  /* [num_agg - level_ptr[fwd_cut] + 1]                                       */
+    const int32_t *ftail_idx;  /* per deep node: the ids of level <= fwd_cut whose sum it is, ascending    */
+    const int64_t *btail_ptr;  /* [num_agg - level_ptr[bwd_cut] + 1]                                       */
+    const int32_t *btail_idx;  /* per deep node: the graph nodes whose output uses it, ascending           */
 } hag_arrays;
 
 /* Algorithm 3, set-Aggregate branch (the paper's graph_to_hag): starting from the
@@ -109,6 +116,15 @@ typedef struct hag_arrays {
  * the lexicographically smallest pair (v1 < v2; aggregation nodes numbered N, N+1,
  * ... as created).  Then lays the result out for the device (levels, level-sorted
  * ids, input pairs, residual CSR, transposed HAG, transposed input graph).
+ * Deep levels are usually tiny, and a launch per level would cost more than the
+ * rows it moves.  So the layout also picks a cut c: levels 1..c are evaluated
+ * level by level (Algorithm 2 lines 5-6), and every deeper node directly as the
+ * sum over its cover restricted to ids of level <= c (Section 3.1: aggr(v) is the
+ * aggregate over cover(v)), all in one launch.  c minimises
+ *   32768 * (launches) + sum over deep nodes of (expanded inputs - 1),
+ * ties to the larger c; c = num_levels means no expansion.  The backward pass
+ * has its own cut: nodes deeper than it gather straight from the graph-node
+ * outputs that use them (transitively), cost term (expanded users - direct users).
  * Host only; the input arrays are read during the call and not kept.
  * Errors: HAG_ERR_NULL; HAG_ERR_ARG (n < 0, capacity < 0, n + capacity or |E| >=
  * 2^31); HAG_ERR_GRAPH; HAG_ERR_OOM_HOST.  On error *out is NULL. */

@@ -268,6 +268,74 @@ def canonical_hag(row_ptr, search: SearchResult) -> CanonicalHag:
     return CanonicalHag(n, k, num_levels, level_ptr, agg_in, res_ptr, res_idx, t_ptr, t_idx, in_degree, c2c)
 
 
+LAUNCH_ROWS = 32768  # what the layout rule charges for one kernel launch, in rows moved
+
+
+def expanded_tails(h: CanonicalHag) -> dict:
+    """The layout's treatment of deep levels, restated from its rule.
+
+    Forward: with a cut c, an aggregation node deeper than level c is the sum over
+    its cover restricted to ids of level <= c (Section 3.1: aggr(v) aggregates
+    cover(v)); c minimises  LAUNCH_ROWS * (c + [some node is deeper than c])
+    + sum over deep nodes of (expanded inputs - 1), ties to the larger c.
+    Backward: a node deeper than the cut collects the gradient of every graph-node
+    output that uses it, directly or through deeper nodes; the cost term is
+    (transitive users - direct users)."""
+    n, k, L = h.n, h.num_agg, h.num_levels
+    level = np.zeros(n + k, dtype=np.int64)
+    for l in range(1, L + 1):
+        level[n + h.level_ptr[l - 1]: n + h.level_ptr[l]] = l
+    pairs = h.agg_in.reshape(-1, 2)
+
+    def fwd_lists(c):
+        lists = {}
+        for j in range(int(h.level_ptr[c]), k):
+            out = []
+            for s in pairs[j]:
+                s = int(s)
+                out.extend([s] if level[s] <= c else lists[s])
+            lists[n + j] = sorted(out)
+        return lists
+
+    best = (LAUNCH_ROWS * L, L)
+    for c in range(L - 1, -1, -1):
+        cost = LAUNCH_ROWS * (c + 1) + sum(len(v) - 1 for v in fwd_lists(c).values())
+        if cost < best[0]:
+            best = (cost, c)
+    fwd_cut = best[1]
+    fl = fwd_lists(fwd_cut)
+
+    users = {}
+    for j in range(k - 1, -1, -1):
+        out = []
+        for d in h.t_idx[h.t_ptr[n + j]: h.t_ptr[n + j + 1]]:
+            d = int(d)
+            out.extend([d] if d < n else users[d])
+        users[n + j] = sorted(out)
+    best = (LAUNCH_ROWS * L, L)
+    for c in range(L - 1, -1, -1):
+        extra = sum(len(users[n + j]) - int(h.t_ptr[n + j + 1] - h.t_ptr[n + j]) for j in range(int(h.level_ptr[c]), k))
+        cost = LAUNCH_ROWS * (c + 1) + extra
+        if cost < best[0]:
+            best = (cost, c)
+    bwd_cut = best[1]
+
+    def pack(ids, lists):
+        ptr = np.zeros(len(ids) + 1, dtype=np.int64)
+        flat = []
+        for i, w in enumerate(ids):
+            flat.extend(lists[w])
+            ptr[i + 1] = len(flat)
+        return ptr, np.asarray(flat, dtype=np.int32)
+
+    f_ids = [n + j for j in range(int(h.level_ptr[fwd_cut]), k)]
+    b_ids = [n + j for j in range(int(h.level_ptr[bwd_cut]), k)]
+    ftail_ptr, ftail_idx = pack(f_ids, fl)
+    btail_ptr, btail_idx = pack(b_ids, users)
+    return dict(fwd_cut=fwd_cut, bwd_cut=bwd_cut, ftail_ptr=ftail_ptr, ftail_idx=ftail_idx,
+                btail_ptr=btail_ptr, btail_idx=btail_idx)
+
+
 def transposed_csr(row_ptr, col_idx):
     """Out-neighbour CSR of the input graph (destinations ascending): (t_ptr int64, t_idx int32)."""
     rp, ci = _csr(row_ptr, col_idx)

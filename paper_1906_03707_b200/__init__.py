@@ -55,7 +55,9 @@ class HagInfo(ctypes.Structure):
 class HagArrays(ctypes.Structure):
     _fields_ = [("n", ctypes.c_int32), ("num_agg", ctypes.c_int32), ("num_levels", ctypes.c_int32)] + [
         (k, ctypes.c_void_p) for k in ("level_ptr", "agg_in", "res_ptr", "res_idx", "t_ptr", "t_idx", "in_degree",
-                                       "trace", "csr_t_ptr", "csr_t_idx")]
+                                       "trace", "csr_t_ptr", "csr_t_idx")] + [
+        ("fwd_cut", ctypes.c_int32), ("bwd_cut", ctypes.c_int32)] + [
+        (k, ctypes.c_void_p) for k in ("ftail_ptr", "ftail_idx", "btail_ptr", "btail_idx")]
 
 
 _lib = None
@@ -177,7 +179,13 @@ class Hag:
         res_ptr = _view(a.res_ptr, n + 1, np.int64)
         t_ptr = _view(a.t_ptr, n + k + 1, np.int64)
         csr_t_ptr = _view(a.csr_t_ptr, n + 1, np.int64)
+        level_ptr = _view(a.level_ptr, lv + 1, np.int64)
+        ftail_ptr = _view(a.ftail_ptr, k - int(level_ptr[a.fwd_cut]) + 1, np.int64)
+        btail_ptr = _view(a.btail_ptr, k - int(level_ptr[a.bwd_cut]) + 1, np.int64)
         return dict(
+            fwd_cut=a.fwd_cut, bwd_cut=a.bwd_cut, ftail_ptr=ftail_ptr, btail_ptr=btail_ptr,
+            ftail_idx=_view(a.ftail_idx, int(ftail_ptr[-1]), np.int32),
+            btail_idx=_view(a.btail_idx, int(btail_ptr[-1]), np.int32),
             n=n, num_agg=k, num_levels=lv,
             level_ptr=_view(a.level_ptr, lv + 1, np.int64),
             agg_in=_view(a.agg_in, 2 * k, np.int32),

@@ -279,6 +279,92 @@ hag_status hag_layout(hag *h, const std::vector<int32_t> &rows_store, const std:
             for (int32_t v = 0; v < n; ++v)
                 for (int64_t i = h->csr_ptr[v]; i < h->csr_ptr[v + 1]; ++i) h->csr_t_idx[fill[h->csr_idx[i]]++] = v;
         }
+        // ---- deep levels in one launch: choose the cuts and expand ----
+        {
+            const int64_t kLaunchRows = 32768;   // what one extra launch costs, in rows moved
+            const int32_t L = max_level;
+            std::vector<int32_t> clevel(k);      // level per canonical aggregation node
+            for (int32_t l = 1; l <= L; ++l)
+                for (int64_t j = h->level_ptr[l - 1]; j < h->level_ptr[l]; ++j) clevel[j] = l;
+            auto level_of = [&](int32_t id) { return id < n ? 0 : clevel[id - n]; };
+            // forward: size of the expansion of every node for a given cut
+            int32_t best_c = L;
+            int64_t best_cost = kLaunchRows * L;
+            std::vector<int64_t> sz(k);
+            for (int32_t c = L - 1; c >= 0; --c) {
+                int64_t extra = 0;
+                for (int64_t j = h->level_ptr[c]; j < k; ++j) {
+                    int64_t t = 0;
+                    for (int q = 0; q < 2; ++q) {
+                        const int32_t in = h->agg_in[2 * j + q];
+                        t += level_of(in) <= c ? 1 : sz[in - n];
+                    }
+                    sz[j] = t;
+                    extra += t - 1;
+                }
+                const int64_t cost = kLaunchRows * (c + 1) + extra;
+                if (cost < best_cost) { best_cost = cost; best_c = c; }
+            }
+            h->fwd_cut = best_c;
+            {
+                const int64_t j0 = h->level_ptr[best_c];
+                std::vector<std::vector<int32_t>> lists(size_t(k - j0));
+                h->ftail_ptr.assign(size_t(k - j0) + 1, 0);
+                for (int64_t j = j0; j < k; ++j) {
+                    std::vector<int32_t> &dst = lists[j - j0];
+                    for (int q = 0; q < 2; ++q) {
+                        const int32_t in = h->agg_in[2 * j + q];
+                        if (level_of(in) <= best_c) dst.push_back(in);
+                        else dst.insert(dst.end(), lists[in - n - j0].begin(), lists[in - n - j0].end());
+                    }
+                    std::sort(dst.begin(), dst.end());
+                    h->ftail_ptr[j - j0 + 1] = h->ftail_ptr[j - j0] + int64_t(dst.size());
+                }
+                h->ftail_idx.clear();
+                h->ftail_idx.reserve(size_t(h->ftail_ptr.back()));
+                for (auto &l : lists) h->ftail_idx.insert(h->ftail_idx.end(), l.begin(), l.end());
+            }
+            // backward: every node's transitive graph-node users (independent of the cut)
+            std::vector<int64_t> usz(k);
+            for (int64_t j = k - 1; j >= 0; --j) {
+                int64_t t = 0;
+                for (int64_t i = h->t_ptr[n + j]; i < h->t_ptr[n + j + 1]; ++i) {
+                    const int32_t d = h->t_idx[i];
+                    t += d < n ? 1 : usz[d - n];
+                }
+                usz[j] = t;
+            }
+            int32_t best_b = L;
+            int64_t best_bcost = kLaunchRows * L;
+            {
+                int64_t extra = 0;
+                for (int32_t c = L - 1; c >= 0; --c) {
+                    for (int64_t j = h->level_ptr[c]; j < h->level_ptr[c + 1]; ++j)
+                        extra += usz[j] - (h->t_ptr[n + j + 1] - h->t_ptr[n + j]);
+                    const int64_t cost = kLaunchRows * (c + 1) + extra;
+                    if (cost < best_bcost) { best_bcost = cost; best_b = c; }
+                }
+            }
+            h->bwd_cut = best_b;
+            {
+                const int64_t j0 = h->level_ptr[best_b];
+                std::vector<std::vector<int32_t>> lists(size_t(k - j0));
+                for (int64_t j = k - 1; j >= j0; --j) {
+                    std::vector<int32_t> &dst = lists[j - j0];
+                    for (int64_t i = h->t_ptr[n + j]; i < h->t_ptr[n + j + 1]; ++i) {
+                        const int32_t d = h->t_idx[i];
+                        if (d < n) dst.push_back(d);
+                        else dst.insert(dst.end(), lists[d - n - j0].begin(), lists[d - n - j0].end());
+                    }
+                    std::sort(dst.begin(), dst.end());
+                }
+                h->btail_ptr.assign(size_t(k - j0) + 1, 0);
+                for (int64_t j = j0; j < k; ++j) h->btail_ptr[j - j0 + 1] = h->btail_ptr[j - j0] + int64_t(lists[j - j0].size());
+                h->btail_idx.clear();
+                h->btail_idx.reserve(size_t(h->btail_ptr.back()));
+                for (auto &l : lists) h->btail_idx.insert(h->btail_idx.end(), l.begin(), l.end());
+            }
+        }
         // counters of the cost function
         hag_info &f = h->info;
         f = hag_info{};
@@ -379,6 +465,12 @@ extern "C" hag_status hag_export(const hag_t *h, hag_arrays *out) {
     out->trace = h->trace.data();
     out->csr_t_ptr = h->csr_t_ptr.data();
     out->csr_t_idx = h->csr_t_idx.data();
+    out->fwd_cut = h->fwd_cut;
+    out->bwd_cut = h->bwd_cut;
+    out->ftail_ptr = h->ftail_ptr.data();
+    out->ftail_idx = h->ftail_idx.data();
+    out->btail_ptr = h->btail_ptr.data();
+    out->btail_idx = h->btail_idx.data();
     return HAG_OK;
 }
 

@@ -51,7 +51,8 @@ void free_device(hag *h) {
     for (cudaEvent_t ev : h->events) cudaEventDestroy(ev);
     h->events.clear();
     void *ptrs[] = {d.agg_in, d.res_ptr, d.res_idx, d.t_ptr, d.t_idx, d.csr_ptr, d.csr_idx, d.csr_t_ptr,
-                    d.csr_t_idx, d.inv_degree, d.stage_in, d.stage_out, d.stage_ws};
+                    d.csr_t_idx, d.inv_degree, d.stage_in, d.stage_out, d.stage_ws,
+                    d.ftail_ptr, d.ftail_idx, d.btail_ptr, d.btail_idx};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     d = hag_device_arrays{};
@@ -172,10 +173,52 @@ hag_status check_call(const hag *h, hag_dtype dtype, int32_t D, const void *in, 
     return HAG_OK;
 }
 
-// Forward over the HAG: level launches (Algorithm 2 lines 5-6), then the gather (lines 7-8).
+// Aggregation nodes of the forward pass (Algorithm 2 lines 5-6): levels 1..fwd_cut
+// level by level with the pair kernel, every deeper node in one gather launch
+// from its expansion.  rec may be null (no bookkeeping).
+template <typename T>
+hag_status enqueue_fwd_agg(const hag *h, int32_t D, const void *x, float *ws, cudaStream_t s, Recorder *rec) {
+    const int n_chunks = D / hagk::Chunk<T>::kElems;
+    const hag_device_arrays &d = h->d;
+    for (int32_t l = 1; l <= h->fwd_cut; ++l) {
+        hagk::PairArgs p{};
+        p.agg_in = d.agg_in;
+        p.first = int32_t(h->level_ptr[l - 1]);
+        p.count = int32_t(h->level_ptr[l] - h->level_ptr[l - 1]);
+        p.x = x;
+        p.ahat = ws;
+        p.n = h->n;
+        p.D = D;
+        if (p.count <= 0) continue;
+        if (rec) rec->begin(0, p.count, 2 * int64_t(p.count));
+        if (launch_pairs<T>(p, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+        if (rec) rec->end();
+    }
+    const int32_t j0 = int32_t(h->level_ptr[h->fwd_cut]);
+    if (j0 < h->num_agg) {
+        hagk::GatherArgs a{};
+        a.row_ptr = d.ftail_ptr - (h->n + j0);     // indexed by absolute row id
+        a.idx = d.ftail_idx;
+        a.row_begin = h->n + j0;
+        a.row_count = h->num_agg - j0;
+        a.prim = x;
+        a.sec = ws;
+        a.n_prim = h->n;
+        a.out = ws;
+        a.out_row_offset = h->n;
+        a.out_is_f32 = 1;
+        a.D = D;
+        if (rec) rec->begin(1, a.row_count, int64_t(h->ftail_idx.size()));
+        if (launch_gather<T>(a, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+        if (rec) rec->end();
+    }
+    return HAG_OK;
+}
+
+// Forward: aggregation nodes, then the gather over the graph nodes (lines 7-8).
 template <typename T>
 hag_status fwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, const void *x, void *out, void *ws,
-                    cudaStream_t s, Recorder &rec) {
+                    cudaStream_t s, Recorder *rec) {
     const int n_chunks = D / hagk::Chunk<T>::kElems;
     const hag_device_arrays &d = h->d;
     hagk::GatherArgs a{};
@@ -185,61 +228,64 @@ hag_status fwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
     a.dst_scale = (reduce == HAG_MEAN) ? d.inv_degree : nullptr;
     a.out = out;
     a.D = D;
-    if (use_hag && h->num_agg > 0) {
-        for (int32_t l = 1; l <= h->num_levels; ++l) {
-            hagk::PairArgs p{};
-            p.agg_in = d.agg_in;
-            p.first = int32_t(h->level_ptr[l - 1]);
-            p.count = int32_t(h->level_ptr[l] - h->level_ptr[l - 1]);
-            p.x = x;
-            p.ahat = static_cast<float *>(ws);
-            p.n = h->n;
-            p.D = D;
-            if (p.count <= 0) continue;
-            rec.begin(0, p.count, 2 * int64_t(p.count));
-            if (launch_pairs<T>(p, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
-            rec.end();
+    a.n_prim = std::numeric_limits<int32_t>::max();
+    if (use_hag) {
+        if (h->num_agg > 0) {
+            hag_status st = enqueue_fwd_agg<T>(h, D, x, static_cast<float *>(ws), s, rec);
+            if (st != HAG_OK) return st;
+            a.sec = static_cast<const float *>(ws);
+            a.n_prim = h->n;
         }
         a.row_ptr = d.res_ptr;
         a.idx = d.res_idx;
-        a.sec = static_cast<const float *>(ws);
-        a.n_prim = h->n;
-    } else if (use_hag) {
-        a.row_ptr = d.res_ptr;
-        a.idx = d.res_idx;
-        a.n_prim = std::numeric_limits<int32_t>::max();
     } else {
         a.row_ptr = d.csr_ptr;
         a.idx = d.csr_idx;
-        a.n_prim = std::numeric_limits<int32_t>::max();
     }
     if (h->n > 0) {
-        rec.begin(2, h->n, (use_hag && h->num_agg > 0) ? h->e_res : (use_hag ? h->e_res : h->e));
+        if (rec) rec->begin(2, h->n, use_hag ? h->e_res : h->e);
         if (launch_gather<T>(a, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
-        rec.end();
+        if (rec) rec->end();
     }
     return HAG_OK;
 }
 
-// Backward: gather over the transposed structure.  Aggregation nodes from the
-// last level to the first (their gradient rows live in the workspace), then the
-// graph nodes as sources.  A destination id < n stands for the output row of
-// that graph node (scaled by 1/|N| for mean), an id >= n for an aggregation node.
+// Backward: gather over the transposed structure.  Nodes deeper than bwd_cut take
+// their gradient straight from the graph-node outputs that use them, in one
+// launch; levels bwd_cut..1 follow from the last to the first (their gradient
+// rows live in the workspace); then the graph nodes as sources.  A destination
+// id < n stands for the output row of that graph node (scaled by 1/|N| for
+// mean), an id >= n for an aggregation node.
 template <typename T>
 hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, const void *g, void *gx, void *ws,
-                    cudaStream_t s, Recorder &rec) {
+                    cudaStream_t s, Recorder *rec) {
     const int n_chunks = D / hagk::Chunk<T>::kElems;
     const hag_device_arrays &d = h->d;
     hagk::GatherArgs a{};
     a.prim = g;
     a.src_scale = (reduce == HAG_MEAN) ? d.inv_degree : nullptr;
     a.D = D;
+    a.n_prim = std::numeric_limits<int32_t>::max();
     if (use_hag && h->num_agg > 0) {
+        const int32_t j0 = int32_t(h->level_ptr[h->bwd_cut]);
+        if (j0 < h->num_agg) {
+            hagk::GatherArgs t = a;              // all sources are graph-node outputs
+            t.row_ptr = d.btail_ptr - (h->n + j0);
+            t.idx = d.btail_idx;
+            t.row_begin = h->n + j0;
+            t.row_count = h->num_agg - j0;
+            t.out = ws;
+            t.out_row_offset = h->n;
+            t.out_is_f32 = 1;
+            if (rec) rec->begin(1, t.row_count, int64_t(h->btail_idx.size()));
+            if (launch_gather<T>(t, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+            if (rec) rec->end();
+        }
         a.row_ptr = d.t_ptr;
         a.idx = d.t_idx;
         a.sec = static_cast<const float *>(ws);
         a.n_prim = h->n;
-        for (int32_t l = h->num_levels; l >= 1; --l) {
+        for (int32_t l = h->bwd_cut; l >= 1; --l) {
             hagk::GatherArgs lv = a;
             lv.row_begin = h->n + int32_t(h->level_ptr[l - 1]);
             lv.row_count = int32_t(h->level_ptr[l] - h->level_ptr[l - 1]);
@@ -247,26 +293,24 @@ hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
             lv.out_row_offset = h->n;
             lv.out_is_f32 = 1;
             if (lv.row_count <= 0) continue;
-            rec.begin(1, lv.row_count, h->t_ptr[size_t(lv.row_begin) + lv.row_count] - h->t_ptr[lv.row_begin]);
+            if (rec) rec->begin(1, lv.row_count, h->t_ptr[size_t(lv.row_begin) + lv.row_count] - h->t_ptr[lv.row_begin]);
             if (launch_gather<T>(lv, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
-            rec.end();
+            if (rec) rec->end();
         }
     } else if (use_hag) {
         a.row_ptr = d.t_ptr;
         a.idx = d.t_idx;
-        a.n_prim = std::numeric_limits<int32_t>::max();
     } else {
         a.row_ptr = d.csr_t_ptr;
         a.idx = d.csr_t_idx;
-        a.n_prim = std::numeric_limits<int32_t>::max();
     }
     a.row_begin = 0;
     a.row_count = h->n;
     a.out = gx;
     if (h->n > 0) {
-        rec.begin(2, h->n, use_hag ? h->t_ptr[h->n] : h->e);
+        if (rec) rec->begin(2, h->n, use_hag ? h->t_ptr[h->n] : h->e);
         if (launch_gather<T>(a, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
-        rec.end();
+        if (rec) rec->end();
     }
     return HAG_OK;
 }
@@ -285,11 +329,11 @@ hag_status run(const hag *h, bool backward, bool use_hag, hag_reduce reduce, hag
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     Recorder rec(h, s);
     if (dtype == HAG_F32)
-        st = backward ? bwd_impl<float>(h, use_hag, reduce, D, in, out, ws, s, rec)
-                      : fwd_impl<float>(h, use_hag, reduce, D, in, out, ws, s, rec);
+        st = backward ? bwd_impl<float>(h, use_hag, reduce, D, in, out, ws, s, &rec)
+                      : fwd_impl<float>(h, use_hag, reduce, D, in, out, ws, s, &rec);
     else
-        st = backward ? bwd_impl<__nv_bfloat16>(h, use_hag, reduce, D, in, out, ws, s, rec)
-                      : fwd_impl<__nv_bfloat16>(h, use_hag, reduce, D, in, out, ws, s, rec);
+        st = backward ? bwd_impl<__nv_bfloat16>(h, use_hag, reduce, D, in, out, ws, s, &rec)
+                      : fwd_impl<__nv_bfloat16>(h, use_hag, reduce, D, in, out, ws, s, &rec);
     if (st == HAG_OK && rec.failed) st = HAG_ERR_CUDA;
     return st;
 }
@@ -340,6 +384,10 @@ extern "C" hag_status hag_to_device(hag_t *h, int device) {
     if (st == HAG_OK) st = upload_i32(&d.csr_idx, h->csr_idx.data(), size_t(h->e));
     if (st == HAG_OK) st = upload_i32(&d.csr_t_ptr, h->csr_t_ptr.data(), n + 1);
     if (st == HAG_OK) st = upload_i32(&d.csr_t_idx, h->csr_t_idx.data(), size_t(h->e));
+    if (st == HAG_OK) st = upload_i32(&d.ftail_ptr, h->ftail_ptr.data(), h->ftail_ptr.size());
+    if (st == HAG_OK) st = upload_i32(&d.ftail_idx, h->ftail_idx.data(), h->ftail_idx.size());
+    if (st == HAG_OK) st = upload_i32(&d.btail_ptr, h->btail_ptr.data(), h->btail_ptr.size());
+    if (st == HAG_OK) st = upload_i32(&d.btail_idx, h->btail_idx.data(), h->btail_idx.size());
     if (st == HAG_OK) {
         std::vector<float> inv(std::max<size_t>(n, 1), 1.0f);
         for (size_t v = 0; v < n; ++v) inv[v] = h->in_degree[v] > 0 ? 1.0f / float(h->in_degree[v]) : 1.0f;
@@ -471,35 +519,11 @@ hag_status static_scratch_address(int device, void **out) {
     return HAG_OK;
 }
 
+// The same launch sequence as hag_aggregate_fwd, with no bookkeeping on the handle.
 template <typename T>
 hag_status fwd_static_impl(const hag *h, hag_reduce reduce, int32_t D, const void *x, void *out, float *scratch,
                            cudaStream_t s) {
-    const int n_chunks = D / hagk::Chunk<T>::kElems;
-    const hag_device_arrays &d = h->d;
-    for (int32_t l = 1; l <= h->num_levels; ++l) {
-        hagk::PairArgs p{};
-        p.agg_in = d.agg_in;
-        p.first = int32_t(h->level_ptr[l - 1]);
-        p.count = int32_t(h->level_ptr[l] - h->level_ptr[l - 1]);
-        p.x = x;
-        p.ahat = scratch;
-        p.n = h->n;
-        p.D = D;
-        if (launch_pairs<T>(p, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
-    }
-    hagk::GatherArgs a{};
-    a.row_ptr = d.res_ptr;
-    a.idx = d.res_idx;
-    a.row_begin = 0;
-    a.row_count = h->n;
-    a.prim = x;
-    a.sec = scratch;
-    a.n_prim = h->num_agg > 0 ? h->n : std::numeric_limits<int32_t>::max();
-    a.dst_scale = (reduce == HAG_MEAN) ? d.inv_degree : nullptr;
-    a.out = out;
-    a.D = D;
-    if (launch_gather<T>(a, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
-    return HAG_OK;
+    return fwd_impl<T>(h, true, reduce, D, x, out, scratch, s, nullptr);
 }
 
 }  // namespace

@@ -20,6 +20,8 @@ struct hag_device_arrays {
     int32_t *csr_idx = nullptr;    // [e]
     int32_t *csr_t_ptr = nullptr;  // [n+1]
     int32_t *csr_t_idx = nullptr;  // [e]
+    int32_t *ftail_ptr = nullptr, *ftail_idx = nullptr;   // forward expansion of the deep levels
+    int32_t *btail_ptr = nullptr, *btail_idx = nullptr;   // backward expansion
     float *inv_degree = nullptr;   // [n] 1/|N(v)| (1 for empty rows)
     // staging for the host-buffer entry point
     void *stage_in = nullptr;
@@ -43,6 +45,10 @@ struct hag {
     std::vector<int32_t> res_idx;
     std::vector<int64_t> t_ptr;      // n + num_agg + 1
     std::vector<int32_t> t_idx;
+    // deep levels expanded (one launch each way)
+    int32_t fwd_cut = 0, bwd_cut = 0;
+    std::vector<int64_t> ftail_ptr, btail_ptr;
+    std::vector<int32_t> ftail_idx, btail_idx;
     hag_info info{};
     int device = -1;
     hag_device_arrays d;

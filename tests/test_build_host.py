@@ -34,6 +34,9 @@ def _same_structure(g, capacity, search=O.greedy_pairmap):
         assert got.dtype == want.dtype and np.array_equal(got, want), key
     t_ptr, t_idx = O.transposed_csr(g.row_ptr, g.col_idx)
     assert np.array_equal(arr["csr_t_ptr"], t_ptr) and np.array_equal(arr["csr_t_idx"], t_idx)
+    tails = O.expanded_tails(ref)
+    for key, want in tails.items():
+        assert np.array_equal(arr[key], want), key
     info = h.info()
     c = O.counters(g.row_ptr, ref)
     assert info["n"] == g.n and info["e"] == c["e"] and info["e_hat"] == c["e_hat"]

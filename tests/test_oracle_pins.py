@@ -328,3 +328,35 @@ def test_integer_features_are_exact():
     a, _ = O.direct_forward(g.row_ptr, g.col_idx, x, "sum")
     assert np.array_equal(O.hag_forward(h, x, "sum"), a)
     assert np.array_equal(a, np.rint(a))
+
+
+def test_expanded_deep_levels_are_covers_and_transitive_users():
+    """The expansion lists must reproduce the level-by-level values: the forward list of a deep
+    node sums to its a-hat, the backward list of a deep node to its gradient."""
+    g = synth.clique_union_graph(seed=16, n=500, n_groups=140, g_lo=3, g_hi=30)
+    res = O.greedy_pairmap(g.row_ptr, g.col_idx, g.n // 2)
+    h = O.canonical_hag(g.row_ptr, res)
+    assert h.num_levels >= 4
+    t = O.expanded_tails(h)
+    rng = np.random.default_rng(0)
+    x = rng.integers(-5, 6, size=(g.n, 3)).astype(np.float64)
+    ahat = np.concatenate([x, np.zeros((h.num_agg, 3))])
+    for j in range(h.num_agg):
+        ahat[g.n + j] = ahat[h.agg_in[2 * j]] + ahat[h.agg_in[2 * j + 1]]
+    j0 = int(h.level_ptr[t["fwd_cut"]])
+    for i in range(h.num_agg - j0):
+        ids = t["ftail_idx"][t["ftail_ptr"][i]: t["ftail_ptr"][i + 1]]
+        assert len(set(ids.tolist())) == len(ids)
+        assert np.array_equal(ahat[ids].sum(0), ahat[g.n + j0 + i])
+    gr = rng.integers(-5, 6, size=(g.n, 3)).astype(np.float64)
+    ghat = np.zeros((h.num_agg, 3))
+    for j in range(h.num_agg - 1, -1, -1):
+        for d in h.t_idx[h.t_ptr[g.n + j]: h.t_ptr[g.n + j + 1]]:
+            ghat[j] += gr[d] if d < g.n else ghat[d - g.n]
+    j0 = int(h.level_ptr[t["bwd_cut"]])
+    for i in range(h.num_agg - j0):
+        ids = t["btail_idx"][t["btail_ptr"][i]: t["btail_ptr"][i + 1]]
+        assert (ids < g.n).all() and len(set(ids.tolist())) == len(ids)
+        assert np.array_equal(gr[ids].sum(0), ghat[j0 + i])
+    # a small graph never pays for a launch per level: everything deeper than the cut is expanded
+    assert t["fwd_cut"] < h.num_levels and t["bwd_cut"] < h.num_levels
