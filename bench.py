@@ -182,8 +182,8 @@ def run_reference(args, w, bytes_per_step_fn):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=2, help="1-5; 2 is the 50 000-node clustered power-law graph")
     ap.add_argument("--scale", type=float, default=1.0)
@@ -215,6 +215,7 @@ def main():
     import torch.distributed as dist
 
     import paper_1906_03707_b200 as hb
+    from paper_1906_03707_b200 import sharding
     from paper_1906_03707_b200.build import build as build_library
 
     build_library()
@@ -282,11 +283,7 @@ def main():
             launches += step(hag)
             stops[i].record(stream)
         barrier()
-        ms = sum(a.elapsed_time(b) for a, b in zip(starts, stops))
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = sharding.max_over_ranks(sum(a.elapsed_time(b) for a, b in zip(starts, stops)), dev)
         return ms / max(steps, 1), launches
 
     for _ in range(args.warmup):
@@ -296,10 +293,11 @@ def main():
     if rank == 0:
         sampler.start()
     hag_ms, launches = timed(True, args.steps, cold=True)
-    clocks = sampler.stop() if rank == 0 else {}
     csr_ms, _ = timed(False, args.steps, cold=True)
     hag_warm_ms, _ = timed(True, args.steps, cold=False)
     csr_warm_ms, _ = timed(False, args.steps, cold=False)
+    # a timed arm lasts milliseconds, far below nvidia-smi's sampling period: the sampler runs across all four arms
+    clocks = sampler.stop() if rank == 0 else {}
 
     # the dominant kernel, timed live with event pairs around every launch
     h.profile(True)
@@ -354,11 +352,7 @@ def main():
             host_step()
         e1.record(stream)
         barrier()
-        e2e_ms = e0.elapsed_time(e1) / max(args.steps, 1)
-        if world > 1:
-            t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = sharding.max_over_ranks(e0.elapsed_time(e1) / max(args.steps, 1), dev)
         io = 2 * w.layers * x.numel() * x.element_size()
         e2e = {"value": world * 2 * w.layers * nbytes["hag_pass"] / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s",
                "h2d_bytes_per_step": io, "d2h_bytes_per_step": io, "ms_per_step": e2e_ms,
@@ -394,6 +388,7 @@ def main():
                             f"|V_A|={info['num_agg']} (capacity {w.capacity}), {w.layers} layer(s), fwd+bwd",
                 "l2": "flushed between timed steps (256 MiB write outside the per-step events)",
                 "timing": "sum of per-step CUDA-event intervals on the launching stream, max over ranks",
+                "clocks": "nvidia-smi sampled every 100 ms across the four timed arms (HAG/plain x cold/warm)",
             },
             "clocks": clocks,
             "e2e": e2e,

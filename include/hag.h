@@ -130,6 +130,16 @@ typedef struct hag_arrays {
  * 2^31); HAG_ERR_GRAPH; HAG_ERR_OOM_HOST.  On error *out is NULL. */
 hag_status hag_build(int32_t n, const int64_t *row_ptr, const int32_t *col_idx, int32_t capacity, hag_t **out);
 
+/* The HAG the same graph would get with a smaller capacity (the capacity study of
+ * Section 5.4 without repeating the search): Algorithm 3 adds one node per
+ * iteration, so its result for capacity c is its first c merges.  Replays the
+ * first min(capacity, |V_A|) merges recorded in `src` and lays the result out;
+ * *out equals hag_build(graph, capacity) bit for bit.  `src` is unchanged and the
+ * new handle is independent of it (host only until hag_to_device).
+ * HAG_ERR_ARG if capacity < 0, or if capacity exceeds the recorded merges while
+ * `src` stopped only because it hit its own capacity. */
+hag_status hag_truncate(const hag_t *src, int32_t capacity, hag_t **out);
+
 /* Frees host and device arrays.  NULL is allowed. */
 hag_status hag_destroy(hag_t *h);
 

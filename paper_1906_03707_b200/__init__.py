@@ -24,7 +24,7 @@ HAG_SUM, HAG_MEAN = 0, 1
 HAG_F32, HAG_BF16 = 0, 1
 
 EXPORTED_SYMBOLS = [
-    "hag_build", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes",
+    "hag_build", "hag_truncate", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes",
     "hag_aggregate_fwd", "hag_aggregate_bwd", "csr_aggregate_fwd", "csr_aggregate_bwd",
     "hag_aggregate_host", "hag_aggregate_fwd_static", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
 ]
@@ -75,6 +75,8 @@ def load_library():
     vp, i32 = ctypes.c_void_p, ctypes.c_int32
     lib.hag_build.argtypes = [i32, vp, vp, i32, ctypes.POINTER(vp)]
     lib.hag_build.restype = ctypes.c_int
+    lib.hag_truncate.argtypes = [vp, i32, ctypes.POINTER(vp)]
+    lib.hag_truncate.restype = ctypes.c_int
     lib.hag_destroy.argtypes = [vp]
     lib.hag_destroy.restype = ctypes.c_int
     lib.hag_get_info.argtypes = [vp, ctypes.POINTER(HagInfo)]
@@ -152,6 +154,12 @@ class Hag:
         st = lib.hag_build(n, rp.ctypes.data, ci.ctypes.data if ci.size else None, int(capacity), ctypes.byref(handle))
         _check(st, "hag_build")
         return cls(handle)
+
+    def truncate(self, capacity: int) -> "Hag":
+        """``hag_truncate``: the HAG of the same graph for a smaller capacity, from the recorded merges."""
+        handle = ctypes.c_void_p()
+        _check(load_library().hag_truncate(self._h, int(capacity), ctypes.byref(handle)), "hag_truncate")
+        return Hag(handle)
 
     def close(self):
         if self._h:

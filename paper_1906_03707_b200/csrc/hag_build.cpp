@@ -68,7 +68,21 @@ struct Searcher {
         }
     }
 
-    hag_status run(std::vector<int32_t> &trace) {
+    // Re-applies the first `count` merges of a recorded trace (no search).
+    hag_status replay(const std::vector<int32_t> &src, int64_t count, std::vector<int32_t> &trace) {
+        init_lists();
+        for (int64_t i = 0; i < count; ++i) {
+            const int32_t x = src[3 * i], p = src[3 * i + 1], k = src[3 * i + 2];
+            if (!(0 <= x && x < p && p < n + i)) return HAG_ERR_ARG;
+            intersect_users(x, p);
+            if (int32_t(users.size()) != k) return HAG_ERR_ARG;
+            int32_t wbest, warg;
+            apply_merge(x, p, i, trace, wbest, warg);
+        }
+        return HAG_OK;
+    }
+
+    void init_lists() {
         const int64_t n_ids = int64_t(n) + cap;
         const int64_t e = row_ptr[n];
         out_ptr.assign(n_ids, nullptr);
@@ -91,6 +105,71 @@ struct Searcher {
                     out_ptr[s][out_len[s]++] = u;
                 }
         }
+    }
+
+    // users <- the graph nodes that hold both x and p
+    void intersect_users(int32_t x, int32_t p) {
+        users.clear();
+        const int32_t *a = out_ptr[x], *b = out_ptr[p];
+        int32_t i = 0, j = 0;
+        const int32_t la = out_len[x], lb = out_len[p];
+        while (i < la && j < lb) {
+            if (a[i] < b[j]) ++i;
+            else if (a[i] > b[j]) ++j;
+            else { users.push_back(a[i]); ++i; ++j; }
+        }
+    }
+
+    // Merge (x, p) with the users already in `users` into node n + num: rewrites the
+    // rows and user lists, marks what became stale, returns the new node's exact key.
+    void apply_merge(int32_t x, int32_t p, int64_t num, std::vector<int32_t> &trace, int32_t &wbest, int32_t &warg) {
+        const int32_t w = int32_t(n + num);
+        trace.push_back(x);
+        trace.push_back(p);
+        trace.push_back(int32_t(users.size()));
+        // rewrite the users' rows; count what else they hold (= the new node's pair counts)
+        touched.clear();
+        for (int32_t u : users) {
+            int32_t *row = rows.data() + row_ptr[u];
+            const int32_t l = row_len[u];
+            int32_t o = 0;
+            for (int32_t j = 0; j < l; ++j) {
+                const int32_t y = row[j];
+                if (y == x || y == p) continue;
+                row[o++] = y;
+                if (cnt[y]++ == 0) touched.push_back(y);
+            }
+            row[o++] = w;                       // larger than every existing id: row stays sorted
+            row_len[u] = o;
+        }
+        wbest = 0;
+        warg = -1;
+        for (int32_t y : touched) {
+            const int32_t c = cnt[y];
+            cnt[y] = 0;
+            if (c > wbest || (c == wbest && y < warg)) { wbest = c; warg = y; }
+            if (!dirty[y] && (partner[y] == x || partner[y] == p)) dirty[y] = 1;
+        }
+        // user lists: x and p lose U, w gets it
+        for (int32_t s : {x, p}) {
+            int32_t *l = out_ptr[s];
+            const int32_t len = out_len[s];
+            int32_t o = 0;
+            size_t q = 0;
+            for (int32_t i = 0; i < len; ++i) {
+                while (q < users.size() && users[q] < l[i]) ++q;
+                if (q < users.size() && users[q] == l[i]) continue;
+                l[o++] = l[i];
+            }
+            out_len[s] = o;
+        }
+        out_new[num] = users;
+        out_ptr[w] = out_new[num].data();
+        out_len[w] = int32_t(users.size());
+    }
+
+    hag_status run(std::vector<int32_t> &trace) {
+        init_lists();
         // a pair cannot be shared by more rows than either member has users
         for (int32_t s = 0; s < n; ++s) {
             key[s] = out_len[s];
@@ -116,66 +195,18 @@ struct Searcher {
             }
             const int32_t p = partner[x];
             if (p <= x) return HAG_ERR_ARG;         // cannot happen (see header comment)
-            // users of the pair
-            users.clear();
-            {
-                const int32_t *a = out_ptr[x], *b = out_ptr[p];
-                int32_t i = 0, j = 0;
-                const int32_t la = out_len[x], lb = out_len[p];
-                while (i < la && j < lb) {
-                    if (a[i] < b[j]) ++i;
-                    else if (a[i] > b[j]) ++j;
-                    else { users.push_back(a[i]); ++i; ++j; }
-                }
-            }
+            intersect_users(x, p);
             if (int32_t(users.size()) != k) return HAG_ERR_ARG;  // internal inconsistency
+            int32_t wbest, warg;
+            apply_merge(x, p, num, trace, wbest, warg);
             const int32_t w = int32_t(n + num);
-            trace.push_back(x);
-            trace.push_back(p);
-            trace.push_back(k);
-            // rewrite the users' rows; count what else they hold (= the new node's pair counts)
-            touched.clear();
-            for (int32_t u : users) {
-                int32_t *row = rows.data() + row_ptr[u];
-                const int32_t l = row_len[u];
-                int32_t o = 0;
-                for (int32_t j = 0; j < l; ++j) {
-                    const int32_t y = row[j];
-                    if (y == x || y == p) continue;
-                    row[o++] = y;
-                    if (cnt[y]++ == 0) touched.push_back(y);
-                }
-                row[o++] = w;                       // larger than every existing id: row stays sorted
-                row_len[u] = o;
-            }
-            int32_t wbest = 0, warg = -1;
-            for (int32_t y : touched) {
-                const int32_t c = cnt[y];
-                cnt[y] = 0;
-                if (c > wbest || (c == wbest && y < warg)) { wbest = c; warg = y; }
-                if (!dirty[y] && (partner[y] == x || partner[y] == p)) dirty[y] = 1;
-            }
-            // user lists: x and p lose U, w gets it
             for (int32_t s : {x, p}) {
-                int32_t *l = out_ptr[s];
-                const int32_t len = out_len[s];
-                int32_t o = 0;
-                size_t q = 0;
-                for (int32_t i = 0; i < len; ++i) {
-                    while (q < users.size() && users[q] < l[i]) ++q;
-                    if (q < users.size() && users[q] == l[i]) continue;
-                    l[o++] = l[i];
-                }
-                out_len[s] = o;
                 dirty[s] = 1;                        // every pair with x or p changed
-                const int32_t bound = std::min(key[s], o);
+                const int32_t bound = std::min(key[s], out_len[s]);
                 // x's entry was popped; p still has one unless its bound moved
                 if ((s == x || bound != key[s]) && bound >= 2) pq.push(enc(bound, s));
                 key[s] = bound;
             }
-            out_new[num] = users;
-            out_ptr[w] = out_new[num].data();
-            out_len[w] = int32_t(users.size());
             key[w] = wbest;
             partner[w] = warg;
             dirty[w] = 0;
@@ -430,6 +461,45 @@ extern "C" hag_status hag_build(int32_t n, const int64_t *row_ptr, const int32_t
         for (int32_t v = 0; v < n; ++v) h->in_degree[v] = int32_t(row_ptr[v + 1] - row_ptr[v]);
         std::vector<int32_t> rows_store, rows_len;
         st = hag_search(h, rows_store, rows_len);
+        if (st == HAG_OK) st = hag_layout(h, rows_store, rows_len);
+    } catch (const std::bad_alloc &) {
+        st = HAG_ERR_OOM_HOST;
+    }
+    if (st != HAG_OK) {
+        delete h;
+        return st;
+    }
+    h->info.build_seconds = std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count();
+    *out = h;
+    return HAG_OK;
+}
+
+extern "C" hag_status hag_truncate(const hag_t *src, int32_t capacity, hag_t **out) {
+    if (!out) return HAG_ERR_NULL;
+    *out = nullptr;
+    if (!src) return HAG_ERR_NULL;
+    if (capacity < 0) return HAG_ERR_ARG;
+    // beyond the recorded merges the answer is known only if the search ended by itself
+    if (capacity > src->num_agg && src->num_agg == src->capacity) return HAG_ERR_ARG;
+    const auto t0 = std::chrono::steady_clock::now();
+    hag *h = new (std::nothrow) hag();
+    if (!h) return HAG_ERR_OOM_HOST;
+    hag_status st = HAG_OK;
+    try {
+        const int32_t k = std::min(capacity, src->num_agg);
+        h->n = src->n;
+        h->capacity = capacity;
+        h->e = src->e;
+        h->csr_ptr = src->csr_ptr;
+        h->csr_idx = src->csr_idx;
+        h->in_degree = src->in_degree;
+        std::vector<int32_t> rows_store = h->csr_idx, rows_len(h->n);
+        for (int32_t u = 0; u < h->n; ++u) rows_len[u] = int32_t(h->csr_ptr[u + 1] - h->csr_ptr[u]);
+        if (k > 0) {
+            Searcher s(h->n, k, h->csr_ptr.data(), rows_store, rows_len);
+            st = s.replay(src->trace, k, h->trace);
+        }
+        h->num_agg = int32_t(h->trace.size() / 3);
         if (st == HAG_OK) st = hag_layout(h, rows_store, rows_len);
     } catch (const std::bad_alloc &) {
         st = HAG_ERR_OOM_HOST;

@@ -80,26 +80,21 @@ cudaError_t launch_pdl(void (*kernel)(Args), unsigned grid, const Args &args, cu
     return cudaLaunchKernelEx(&cfg, kernel, args);
 }
 
-int g_tune = 0;
-int tune_variant() { return g_tune; }
+// Launch shape of the gather, from measurements on B200 (resident warps beat
+// loads per warp once there are enough rows to fill the machine):
+//   fp32, >= 131072 rows : 2 loads in flight per lane, 64 warps per SM
+//   fp32, fewer rows     : 8 loads in flight per lane, 32 warps per SM (fewer rounds per row: latency bound)
+//   bf16                 : 2 loads in flight per lane, 48 warps per SM
+constexpr int32_t kManyRows = 131072;
 
 template <typename T, int LPR, bool SS>
 cudaError_t launch_gather_lpr(const hagk::GatherArgs &a, cudaStream_t s) {
     const unsigned grid = unsigned((a.row_count + hagk::kWarps - 1) / hagk::kWarps);
     if constexpr (sizeof(T) == 4) {
-        switch (tune_variant()) {
-            case 1: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 8, SS, 6>, grid, a, s);
-            case 2: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 16, SS, 4>, grid, a, s);
-            case 3: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 12>, grid, a, s);
-            default: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 8, SS, 8>, grid, a, s);
-        }
+        if (a.row_count >= kManyRows) return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 16>, grid, a, s);
+        return launch_pdl(hagk::gather_sum_kernel<T, LPR, 8, SS, 8>, grid, a, s);
     } else {
-        switch (tune_variant()) {
-            case 1: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 8, SS, 4>, grid, a, s);
-            case 2: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 6>, grid, a, s);
-            case 3: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 12>, grid, a, s);
-            default: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 8>, grid, a, s);
-        }
+        return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 12>, grid, a, s);
     }
 }
 
@@ -543,5 +538,3 @@ extern "C" hag_status hag_aggregate_fwd_static(const hag_t *h, hag_reduce reduce
     if (dtype == HAG_F32) return fwd_static_impl<float>(h, reduce, D, x, out, static_cast<float *>(scratch), s);
     return fwd_static_impl<__nv_bfloat16>(h, reduce, D, x, out, static_cast<float *>(scratch), s);
 }
-
-extern "C" void hag_debug_set_tune(int v) { g_tune = v; }

@@ -171,3 +171,31 @@ def test_argument_and_graph_validation():
     assert lib.hag_workspace_bytes(None, 4) == 0 and lib.hag_last_launch_count(None) == 0
     assert hb.status_str(3).startswith("malformed") and hb.status_str(99) == "unknown status"
     assert lib.hag_destroy(None) == 0
+
+
+def test_truncate_equals_a_fresh_build_with_the_smaller_capacity():
+    import hashlib
+
+    def digest(h):
+        arr = h.arrays()
+        dig = hashlib.sha256()
+        for k in sorted(arr):
+            dig.update(np.ascontiguousarray(arr[k]).tobytes() if hasattr(arr[k], "tobytes") else str(arr[k]).encode())
+        info = {k: v for k, v in h.info().items() if k != "build_seconds"}
+        return dig.hexdigest(), info
+
+    g = synth.config5_graph(seed=14, n=4000, n_comm=12, s_lo=60, s_hi=900, d_lo=8, d_hi=150)
+    full = hb.Hag.build(g.row_ptr, g.col_idx, g.n // 2)
+    assert full.info()["num_agg"] == g.n // 2
+    for cap in (0, 1, g.n // 8, g.n // 4, g.n // 2):
+        assert digest(full.truncate(cap)) == digest(hb.Hag.build(g.row_ptr, g.col_idx, cap)), cap
+    lib = hb.load_library()
+    out = ctypes.c_void_p()
+    assert lib.hag_truncate(full._h, g.n, ctypes.byref(out)) == 2      # the search was cut off by its capacity
+    assert lib.hag_truncate(full._h, -1, ctypes.byref(out)) == 2
+    assert lib.hag_truncate(None, 1, ctypes.byref(out)) == 1 and lib.hag_truncate(full._h, 1, None) == 1
+    # a search that ended by itself knows the answer for any larger capacity
+    ring = synth.csr_from_rows([[1, 3], [0, 2], [1, 3], [0, 2]])
+    done = hb.Hag.build(ring.row_ptr, ring.col_idx, 100)
+    assert done.info()["num_agg"] == 2
+    assert digest(done.truncate(50))[0] == digest(hb.Hag.build(ring.row_ptr, ring.col_idx, 50))[0]

@@ -226,7 +226,7 @@ def test_device_call_errors_are_statuses():
     assert lib.hag_to_device(h._h, 10_000) == 2
 
 
-@pytest.mark.parametrize("index", [2, 4])
+@pytest.mark.parametrize("index", [2, 4, 3, 5])
 def test_full_size_workloads_sampled_rows(index):
     """The benchmark's launch configuration at full size; the oracle computes sampled rows one by one."""
     w = synth.workload(index)
