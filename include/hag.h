@@ -130,6 +130,12 @@ typedef struct hag_arrays {
  * 2^31); HAG_ERR_GRAPH; HAG_ERR_OOM_HOST.  On error *out is NULL. */
 hag_status hag_build(int32_t n, const int64_t *row_ptr, const int32_t *col_idx, int32_t capacity, hag_t **out);
 
+/* Host threads hag_build may use for recounting pair redundancies (process-wide).
+ * 0 = as many as the host has, at most 16 (the default); 1 = single-threaded;
+ * a negative value only queries.  Returns the previous setting.  The merge
+ * sequence, and so every array of the result, does not depend on it. */
+int32_t hag_build_threads(int32_t threads);
+
 /* The HAG the same graph would get with a smaller capacity (the capacity study of
  * Section 5.4 without repeating the search): Algorithm 3 adds one node per
  * iteration, so its result for capacity c is its first c merges.  Replays the

@@ -24,7 +24,7 @@ HAG_SUM, HAG_MEAN = 0, 1
 HAG_F32, HAG_BF16 = 0, 1
 
 EXPORTED_SYMBOLS = [
-    "hag_build", "hag_truncate", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes",
+    "hag_build", "hag_build_threads", "hag_truncate", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes",
     "hag_aggregate_fwd", "hag_aggregate_bwd", "csr_aggregate_fwd", "csr_aggregate_bwd",
     "hag_aggregate_host", "hag_aggregate_fwd_static", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
 ]
@@ -75,6 +75,8 @@ def load_library():
     vp, i32 = ctypes.c_void_p, ctypes.c_int32
     lib.hag_build.argtypes = [i32, vp, vp, i32, ctypes.POINTER(vp)]
     lib.hag_build.restype = ctypes.c_int
+    lib.hag_build_threads.argtypes = [i32]
+    lib.hag_build_threads.restype = i32
     lib.hag_truncate.argtypes = [vp, i32, ctypes.POINTER(vp)]
     lib.hag_truncate.restype = ctypes.c_int
     lib.hag_destroy.argtypes = [vp]
@@ -109,6 +111,11 @@ def load_library():
     lib.hag_status_str.restype = ctypes.c_char_p
     _lib = lib
     return lib
+
+
+def build_threads(threads: int = -1) -> int:
+    """``hag_build_threads``: set (>= 0) or query (< 0) the host threads of the search; returns the previous value."""
+    return int(load_library().hag_build_threads(int(threads)))
 
 
 def status_str(status: int) -> str:

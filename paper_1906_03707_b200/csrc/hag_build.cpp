@@ -16,15 +16,23 @@
 // arg-max with the required tie-break (its partner is the smallest id attaining
 // the count, and is larger than the node itself, otherwise the partner would
 // have been on top).  Memory is O(|E|).
+// Recounts are nine tenths of the time and independent of each other while no
+// merge happens, so a run of stale nodes at the top of the queue is recounted
+// by a pool of threads at once.  Recounting a stale node early only tightens a
+// bound sooner: the merge sequence is the same for any number of threads.
 #include <algorithm>
+#include <atomic>
 #include <chrono>
 #include <cstring>
 #include <new>
 #include <queue>
+#include <thread>
 
 #include "hag_internal.h"
 
 namespace {
+
+std::atomic<int> g_build_threads{0};   // 0 = as many as the host has, at most 16
 
 struct Searcher {
     int32_t n;
@@ -46,8 +54,8 @@ struct Searcher {
 
     static uint64_t enc(int32_t k, int32_t id) { return (uint64_t(uint32_t(k)) << 32) | uint32_t(0x7fffffff - id); }
 
-    // exact max_b Redundancy(x, b) and the smallest b attaining it
-    void recount(int32_t x, int32_t &best, int32_t &arg) {
+    // exact max_b Redundancy(x, b) and the smallest b attaining it (reads shared state only)
+    void recount(int32_t x, int32_t &best, int32_t &arg, std::vector<int32_t> &cnt, std::vector<int32_t> &touched) const {
         touched.clear();
         const int32_t *ou = out_ptr[x];
         for (int32_t i = 0, m = out_len[x]; i < m; ++i) {
@@ -168,8 +176,73 @@ struct Searcher {
         out_len[w] = int32_t(users.size());
     }
 
-    hag_status run(std::vector<int32_t> &trace) {
+    // ---- pool for batches of recounts ----
+    int n_threads = 1;
+    std::vector<std::thread> workers;
+    std::vector<std::vector<int32_t>> w_cnt, w_touched;   // scratch per worker (index 0 = calling thread)
+    std::vector<int32_t> batch, batch_best, batch_arg;
+    std::atomic<int64_t> generation{0};
+    std::atomic<int32_t> next_task{0}, tasks_done{0}, acks{0};
+    std::atomic<bool> stop{false};
+
+    void work_on_batch(int self) {
+        const int32_t total = int32_t(batch.size());
+        for (;;) {
+            const int32_t i = next_task.fetch_add(1, std::memory_order_relaxed);
+            if (i >= total) break;
+            recount(batch[i], batch_best[i], batch_arg[i], w_cnt[self], w_touched[self]);
+            tasks_done.fetch_add(1, std::memory_order_release);
+        }
+    }
+    void worker_loop(int self) {
+        int64_t seen = 0;
+        for (;;) {
+            int spins = 0;
+            while (generation.load(std::memory_order_acquire) == seen) {
+                if (stop.load(std::memory_order_acquire)) return;
+                if (++spins > 2000) std::this_thread::yield();
+            }
+            seen = generation.load(std::memory_order_acquire);
+            work_on_batch(self);
+            acks.fetch_add(1, std::memory_order_release);   // this worker no longer touches the batch
+        }
+    }
+    void start_pool(int threads) {
+        n_threads = std::max(1, threads);
+        w_cnt.assign(n_threads, std::vector<int32_t>());
+        w_touched.assign(n_threads, std::vector<int32_t>());
+        for (int t = 0; t < n_threads; ++t) w_cnt[t].assign(size_t(n) + cap, 0);
+        for (int t = 1; t < n_threads; ++t) workers.emplace_back([this, t] { worker_loop(t); });
+    }
+    void stop_pool() {
+        stop.store(true, std::memory_order_release);
+        for (auto &t : workers) t.join();
+        workers.clear();
+    }
+    // recounts every node of `batch` (all threads), results in batch_best / batch_arg
+    void recount_batch() {
+        const int32_t total = int32_t(batch.size());
+        batch_best.assign(total, 0);
+        batch_arg.assign(total, -1);
+        next_task.store(0, std::memory_order_relaxed);
+        tasks_done.store(0, std::memory_order_relaxed);
+        const bool shared = n_threads > 1 && total > 1;
+        if (shared) {
+            acks.store(0, std::memory_order_relaxed);
+            generation.fetch_add(1, std::memory_order_release);
+        }
+        work_on_batch(0);
+        while (tasks_done.load(std::memory_order_acquire) < total) std::this_thread::yield();
+        // the batch vectors are rebuilt next: wait until every worker has left this one
+        if (shared)
+            while (acks.load(std::memory_order_acquire) < n_threads - 1) std::this_thread::yield();
+    }
+    ~Searcher() { stop_pool(); }
+
+    hag_status run(std::vector<int32_t> &trace, int threads) {
         init_lists();
+        start_pool(threads);
+        const size_t max_batch = size_t(4) * n_threads;
         // a pair cannot be shared by more rows than either member has users
         for (int32_t s = 0; s < n; ++s) {
             key[s] = out_len[s];
@@ -185,12 +258,31 @@ struct Searcher {
             if (k != key[x]) continue;              // superseded entry
             if (k < 2) break;
             if (dirty[x]) {
-                int32_t m, p;
-                recount(x, m, p);
-                key[x] = m;
-                partner[x] = p;
-                dirty[x] = 0;
-                if (m >= 2) pq.push(enc(m, x));
+                // gather the run of stale nodes at the top of the queue and recount them together
+                batch.clear();
+                batch.push_back(x);
+                while (batch.size() < max_batch && !pq.empty()) {
+                    const uint64_t t2 = pq.top();
+                    const int32_t k2 = int32_t(t2 >> 32);
+                    const int32_t x2 = int32_t(0x7fffffff - uint32_t(t2 & 0xffffffffu));
+                    if (k2 != key[x2]) { pq.pop(); continue; }      // superseded entry
+                    if (!dirty[x2] || k2 < 2) break;                // a clean node: stop before it
+                    pq.pop();
+                    dirty[x2] = 2;                                  // in the batch (guards against duplicate entries)
+                    batch.push_back(x2);
+                }
+                dirty[x] = 2;
+                // drop duplicates of one node (several live entries with the same key)
+                std::sort(batch.begin(), batch.end());
+                batch.erase(std::unique(batch.begin(), batch.end()), batch.end());
+                recount_batch();
+                for (size_t i = 0; i < batch.size(); ++i) {
+                    const int32_t y = batch[i];
+                    key[y] = batch_best[i];
+                    partner[y] = batch_arg[i];
+                    dirty[y] = 0;
+                    if (key[y] >= 2) pq.push(enc(key[y], y));
+                }
                 continue;
             }
             const int32_t p = partner[x];
@@ -227,7 +319,9 @@ hag_status hag_search(hag *h, std::vector<int32_t> &rows_store, std::vector<int3
         h->trace.clear();
         if (h->capacity == 0 || h->n == 0) return HAG_OK;
         Searcher s(h->n, h->capacity, h->csr_ptr.data(), rows_store, rows_len);
-        hag_status st = s.run(h->trace);
+        int threads = g_build_threads.load();
+        if (threads <= 0) threads = int(std::min<unsigned>(std::max<unsigned>(std::thread::hardware_concurrency(), 1u), 16u));
+        hag_status st = s.run(h->trace, threads);
         if (st != HAG_OK) return st;
     } catch (const std::bad_alloc &) {
         return HAG_ERR_OOM_HOST;
@@ -472,6 +566,12 @@ extern "C" hag_status hag_build(int32_t n, const int64_t *row_ptr, const int32_t
     h->info.build_seconds = std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count();
     *out = h;
     return HAG_OK;
+}
+
+extern "C" int32_t hag_build_threads(int32_t threads) {
+    const int prev = g_build_threads.load();
+    if (threads >= 0) g_build_threads.store(threads);
+    return prev;
 }
 
 extern "C" hag_status hag_truncate(const hag_t *src, int32_t capacity, hag_t **out) {

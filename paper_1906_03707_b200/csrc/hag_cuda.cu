@@ -87,9 +87,24 @@ cudaError_t launch_pdl(void (*kernel)(Args), unsigned grid, const Args &args, cu
 //   bf16                 : 2 loads in flight per lane, 48 warps per SM
 constexpr int32_t kManyRows = 131072;
 
+#ifdef HAG_TUNING
+int g_tune = -1;   // tuning builds only: force a launch shape
+#endif
+
 template <typename T, int LPR, bool SS>
 cudaError_t launch_gather_lpr(const hagk::GatherArgs &a, cudaStream_t s) {
     const unsigned grid = unsigned((a.row_count + hagk::kWarps - 1) / hagk::kWarps);
+#ifdef HAG_TUNING
+    switch (g_tune) {
+        case 0: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 8, SS, 8>, grid, a, s);
+        case 1: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 8>, grid, a, s);
+        case 2: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 12>, grid, a, s);
+        case 3: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 12>, grid, a, s);
+        case 4: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 16>, grid, a, s);
+        case 5: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 10>, grid, a, s);
+        default: break;
+    }
+#endif
     if constexpr (sizeof(T) == 4) {
         if (a.row_count >= kManyRows) return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 16>, grid, a, s);
         return launch_pdl(hagk::gather_sum_kernel<T, LPR, 8, SS, 8>, grid, a, s);
@@ -538,3 +553,7 @@ extern "C" hag_status hag_aggregate_fwd_static(const hag_t *h, hag_reduce reduce
     if (dtype == HAG_F32) return fwd_static_impl<float>(h, reduce, D, x, out, static_cast<float *>(scratch), s);
     return fwd_static_impl<__nv_bfloat16>(h, reduce, D, x, out, static_cast<float *>(scratch), s);
 }
+
+#ifdef HAG_TUNING
+extern "C" void hag_debug_set_tune(int v) { g_tune = v; }
+#endif

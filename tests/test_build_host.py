@@ -199,3 +199,18 @@ def test_truncate_equals_a_fresh_build_with_the_smaller_capacity():
     done = hb.Hag.build(ring.row_ptr, ring.col_idx, 100)
     assert done.info()["num_agg"] == 2
     assert digest(done.truncate(50))[0] == digest(hb.Hag.build(ring.row_ptr, ring.col_idx, 50))[0]
+
+
+def test_build_does_not_depend_on_the_thread_count():
+    g = synth.config2_graph(seed=17, n=6000, n_comm=40)
+    prev = hb.build_threads(1)
+    try:
+        one = hb.Hag.build(g.row_ptr, g.col_idx, g.n // 4).arrays()
+        for threads in (2, 5, 0):
+            hb.build_threads(threads)
+            many = hb.Hag.build(g.row_ptr, g.col_idx, g.n // 4).arrays()
+            for k, v in one.items():
+                assert np.array_equal(np.asarray(v), np.asarray(many[k])), (threads, k)
+        assert hb.build_threads(-1) == 0
+    finally:
+        hb.build_threads(prev)
