@@ -80,11 +80,13 @@ cudaError_t launch_pdl(void (*kernel)(Args), unsigned grid, const Args &args, cu
     return cudaLaunchKernelEx(&cfg, kernel, args);
 }
 
-// Launch shape of the gather, from measurements on B200 (resident warps beat
-// loads per warp once there are enough rows to fill the machine):
-//   fp32, >= 131072 rows : 2 loads in flight per lane, 64 warps per SM
-//   fp32, fewer rows     : 8 loads in flight per lane, 32 warps per SM (fewer rounds per row: latency bound)
-//   bf16                 : 2 loads in flight per lane, 48 warps per SM
+// Launch shape of the gather (loads in flight per lane, resident warps per SM),
+// from sweeps on B200 over the five workload shapes: resident warps beat loads
+// per warp once there are enough rows to fill the machine.
+//   fp32, 512-byte rows (32 lanes per row) : 4 loads, 48 warps
+//   fp32, narrower rows, >= 131072 rows    : 2 loads, 64 warps
+//   fp32, narrower rows, fewer rows        : 4 loads, 40 warps
+//   bf16                                   : 2 loads, 48 warps
 constexpr int32_t kManyRows = 131072;
 
 #ifdef HAG_TUNING
@@ -106,8 +108,9 @@ cudaError_t launch_gather_lpr(const hagk::GatherArgs &a, cudaStream_t s) {
     }
 #endif
     if constexpr (sizeof(T) == 4) {
+        if constexpr (LPR == 32) return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 12>, grid, a, s);
         if (a.row_count >= kManyRows) return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 16>, grid, a, s);
-        return launch_pdl(hagk::gather_sum_kernel<T, LPR, 8, SS, 8>, grid, a, s);
+        return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 10>, grid, a, s);
     } else {
         return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 12>, grid, a, s);
     }
