@@ -188,6 +188,8 @@ def main():
     ap.add_argument("--workload", type=int, default=2, help="1-5; 2 is the 50 000-node clustered power-law graph")
     ap.add_argument("--scale", type=float, default=1.0)
     ap.add_argument("--capacity-frac", type=float, default=0.25)
+    ap.add_argument("--capacity-sweep", action="store_true",
+                    help="also time capacities 0, N/8, N/4, N/2 from ONE search (hag_truncate); reported under capacity_sweep")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -296,8 +298,6 @@ def main():
     csr_ms, _ = timed(False, args.steps, cold=True)
     hag_warm_ms, _ = timed(True, args.steps, cold=False)
     csr_warm_ms, _ = timed(False, args.steps, cold=False)
-    # a timed arm lasts milliseconds, far below nvidia-smi's sampling period: the sampler runs across all four arms
-    clocks = sampler.stop() if rank == 0 else {}
 
     # the dominant kernel, timed live with event pairs around every launch
     h.profile(True)
@@ -316,6 +316,8 @@ def main():
             kinds[kind].append(ms)
         bwd_gather.append(rec[-1][0])
     h.profile(False)
+    # a timed arm lasts milliseconds, below nvidia-smi's sampling period: the sampler ran across all GPU arms
+    clocks = sampler.stop() if rank == 0 else {}
     peak, peak_kind = measured_peak()
     fg_ms = float(np.mean(fwd_gather))
     achieved = nbytes["fwd_gather"] / (fg_ms * 1e-3) / 1e9
@@ -375,6 +377,33 @@ def main():
                "sample": f"{what}; {reps} repetitions; bytes counted as (|E|+N)*D*{s} per pass like the GPU's plain path",
                "ms_per_step_full_workload": sec / frac * 1e3}
 
+    sweep = None
+    if args.capacity_sweep and rank == 0:
+        # Section 5.4's capacity study: one search at N/2, every smaller capacity is a prefix of its merges
+        t0 = time.perf_counter()
+        big = hb.Hag.build(g.row_ptr, g.col_idx, g.n // 2)
+        search_s = time.perf_counter() - t0
+        sweep = {"search_seconds_at_half_n": search_s, "points": []}
+        keep_h, keep_ws = h, ws
+        for frac_name, cap in (("0", 0), ("N/8", g.n // 8), ("N/4", g.n // 4), ("N/2", g.n // 2)):
+            hc = big.truncate(cap).to_device(local_rank)
+            ic, ac = hc.info(), hc.arrays()
+            nb = algorithmic_bytes(g.n, w.d, w.dtype, ac, ic)
+            h = hc
+            ws = torch.empty(max(hc.workspace_bytes(w.d) // 4, 4), dtype=torch.float32, device=dev)
+            for _ in range(3):
+                step(True)
+            ms, _ = timed(True, max(args.steps // 4, 5), cold=True)
+            sweep["points"].append({"capacity": frac_name, "num_agg": ic["num_agg"], "levels": ic["num_levels"],
+                                    "e_hat": ic["e_hat"], "ms_per_step": ms,
+                                    "gbps": 2 * w.layers * nb["hag_pass"] / (ms * 1e-3) / 1e9,
+                                    "speedup_vs_capacity_0": None})
+            hc.close()
+        h, ws = keep_h, keep_ws
+        base_ms = sweep["points"][0]["ms_per_step"]
+        for pt in sweep["points"]:
+            pt["speedup_vs_capacity_0"] = base_ms / pt["ms_per_step"]
+
     if rank == 0:
         bytes_step = 2 * w.layers * nbytes["hag_pass"]
         value = world * bytes_step / (hag_ms * 1e-3) / 1e9
@@ -388,7 +417,7 @@ def main():
                             f"|V_A|={info['num_agg']} (capacity {w.capacity}), {w.layers} layer(s), fwd+bwd",
                 "l2": "flushed between timed steps (256 MiB write outside the per-step events)",
                 "timing": "sum of per-step CUDA-event intervals on the launching stream, max over ranks",
-                "clocks": "nvidia-smi sampled every 100 ms across the four timed arms (HAG/plain x cold/warm)",
+                "clocks": "nvidia-smi sampled every 100 ms across the GPU arms (HAG/plain x cold/warm, per-kernel pass)",
             },
             "clocks": clocks,
             "e2e": e2e,
@@ -413,6 +442,8 @@ def main():
                          "algorithmic_bytes_per_launch": nbytes["fwd_gather"], "ms_per_launch": fg_ms},
             "cpu_baseline": cpu,
         }
+        if sweep is not None:
+            line["capacity_sweep"] = sweep
         if w.dtype == "bf16":
             line["dtype"] = "f32 accumulate, bf16 storage"
         print(json.dumps(line))

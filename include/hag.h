@@ -30,7 +30,10 @@
  *   errors     every function returns a hag_status; nothing throws, aborts or
  *              traps.  Argument checks are synchronous.  A failing kernel surfaces
  *              at the caller's next synchronisation, as usual for CUDA.
- *   threads    a handle may be used from one thread at a time.
+ *   threads    a handle may be used from one thread at a time, and its aggregate calls
+ *              must be ordered on the device (one stream, or events between
+ *              streams): the handle owns small scheduling counters that the
+ *              kernels of consecutive calls take turns on.
  *   results    no floating-point atomics anywhere: the same inputs give the same
  *              bits on every run.
  */

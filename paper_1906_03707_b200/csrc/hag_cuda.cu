@@ -52,7 +52,7 @@ void free_device(hag *h) {
     h->events.clear();
     void *ptrs[] = {d.agg_in, d.res_ptr, d.res_idx, d.t_ptr, d.t_idx, d.csr_ptr, d.csr_idx, d.csr_t_ptr,
                     d.csr_t_idx, d.inv_degree, d.stage_in, d.stage_out, d.stage_ws,
-                    d.ftail_ptr, d.ftail_idx, d.btail_ptr, d.btail_idx};
+                    d.ftail_ptr, d.ftail_idx, d.btail_ptr, d.btail_idx, d.sched};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     d = hag_device_arrays{};
@@ -80,21 +80,38 @@ cudaError_t launch_pdl(void (*kernel)(Args), unsigned grid, const Args &args, cu
     return cudaLaunchKernelEx(&cfg, kernel, args);
 }
 
-// Launch shape of the gather (loads in flight per lane, resident warps per SM),
-// from sweeps on B200 over the five workload shapes: resident warps beat loads
-// per warp once there are enough rows to fill the machine.
-//   fp32, 512-byte rows (32 lanes per row) : 4 loads, 48 warps
-//   fp32, narrower rows, >= 131072 rows    : 2 loads, 64 warps
-//   fp32, narrower rows, fewer rows        : 4 loads, 40 warps
-//   bf16                                   : 2 loads, 48 warps
+// Launch shape of the gather (loads in flight per lane, resident warps per SM,
+// one row per launched warp or resident warps that pull rows), from sweeps on
+// B200 over the five workload shapes:
+//   fp32, large launch, 512-byte rows   : resident warps, 8 loads, 32 warps/SM
+//   fp32, large launch, narrower rows   : resident warps, 4 loads, 32 warps/SM
+//   fp32, small launch, 512-byte rows   : one row per warp, 4 loads, 48 warps/SM
+//   fp32, small launch, narrower rows   : one row per warp, 4 loads, 40 warps/SM
+// (large = at least 131072 rows or 4 Mi source entries)
+//   bf16                                : one row per warp, 2 loads, 48 warps/SM
+// Resident warps hide the pointer -> ids latency of the next row behind the
+// current one, which pays once there are many rows per warp; with few rows the
+// hardware's own block scheduling balances better.
 constexpr int32_t kManyRows = 131072;
+constexpr int64_t kManyEdges = int64_t(4) << 20;
 
 #ifdef HAG_TUNING
 int g_tune = -1;   // tuning builds only: force a launch shape
 #endif
 
+// Persistent form: exactly as many CTAs as stay resident, rows handed out through a.sched.
+template <typename Kernel>
+cudaError_t launch_persistent(Kernel kernel, const hagk::GatherArgs &a, int sm_count, cudaStream_t s) {
+    int per_sm = 0;
+    cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, hagk::kThreads, 0);
+    if (err != cudaSuccess) return err;
+    const int64_t want = (int64_t(a.row_count) + hagk::kWarps - 1) / hagk::kWarps;
+    const unsigned grid = unsigned(std::max<int64_t>(1, std::min<int64_t>(want, int64_t(per_sm) * sm_count)));
+    return launch_pdl(kernel, grid, a, s);
+}
+
 template <typename T, int LPR, bool SS>
-cudaError_t launch_gather_lpr(const hagk::GatherArgs &a, cudaStream_t s) {
+cudaError_t launch_gather_lpr(const hagk::GatherArgs &a, int sm_count, cudaStream_t s) {
     const unsigned grid = unsigned((a.row_count + hagk::kWarps - 1) / hagk::kWarps);
 #ifdef HAG_TUNING
     switch (g_tune) {
@@ -104,12 +121,21 @@ cudaError_t launch_gather_lpr(const hagk::GatherArgs &a, cudaStream_t s) {
         case 3: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 12>, grid, a, s);
         case 4: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 16>, grid, a, s);
         case 5: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 10>, grid, a, s);
+        case 6: return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 2, SS, 16>, a, sm_count, s);
+        case 7: return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 2, SS, 12>, a, sm_count, s);
+        case 8: return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 4, SS, 12>, a, sm_count, s);
+        case 9: return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 4, SS, 10>, a, sm_count, s);
+        case 10: return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 4, SS, 8>, a, sm_count, s);
+        case 11: return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 8, SS, 8>, a, sm_count, s);
         default: break;
     }
 #endif
     if constexpr (sizeof(T) == 4) {
+        if (a.resident) {
+            if constexpr (LPR == 32) return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 8, SS, 8>, a, sm_count, s);
+            return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 4, SS, 8>, a, sm_count, s);
+        }
         if constexpr (LPR == 32) return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 12>, grid, a, s);
-        if (a.row_count >= kManyRows) return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 16>, grid, a, s);
         return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 10>, grid, a, s);
     } else {
         return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 12>, grid, a, s);
@@ -117,15 +143,18 @@ cudaError_t launch_gather_lpr(const hagk::GatherArgs &a, cudaStream_t s) {
 }
 
 template <typename T>
-cudaError_t launch_gather(const hagk::GatherArgs &a, int n_chunks, cudaStream_t s) {
+cudaError_t launch_gather(const hag *h, hagk::GatherArgs a, int64_t edges, int n_chunks, cudaStream_t s) {
     if (a.row_count <= 0) return cudaSuccess;
+    a.resident = (a.row_count >= kManyRows || edges >= kManyEdges) ? 1 : 0;
+    hag *hm = const_cast<hag *>(h);
+    a.sched = h->d.sched + 2 * (hm->sched_seq++ % kSchedSlots);
     const int lpr = lanes_per_row(n_chunks);
     const bool ss = a.src_scale != nullptr;
     switch (lpr) {
-        case 4: return ss ? launch_gather_lpr<T, 4, true>(a, s) : launch_gather_lpr<T, 4, false>(a, s);
-        case 8: return ss ? launch_gather_lpr<T, 8, true>(a, s) : launch_gather_lpr<T, 8, false>(a, s);
-        case 16: return ss ? launch_gather_lpr<T, 16, true>(a, s) : launch_gather_lpr<T, 16, false>(a, s);
-        default: return ss ? launch_gather_lpr<T, 32, true>(a, s) : launch_gather_lpr<T, 32, false>(a, s);
+        case 4: return ss ? launch_gather_lpr<T, 4, true>(a, h->sm_count, s) : launch_gather_lpr<T, 4, false>(a, h->sm_count, s);
+        case 8: return ss ? launch_gather_lpr<T, 8, true>(a, h->sm_count, s) : launch_gather_lpr<T, 8, false>(a, h->sm_count, s);
+        case 16: return ss ? launch_gather_lpr<T, 16, true>(a, h->sm_count, s) : launch_gather_lpr<T, 16, false>(a, h->sm_count, s);
+        default: return ss ? launch_gather_lpr<T, 32, true>(a, h->sm_count, s) : launch_gather_lpr<T, 32, false>(a, h->sm_count, s);
     }
 }
 
@@ -222,7 +251,7 @@ hag_status enqueue_fwd_agg(const hag *h, int32_t D, const void *x, float *ws, cu
         a.out_is_f32 = 1;
         a.D = D;
         if (rec) rec->begin(1, a.row_count, int64_t(h->ftail_idx.size()));
-        if (launch_gather<T>(a, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+        if (launch_gather<T>(h, a, int64_t(h->ftail_idx.size()), n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
         if (rec) rec->end();
     }
     return HAG_OK;
@@ -257,7 +286,7 @@ hag_status fwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
     }
     if (h->n > 0) {
         if (rec) rec->begin(2, h->n, use_hag ? h->e_res : h->e);
-        if (launch_gather<T>(a, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+        if (launch_gather<T>(h, a, use_hag ? h->e_res : h->e, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
         if (rec) rec->end();
     }
     return HAG_OK;
@@ -291,7 +320,7 @@ hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
             t.out_row_offset = h->n;
             t.out_is_f32 = 1;
             if (rec) rec->begin(1, t.row_count, int64_t(h->btail_idx.size()));
-            if (launch_gather<T>(t, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+            if (launch_gather<T>(h, t, int64_t(h->btail_idx.size()), n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
             if (rec) rec->end();
         }
         a.row_ptr = d.t_ptr;
@@ -306,8 +335,9 @@ hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
             lv.out_row_offset = h->n;
             lv.out_is_f32 = 1;
             if (lv.row_count <= 0) continue;
-            if (rec) rec->begin(1, lv.row_count, h->t_ptr[size_t(lv.row_begin) + lv.row_count] - h->t_ptr[lv.row_begin]);
-            if (launch_gather<T>(lv, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+            const int64_t lv_edges = h->t_ptr[size_t(lv.row_begin) + lv.row_count] - h->t_ptr[lv.row_begin];
+            if (rec) rec->begin(1, lv.row_count, lv_edges);
+            if (launch_gather<T>(h, lv, lv_edges, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
             if (rec) rec->end();
         }
     } else if (use_hag) {
@@ -322,7 +352,7 @@ hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
     a.out = gx;
     if (h->n > 0) {
         if (rec) rec->begin(2, h->n, use_hag ? h->t_ptr[h->n] : h->e);
-        if (launch_gather<T>(a, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+        if (launch_gather<T>(h, a, use_hag ? h->t_ptr[h->n] : h->e, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
         if (rec) rec->end();
     }
     return HAG_OK;
@@ -409,6 +439,14 @@ extern "C" hag_status hag_to_device(hag_t *h, int device) {
             cudaGetLastError();
             st = err == cudaErrorMemoryAllocation ? HAG_ERR_OOM_DEVICE : HAG_ERR_CUDA;
         } else if (cudaMemcpy(d.inv_degree, inv.data(), inv.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaGetLastError();
+            st = HAG_ERR_CUDA;
+        }
+    }
+    if (st == HAG_OK) {
+        const size_t bytes = size_t(2) * kSchedSlots * sizeof(unsigned int);
+        if (cudaMalloc(reinterpret_cast<void **>(&d.sched), bytes) != cudaSuccess || cudaMemset(d.sched, 0, bytes) != cudaSuccess ||
+            cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
             cudaGetLastError();
             st = HAG_ERR_CUDA;
         }

@@ -8,6 +8,8 @@
 
 #include "hag.h"
 
+constexpr int kSchedSlots = 64;      // far more than the kernels that can overlap on one stream
+
 struct hag_device_arrays {
     // HAG
     int32_t *agg_in = nullptr;     // [2*num_agg]
@@ -23,6 +25,7 @@ struct hag_device_arrays {
     int32_t *ftail_ptr = nullptr, *ftail_idx = nullptr;   // forward expansion of the deep levels
     int32_t *btail_ptr = nullptr, *btail_idx = nullptr;   // backward expansion
     float *inv_degree = nullptr;   // [n] 1/|N(v)| (1 for empty rows)
+    unsigned int *sched = nullptr; // ring of kSchedSlots (next row, finished warps) pairs, zero between launches
     // staging for the host-buffer entry point
     void *stage_in = nullptr;
     void *stage_out = nullptr;
@@ -53,6 +56,8 @@ struct hag {
     int device = -1;
     hag_device_arrays d;
     int32_t last_launches = 0;
+    int32_t sm_count = 0;            // of the device holding the arrays
+    uint32_t sched_seq = 0;          // next slot of the scheduling ring
     // per-launch timing (hag_profile_*)
     bool profile = false;
     std::vector<cudaEvent_t> events;          // pairs: 2*i start, 2*i+1 stop

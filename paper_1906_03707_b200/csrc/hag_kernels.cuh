@@ -42,10 +42,12 @@ struct GatherArgs {
     int32_t n_prim;
     const float *src_scale;   // optional per-source factor for primary rows (backward of mean)
     const float *dst_scale;   // optional per-destination factor, indexed by absolute row id
+    unsigned int *sched;      // persistent kernel only: [0] next row to hand out, [1] finished warps (both zero at launch)
     void *out;                // T rows (out_is_f32 == 0) or fp32 rows (out_is_f32 == 1)
     int32_t out_row_offset;   // absolute row r is written to output row r - out_row_offset
     int32_t out_is_f32;
     int32_t D;
+    int32_t resident;         // host-side choice of the launch form; the kernels ignore it
 };
 
 template <typename T> struct Chunk;
@@ -132,24 +134,39 @@ __device__ __forceinline__ void store_chunk(void *out, int out_is_f32, int32_t D
     }
 }
 
-// Gather-sum of one row by one warp; used by the grid kernel and by the fused
-// small-level kernel.  Returns with the result stored.
+// What a warp needs before it can start on a row: the first 32 source ids (one per
+// lane, -1 past the end), their factors, and the row's own factor.  All of it is
+// static structure, so it can be fetched while the previous row is still summed.
+struct RowHead {
+    int32_t id;
+    float src_scale;
+    float dst_scale;
+};
+
+template <bool SRC_SCALE>
+__device__ __forceinline__ RowHead load_head(const GatherArgs &a, int32_t row, int32_t b, int32_t e, int lane) {
+    RowHead h;
+    h.id = (b + lane < e) ? __ldg(a.idx + b + lane) : -1;
+    // the factor of each source travels with its id: fetched a batch ahead, handed round by shuffle
+    h.src_scale = 1.0f;
+    if constexpr (SRC_SCALE) h.src_scale = (h.id >= 0 && h.id < a.n_prim) ? __ldg(a.src_scale + h.id) : 1.0f;
+    h.dst_scale = a.dst_scale ? __ldg(a.dst_scale + row) : 1.0f;
+    return h;
+}
+
+// Gather-sum of one row [b, e) by one warp.  Returns with the result stored.
 template <typename T, int LPR, int UNROLL, bool SRC_SCALE>
-__device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int lane, bool first_row_of_kernel) {
+__device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int32_t b, int32_t e, const RowHead &head, int lane) {
     constexpr int E = Chunk<T>::kElems;
     constexpr int G = 32 / LPR;                 // slices per warp
     constexpr int PER_BATCH = LPR;              // neighbours each slice takes from a batch of 32 ids
     constexpr int U = (UNROLL < PER_BATCH) ? UNROLL : PER_BATCH;
     const int slice = lane / LPR;
     const int gl = lane % LPR;
-    const int32_t b = __ldg(a.row_ptr + row), e = __ldg(a.row_ptr + row + 1);
     const int n_chunks = a.D / E;
-    const float dscale = a.dst_scale ? __ldg(a.dst_scale + row) : 1.0f;
-    int32_t first = (b + lane < e) ? __ldg(a.idx + b + lane) : -1;
-    // the factor of each source travels with its id: fetched a batch ahead, handed round by shuffle
-    float first_s = 1.0f;
-    if constexpr (SRC_SCALE) first_s = (first >= 0 && first < a.n_prim) ? __ldg(a.src_scale + first) : 1.0f;
-    if (first_row_of_kernel) pdl_wait();        // structure arrays are static; features may come from the previous kernel
+    const float dscale = head.dst_scale;
+    const int32_t first = head.id;
+    const float first_s = head.src_scale;
 
     for (int c0 = 0; c0 < n_chunks; c0 += LPR) {
         const int chunk = c0 + gl;
@@ -221,13 +238,80 @@ __device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int
 }
 
 // out[row] = (dst_scale[row]) * sum_{e in row} (src_scale[id_e]) * table[id_e]
+// One warp per row, one launch-time row per warp.
 template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS>
 __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_kernel(const GatherArgs a) {
     pdl_launch_dependents();
     const int lane = threadIdx.x & 31;
     const int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
     if (r_local >= a.row_count) return;
-    gather_row<T, LPR, UNROLL, SRC_SCALE>(a, a.row_begin + r_local, lane, true);
+    const int32_t row = a.row_begin + r_local;
+    const int32_t b = __ldg(a.row_ptr + row), e = __ldg(a.row_ptr + row + 1);
+    const RowHead head = load_head<SRC_SCALE>(a, row, b, e, lane);
+    pdl_wait();        // structure arrays are static; features may come from the previous kernel
+    gather_row<T, LPR, UNROLL, SRC_SCALE>(a, row, b, e, head, lane);
+}
+
+// The same, with resident warps that take rows four at a time from a shared
+// counter (a.sched[0]) and fetch the next row's pointers and first ids while the
+// current row is summed, so the pointer -> ids -> rows latency chain is paid once
+// per warp instead of once per row.  The last warp to finish zeroes the counters
+// (a.sched[1] counts finished warps) for the slot's next use.  No warp waits on
+// another: there is no spin anywhere.
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS>
+__global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_persistent_kernel(const GatherArgs a) {
+    pdl_launch_dependents();
+    constexpr int CH = 4;
+    constexpr unsigned FULL = 0xffffffffu;
+    const int lane = threadIdx.x & 31;
+    const int32_t count = a.row_count;
+    const int32_t *rp_base = a.row_ptr + a.row_begin;
+    auto grab = [&]() -> int32_t {          // meaningful in lane 0
+        int32_t v = 0;
+        if (lane == 0) v = int32_t(atomicAdd(a.sched, unsigned(CH)));
+        return v;
+    };
+    auto load_rp = [&](int32_t base) -> int32_t {   // lane i <= CH: pointer of row base + i (clamped to the end)
+        return (lane <= CH && base < count) ? __ldg(rp_base + min(base + lane, count)) : 0;
+    };
+    int32_t base = __shfl_sync(FULL, grab(), 0);
+    int32_t rp = load_rp(base);
+    RowHead head{-1, 1.0f, 1.0f};
+    if (base < count) head = load_head<SRC_SCALE>(a, a.row_begin + base, __shfl_sync(FULL, rp, 0), __shfl_sync(FULL, rp, 1), lane);
+    pdl_wait();
+    while (base < count) {
+        const int32_t grabbed = grab();     // the next four rows; consumed after the first row below
+        const int nrows = min(CH, count - base);
+        int32_t nbase = count, rp_next = 0;
+        for (int i = 0; i < nrows; ++i) {
+            const int32_t b = __shfl_sync(FULL, rp, i), e = __shfl_sync(FULL, rp, i + 1);
+            const RowHead cur = head;
+            if (i + 1 < nrows) {
+                head = load_head<SRC_SCALE>(a, a.row_begin + base + i + 1, e, __shfl_sync(FULL, rp, i + 2), lane);
+            } else {
+                if (nrows == 1) {
+                    nbase = __shfl_sync(FULL, grabbed, 0);
+                    rp_next = load_rp(nbase);
+                }
+                const int32_t nb = __shfl_sync(FULL, rp_next, 0), ne = __shfl_sync(FULL, rp_next, 1);
+                if (nbase < count) head = load_head<SRC_SCALE>(a, a.row_begin + nbase, nb, ne, lane);
+            }
+            gather_row<T, LPR, UNROLL, SRC_SCALE>(a, a.row_begin + base + i, b, e, cur, lane);
+            if (i == 0 && nrows > 1) {
+                nbase = __shfl_sync(FULL, grabbed, 0);
+                rp_next = load_rp(nbase);
+            }
+        }
+        base = nbase;
+        rp = rp_next;
+    }
+    if (lane == 0) {
+        const unsigned finished = atomicAdd(a.sched + 1, 1u);
+        if (finished == gridDim.x * kWarps - 1) {   // every warp has made its last grab
+            a.sched[0] = 0;
+            a.sched[1] = 0;
+        }
+    }
 }
 
 // Level kernel of Algorithm 2 (lines 5-6): every aggregation node of one level is

@@ -234,6 +234,18 @@ def test_full_size_workloads_sampled_rows(index):
     h = hb.Hag.build(g.row_ptr, g.col_idx, w.capacity).to_device(0)
     info = h.info()
     assert info["num_agg"] == w.capacity
+    # structure: bit-exact against the digest the oracle's own search and layout left under tests/golden
+    import hashlib
+    import json
+    import os
+    stored = json.load(open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "structure_hashes.json")))
+    rec = stored["cases"].get(f"cfg{index}@1")
+    if rec is not None:
+        arr = h.arrays()
+        dig = hashlib.sha256()
+        for k in stored["array_order"]:
+            dig.update(np.ascontiguousarray(arr[k]).tobytes())
+        assert dig.hexdigest() == rec["sha256"], "structure differs from the oracle's"
     x = synth.features(w.seed, g.n, w.d, w.feat_dist, w.dtype)
     gr = synth.upstream_grad(w.seed, g.n, w.d, w.feat_dist, w.dtype)
     rng = np.random.default_rng(0)
