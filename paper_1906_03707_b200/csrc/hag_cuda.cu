@@ -85,8 +85,7 @@ cudaError_t launch_pdl(void (*kernel)(Args), unsigned grid, const Args &args, cu
 // B200 over the five workload shapes:
 //   fp32, large launch, 512-byte rows   : resident warps, 8 loads, 32 warps/SM
 //   fp32, large launch, narrower rows   : resident warps, 4 loads, 32 warps/SM
-//   fp32, small launch, 512-byte rows   : one row per warp, 4 loads, 48 warps/SM
-//   fp32, small launch, narrower rows   : one row per warp, 4 loads, 40 warps/SM
+//   fp32, small launch                  : one row per warp, 4 loads, 40 warps/SM
 // (large = at least 131072 rows or 4 Mi source entries)
 //   bf16                                : one row per warp, 2 loads, 48 warps/SM
 // Resident warps hide the pointer -> ids latency of the next row behind the
@@ -135,7 +134,6 @@ cudaError_t launch_gather_lpr(const hagk::GatherArgs &a, int sm_count, cudaStrea
             if constexpr (LPR == 32) return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 8, SS, 8>, a, sm_count, s);
             return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 4, SS, 8>, a, sm_count, s);
         }
-        if constexpr (LPR == 32) return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 12>, grid, a, s);
         return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 10>, grid, a, s);
     } else {
         return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 12>, grid, a, s);

@@ -10,9 +10,10 @@
 //   * neighbour ids are read coalesced, 32 at a time, and handed round with
 //     shuffles; the next batch of ids is fetched before the current one is used;
 //   * UNROLL row loads per lane are issued back to back, then summed as a
-//     balanced tree and added to ONE fp32 accumulator: the rounding error grows
-//     like n/UNROLL + log2(UNROLL) ulps, as with UNROLL independent partial sums,
-//     at a quarter of the registers (more resident warps);
+//     balanced tree into a per-batch partial that is folded into the row's
+//     accumulator once per 32 ids: the rounding error grows like
+//     n/32 + 32/UNROLL + log2(UNROLL) ulps with two accumulators' worth of
+//     registers (more resident warps than UNROLL independent partial sums);
 //   * slices are combined with butterfly shuffles in a fixed order; no atomics,
 //     one writer per output row: same bits every run;
 //   * a source id below n_prim reads the primary table (the layer input, fp32
@@ -172,7 +173,9 @@ __device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int
         const int chunk = c0 + gl;
         const bool live = chunk < n_chunks;
         const Tables<T> tab(a.prim, a.sec, a.n_prim, a.D, live ? chunk : 0);
-        float acc[E];
+        // two-level sum: `part` collects the tree sums of one batch of 32 ids, `acc` the batches, so a row of n
+        // terms passes through about n/32 + 32/U + log2(U) roundings instead of n/U
+        float acc[E], part[E];
 #pragma unroll
         for (int j = 0; j < E; ++j) acc[j] = 0.0f;
 
@@ -189,6 +192,10 @@ __device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int
             mine = (nb + lane < e) ? __ldg(a.idx + nb + lane) : -1;      // next batch of ids, in flight early
             if constexpr (SRC_SCALE) mine_s = (mine >= 0 && mine < a.n_prim) ? __ldg(a.src_scale + mine) : 1.0f;
             const int cnt = min(32, e - base);
+            if constexpr (E == 4) {       // fp32 storage only: bf16 results are rounded to 8 bits anyway
+#pragma unroll
+                for (int j = 0; j < E; ++j) part[j] = 0.0f;
+            }
 #pragma unroll
             for (int k = 0; k < PER_BATCH; k += U) {
                 if (k * G < cnt) {
@@ -219,9 +226,18 @@ __device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int
                         for (int u = 0; u < w; ++u)
 #pragma unroll
                             for (int j = 0; j < E; ++j) v[u][j] += v[u + w][j];
+                    if constexpr (E == 4) {
 #pragma unroll
-                    for (int j = 0; j < E; ++j) acc[j] += v[0][j];
+                        for (int j = 0; j < E; ++j) part[j] += v[0][j];
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < E; ++j) acc[j] += v[0][j];
+                    }
                 }
+            }
+            if constexpr (E == 4) {
+#pragma unroll
+                for (int j = 0; j < E; ++j) acc[j] += part[j];
             }
         }
         // combine the slices (fixed butterfly), then slice 0 stores

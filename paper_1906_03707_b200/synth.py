@@ -293,15 +293,19 @@ def config5_graph(seed: int = 4, n: int = 1_000_000, n_comm: int = 2000, s_lo: i
 def clique_union_graph(seed: int, n: int, n_groups: int, g_lo: int, g_hi: int, g_alpha: float = 2.0,
                        self_loops: bool = True) -> Graph:
     """Bipartite-projection shape (co-authorship / shared-commenter style): every
-    group is a clique over its members, members drawn uniformly."""
+    group is a clique over its members; group sizes from a truncated power law,
+    members drawn uniformly (a member drawn twice for one group counts once)."""
     rng = _rng(seed)
-    sizes = truncated_power_law(rng, n_groups, g_lo, g_hi, g_alpha)
+    sizes = truncated_power_law(rng, n_groups, g_lo, min(g_hi, n), g_alpha)
+    members = rng.integers(0, n, size=int(sizes.sum()))
+    starts = np.concatenate([[0], np.cumsum(sizes)[:-1]])
     a_parts, b_parts = [], []
-    for s in sizes:
-        m = rng.choice(n, size=int(min(s, n)), replace=False)
-        iu, ju = np.triu_indices(m.size, k=1)
-        a_parts.append(m[iu])
-        b_parts.append(m[ju])
+    for sz in np.unique(sizes):
+        rows = np.nonzero(sizes == sz)[0]
+        block = members[starts[rows][:, None] + np.arange(sz)[None, :]]       # one group per row
+        iu, ju = np.triu_indices(int(sz), k=1)
+        a_parts.append(block[:, iu].ravel())
+        b_parts.append(block[:, ju].ravel())
     a = np.concatenate(a_parts) if a_parts else np.zeros(0, np.int64)
     b = np.concatenate(b_parts) if b_parts else np.zeros(0, np.int64)
     return csr_from_undirected_pairs(n, a, b, self_loops=self_loops, name="clique-union",
