@@ -32,6 +32,9 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "HAG fwd+bwd aggregation GB/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE forward-gather launch, from ncu captures of this
+# program at the workload's full size (None: not captured)
+NCU_DRAM_BYTES_FWD_GATHER = {"cfg2": 23.36e6 + 0.04e6, "cfg4": 228.1e6 + 104.0e6}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 256 << 20
@@ -185,7 +188,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=2, help="1-5; 2 is the 50 000-node clustered power-law graph")
+    ap.add_argument("--workload", type=int, default=2, help="1-5: the named shapes (2 = the 50 000-node clustered power-law graph); 6: clique-union graph")
     ap.add_argument("--scale", type=float, default=1.0)
     ap.add_argument("--capacity-frac", type=float, default=0.25)
     ap.add_argument("--capacity-sweep", action="store_true",
@@ -241,7 +244,7 @@ def main():
     x = torch.from_numpy(synth.features(w.seed, g.n, w.d, w.feat_dist, w.dtype)).to(dev).to(tdt)
     gr = torch.from_numpy(synth.upstream_grad(w.seed, g.n, w.d, w.feat_dist, w.dtype)).to(dev).to(tdt)
     bufs = [torch.empty_like(x) for _ in range(2 * w.layers)]
-    ws_bytes = h.workspace_bytes(w.d)
+    ws_bytes = max(h.workspace_bytes(w.d), h.csr_workspace_bytes(w.d))
     ws = torch.empty(max(ws_bytes // 4, 4), dtype=torch.float32, device=dev)
     flush = torch.empty(L2_FLUSH_BYTES // 4, dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream(dev)
@@ -253,7 +256,7 @@ def main():
             if hag:
                 h.aggregate_fwd(cur, w.reduce, out=bufs[l], workspace=ws)
             else:
-                h.csr_fwd(cur, w.reduce, out=bufs[l])
+                h.csr_fwd(cur, w.reduce, out=bufs[l], workspace=ws)
             launches += h.last_launch_count
             cur = bufs[l]
         cur = gr
@@ -262,7 +265,7 @@ def main():
             if hag:
                 h.aggregate_bwd(cur, w.reduce, out=o, workspace=ws)
             else:
-                h.csr_bwd(cur, w.reduce, out=o)
+                h.csr_bwd(cur, w.reduce, out=o, workspace=ws)
             launches += h.last_launch_count
             cur = o
         return launches
@@ -390,7 +393,7 @@ def main():
             ic, ac = hc.info(), hc.arrays()
             nb = algorithmic_bytes(g.n, w.d, w.dtype, ac, ic)
             h = hc
-            ws = torch.empty(max(hc.workspace_bytes(w.d) // 4, 4), dtype=torch.float32, device=dev)
+            ws = torch.empty(max(hc.workspace_bytes(w.d), hc.csr_workspace_bytes(w.d), 16) // 4, dtype=torch.float32, device=dev)
             for _ in range(3):
                 step(True)
             ms, _ = timed(True, max(args.steps // 4, 5), cold=True)
@@ -438,7 +441,8 @@ def main():
                            "fwd_final_gather": fg_ms, "bwd_final_gather": float(np.mean(bwd_gather))},
             "roofline": {"bound": "hbm", "kernel": "gather_sum_kernel (forward gather over the residual rows)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_kind": f"{peak_kind} copy bandwidth", "traffic": None,
+                         "peak_kind": f"{peak_kind} copy bandwidth",
+                         "traffic": NCU_DRAM_BYTES_FWD_GATHER.get(w.name) if args.scale == 1.0 else None,
                          "algorithmic_bytes_per_launch": nbytes["fwd_gather"], "ms_per_launch": fg_ms},
             "cpu_baseline": cpu,
         }

@@ -23,8 +23,9 @@
  *              D * sizeof(dtype) a multiple of 16.
  *   workspace  DEVICE pointer to hag_workspace_bytes() bytes, 16-byte aligned; holds
  *              the fp32 rows of the aggregation nodes (a-hat of Algorithm 2, or their
- *              gradients).  It carries nothing between calls and may be shared by
- *              all layers and by forward and backward (Algorithm 2's caption).
+ *              gradients) and the partial sums of split long rows.  It carries
+ *              nothing between calls and may be shared by all layers and by
+ *              forward and backward (Algorithm 2's caption).
  *   streams    cuda_stream is a cudaStream_t passed as void* (NULL = default
  *              stream).  Calls only enqueue work; they never synchronise.
  *   errors     every function returns a hag_status; nothing throws, aborts or
@@ -163,10 +164,14 @@ hag_status hag_export(const hag_t *h, hag_arrays *out);
  * cudaMalloc; HAG_ERR_OOM_DEVICE / HAG_ERR_CUDA on failure. */
 hag_status hag_to_device(hag_t *h, int device);
 
-/* Bytes of workspace the aggregate calls need for feature width D:
- * |V_A| * D * 4 (fp32 rows whatever the dtype); 0 when the HAG has no
- * aggregation node or on bad arguments. */
+/* Bytes of workspace hag_aggregate_* need for feature width D: fp32 rows (whatever
+ * the dtype) for the |V_A| aggregation nodes, plus one partial row per 128-entry
+ * segment of the rows with more than 256 entries (such rows are summed by several
+ * warps; the largest of the HAG's tables decides).  0 on bad arguments or when
+ * neither exists.  csr_workspace_bytes: the same for csr_aggregate_* (segments of
+ * the input graph's long rows only; 0 for graphs without such rows). */
 size_t hag_workspace_bytes(const hag_t *h, int32_t D);
+size_t csr_workspace_bytes(const hag_t *h, int32_t D);
 
 /* Algorithm 2 (the paper's hag_aggregate), one layer:
  *   a-hat_w = a-hat_in0(w) + a-hat_in1(w)  for aggregation nodes, level by level;
@@ -188,11 +193,11 @@ hag_status hag_aggregate_bwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype,
 
 /* The GNN-graph itself (Algorithm 1 line 4; V_A = {} in Section 3.1): the same
  * gather kernel over the input CSR held by the handle, and over its transpose for
- * the gradient.  No workspace. */
+ * the gradient.  workspace: csr_workspace_bytes() bytes (may be NULL when that is 0). */
 hag_status csr_aggregate_fwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D,
-                             const void *x, void *out, void *cuda_stream);
+                             const void *x, void *out, void *workspace, void *cuda_stream);
 hag_status csr_aggregate_bwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D,
-                             const void *grad_out, void *grad_x, void *cuda_stream);
+                             const void *grad_out, void *grad_x, void *workspace, void *cuda_stream);
 
 /* Host-buffer variants for callers that keep features in host memory: x_host and
  * out_host are HOST pointers to N x D matrices (pinned memory makes the copies
@@ -230,7 +235,8 @@ int32_t hag_profile_read(hag_t *h, int32_t max, float *ms, int32_t *kind, int64_
  *
  * Same arguments, results and errors as hag_aggregate_fwd, without `workspace`.
  * Bit-identical output to hag_aggregate_fwd.  Additionally:
- *   - HAG_ERR_TOO_LARGE when hag_workspace_bytes(h, D) exceeds
+ *   - HAG_ERR_TOO_LARGE when hag_workspace_bytes(h, D) (aggregation-node rows plus
+ *     the partial rows of split long rows) exceeds
  *     HAG_STATIC_SCRATCH_BYTES (nothing is launched);
  *   - the call itself allocates nothing: no cudaMalloc, cudaFree, event or stream
  *     creation, and no host heap use;

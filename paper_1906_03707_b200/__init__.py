@@ -24,7 +24,7 @@ HAG_SUM, HAG_MEAN = 0, 1
 HAG_F32, HAG_BF16 = 0, 1
 
 EXPORTED_SYMBOLS = [
-    "hag_build", "hag_build_threads", "hag_truncate", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes",
+    "hag_build", "hag_build_threads", "hag_truncate", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes", "csr_workspace_bytes",
     "hag_aggregate_fwd", "hag_aggregate_bwd", "csr_aggregate_fwd", "csr_aggregate_bwd",
     "hag_aggregate_host", "hag_aggregate_fwd_static", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
 ]
@@ -89,13 +89,11 @@ def load_library():
     lib.hag_to_device.restype = ctypes.c_int
     lib.hag_workspace_bytes.argtypes = [vp, i32]
     lib.hag_workspace_bytes.restype = ctypes.c_size_t
-    for name in ("hag_aggregate_fwd", "hag_aggregate_bwd"):
+    lib.csr_workspace_bytes.argtypes = [vp, i32]
+    lib.csr_workspace_bytes.restype = ctypes.c_size_t
+    for name in ("hag_aggregate_fwd", "hag_aggregate_bwd", "csr_aggregate_fwd", "csr_aggregate_bwd"):
         f = getattr(lib, name)
         f.argtypes = [vp, ctypes.c_int, ctypes.c_int, i32, vp, vp, vp, vp]
-        f.restype = ctypes.c_int
-    for name in ("csr_aggregate_fwd", "csr_aggregate_bwd"):
-        f = getattr(lib, name)
-        f.argtypes = [vp, ctypes.c_int, ctypes.c_int, i32, vp, vp, vp]
         f.restype = ctypes.c_int
     lib.hag_aggregate_host.argtypes = [vp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, i32, vp, vp, vp]
     lib.hag_aggregate_host.restype = ctypes.c_int
@@ -214,6 +212,9 @@ class Hag:
     def workspace_bytes(self, d: int) -> int:
         return int(load_library().hag_workspace_bytes(self._h, int(d)))
 
+    def csr_workspace_bytes(self, d: int) -> int:
+        return int(load_library().csr_workspace_bytes(self._h, int(d)))
+
     @property
     def last_launch_count(self) -> int:
         return int(load_library().hag_last_launch_count(self._h))
@@ -245,7 +246,7 @@ class Hag:
 
     def _workspace(self, d: int, device):
         import torch
-        need = self.workspace_bytes(d)
+        need = max(self.workspace_bytes(d), self.csr_workspace_bytes(d))
         if need == 0:
             return None
         if self._ws is None or self._ws.numel() * 4 < need or self._ws.device != device:
@@ -273,12 +274,9 @@ class Hag:
         stream = torch.cuda.current_stream(inp.device).cuda_stream
         lib = load_library()
         code = self._dtype_code(inp)
-        if use_hag:
-            ws = workspace if workspace is not None else self._workspace(d, inp.device)
-            st = getattr(lib, name)(self._h, _reduce_code(reduce), code, d, inp.data_ptr(), out.data_ptr(),
-                                    ws.data_ptr() if ws is not None else None, stream)
-        else:
-            st = getattr(lib, name)(self._h, _reduce_code(reduce), code, d, inp.data_ptr(), out.data_ptr(), stream)
+        ws = workspace if workspace is not None else self._workspace(d, inp.device)
+        st = getattr(lib, name)(self._h, _reduce_code(reduce), code, d, inp.data_ptr(), out.data_ptr(),
+                                ws.data_ptr() if ws is not None else None, stream)
         _check(st, name)
         return out
 
@@ -304,13 +302,13 @@ class Hag:
         _check(st, "hag_aggregate_fwd_static")
         return out
 
-    def csr_fwd(self, x, reduce="sum", out=None):
+    def csr_fwd(self, x, reduce="sum", out=None, workspace=None):
         """``csr_aggregate_fwd``: the plain GNN-graph, same kernel."""
-        return self._run("csr_aggregate_fwd", False, x, reduce, out, None)
+        return self._run("csr_aggregate_fwd", False, x, reduce, out, workspace)
 
-    def csr_bwd(self, grad_out, reduce="sum", out=None):
+    def csr_bwd(self, grad_out, reduce="sum", out=None, workspace=None):
         """``csr_aggregate_bwd``."""
-        return self._run("csr_aggregate_bwd", False, grad_out, reduce, out, None)
+        return self._run("csr_aggregate_bwd", False, grad_out, reduce, out, workspace)
 
     def aggregate_host(self, inp, out, reduce="sum", backward=False, use_hag=True, stream=None):
         """``hag_aggregate_host``: host tensors in and out (pinned for async copies);

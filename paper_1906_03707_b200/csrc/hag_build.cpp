@@ -490,6 +490,41 @@ hag_status hag_layout(hag *h, const std::vector<int32_t> &rows_store, const std:
                 for (auto &l : lists) h->btail_idx.insert(h->btail_idx.end(), l.begin(), l.end());
             }
         }
+        // ---- segments of the long rows of every table the gather walks ----
+        {
+            auto build = [](seg_set &set, const std::vector<int64_t> &ptr, int64_t rows, int32_t first_row_id) {
+                for (int gran = 0; gran < kSegGrans; ++gran) {
+                    seg_table &t = set.g[gran];
+                    const int64_t long_row = kSegLongRow[gran], seg_len = kSegLength[gran];
+                    t.segs.clear();
+                    t.slots.clear();
+                    for (int64_t r = 0; r < rows; ++r) {
+                        const int64_t b = ptr[r], e = ptr[r + 1];
+                        if (e - b <= long_row) continue;
+                        const int32_t slot = int32_t(t.slots.size() / 2);
+                        const int32_t first = int32_t(t.segs.size() / 4);
+                        int32_t n_seg = 0;
+                        for (int64_t sb = b; sb < e; sb += seg_len, ++n_seg) {
+                            t.segs.push_back(int32_t(first_row_id + r));
+                            t.segs.push_back(int32_t(sb));
+                            t.segs.push_back(int32_t(std::min<int64_t>(sb + seg_len, e)));
+                            t.segs.push_back(slot);
+                        }
+                        t.slots.push_back(first);
+                        t.slots.push_back(n_seg);
+                    }
+                }
+            };
+            build(h->seg_res, h->res_ptr, n, 0);
+            build(h->seg_t, h->t_ptr, int64_t(n) + k, 0);
+            build(h->seg_csr, h->csr_ptr, n, 0);
+            build(h->seg_csr_t, h->csr_t_ptr, n, 0);
+            build(h->seg_ftail, h->ftail_ptr, int64_t(h->ftail_ptr.size()) - 1, int32_t(n + h->level_ptr[h->fwd_cut]));
+            build(h->seg_btail, h->btail_ptr, int64_t(h->btail_ptr.size()) - 1, int32_t(n + h->level_ptr[h->bwd_cut]));
+            h->max_segs_hag = std::max(std::max(h->seg_res.max_count(), h->seg_t.max_count()),
+                                       std::max(h->seg_ftail.max_count(), h->seg_btail.max_count()));
+            h->max_segs_csr = std::max(h->seg_csr.max_count(), h->seg_csr_t.max_count());
+        }
         // counters of the cost function
         hag_info &f = h->info;
         f = hag_info{};

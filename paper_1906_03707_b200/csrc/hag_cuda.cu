@@ -50,6 +50,14 @@ void free_device(hag *h) {
     hag_device_arrays &d = h->d;
     for (cudaEvent_t ev : h->events) cudaEventDestroy(ev);
     h->events.clear();
+    for (seg_set *set : {&h->seg_res, &h->seg_t, &h->seg_csr, &h->seg_csr_t, &h->seg_ftail, &h->seg_btail})
+    for (seg_table *t = set->g; t != set->g + kSegGrans; ++t) {
+        if (t->d_segs) cudaFree(t->d_segs);
+        if (t->d_slots) cudaFree(t->d_slots);
+        if (t->d_done) cudaFree(t->d_done);
+        t->d_segs = t->d_slots = nullptr;
+        t->d_done = nullptr;
+    }
     void *ptrs[] = {d.agg_in, d.res_ptr, d.res_idx, d.t_ptr, d.t_idx, d.csr_ptr, d.csr_idx, d.csr_t_ptr,
                     d.csr_t_idx, d.inv_degree, d.stage_in, d.stage_out, d.stage_ws,
                     d.ftail_ptr, d.ftail_idx, d.btail_ptr, d.btail_idx, d.sched};
@@ -99,60 +107,107 @@ int g_tune = -1;   // tuning builds only: force a launch shape
 #endif
 
 // Persistent form: exactly as many CTAs as stay resident, rows handed out through a.sched.
-template <typename Kernel>
-cudaError_t launch_persistent(Kernel kernel, const hagk::GatherArgs &a, int sm_count, cudaStream_t s) {
+template <typename Kernel, typename Args>
+cudaError_t launch_persistent(Kernel kernel, const Args &a, int64_t items, int sm_count, cudaStream_t s) {
     int per_sm = 0;
     cudaError_t err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, hagk::kThreads, 0);
     if (err != cudaSuccess) return err;
-    const int64_t want = (int64_t(a.row_count) + hagk::kWarps - 1) / hagk::kWarps;
+    const int64_t want = (items + hagk::kWarps - 1) / hagk::kWarps;
     const unsigned grid = unsigned(std::max<int64_t>(1, std::min<int64_t>(want, int64_t(per_sm) * sm_count)));
     return launch_pdl(kernel, grid, a, s);
 }
 
-template <typename T, int LPR, bool SS>
-cudaError_t launch_gather_lpr(const hagk::GatherArgs &a, int sm_count, cudaStream_t s) {
-    const unsigned grid = unsigned((a.row_count + hagk::kWarps - 1) / hagk::kWarps);
+template <bool SEGS>
+hagk::KernelArgs<SEGS> pack_args(const hagk::GatherArgs &a, const hagk::SegArgs &sg) {
+    hagk::KernelArgs<SEGS> k;
+    k.a = a;
+    if constexpr (SEGS) k.sg = sg;
+    return k;
+}
+
+// The kernel entry for a shape: plain parameters without long rows, grid-constant ones with.
+template <typename T, int LPR, int U, bool SS, int MINB, bool SEGS>
+auto plain_kernel() {
+    if constexpr (SEGS) return hagk::gather_sum_long_kernel<T, LPR, U, SS, MINB>;
+    else return hagk::gather_sum_kernel<T, LPR, U, SS, MINB>;
+}
+template <typename T, int LPR, int U, bool SS, int MINB, bool SEGS>
+auto resident_kernel() {
+    if constexpr (SEGS) return hagk::gather_sum_persistent_long_kernel<T, LPR, U, SS, MINB>;
+    else return hagk::gather_sum_persistent_kernel<T, LPR, U, SS, MINB>;
+}
+
+template <typename T, int LPR, bool SS, bool SEGS>
+cudaError_t launch_gather_shape(const hagk::GatherArgs &ga, const hagk::SegArgs &sg, int sm_count, cudaStream_t s) {
+    const hagk::KernelArgs<SEGS> a = pack_args<SEGS>(ga, sg);
+    const int64_t items = int64_t(ga.row_count) + (SEGS ? sg.seg_count : 0);
+    const unsigned grid = unsigned((items + hagk::kWarps - 1) / hagk::kWarps);
 #ifdef HAG_TUNING
     switch (g_tune) {
-        case 0: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 8, SS, 8>, grid, a, s);
-        case 1: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 8>, grid, a, s);
-        case 2: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 12>, grid, a, s);
-        case 3: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 12>, grid, a, s);
-        case 4: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 16>, grid, a, s);
-        case 5: return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 10>, grid, a, s);
-        case 6: return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 2, SS, 16>, a, sm_count, s);
-        case 7: return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 2, SS, 12>, a, sm_count, s);
-        case 8: return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 4, SS, 12>, a, sm_count, s);
-        case 9: return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 4, SS, 10>, a, sm_count, s);
-        case 10: return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 4, SS, 8>, a, sm_count, s);
-        case 11: return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 8, SS, 8>, a, sm_count, s);
+        case 0: return launch_pdl(plain_kernel<T, LPR, 8, SS, 8, SEGS>(), grid, a, s);
+        case 2: return launch_pdl(plain_kernel<T, LPR, 4, SS, 12, SEGS>(), grid, a, s);
+        case 4: return launch_pdl(plain_kernel<T, LPR, 2, SS, 16, SEGS>(), grid, a, s);
+        case 5: return launch_pdl(plain_kernel<T, LPR, 4, SS, 10, SEGS>(), grid, a, s);
+        case 9: return launch_persistent(resident_kernel<T, LPR, 4, SS, 10, SEGS>(), a, items, sm_count, s);
+        case 10: return launch_persistent(resident_kernel<T, LPR, 4, SS, 8, SEGS>(), a, items, sm_count, s);
+        case 11: return launch_persistent(resident_kernel<T, LPR, 8, SS, 8, SEGS>(), a, items, sm_count, s);
         default: break;
     }
 #endif
     if constexpr (sizeof(T) == 4) {
-        if (a.resident) {
-            if constexpr (LPR == 32) return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 8, SS, 8>, a, sm_count, s);
-            return launch_persistent(hagk::gather_sum_persistent_kernel<T, LPR, 4, SS, 8>, a, sm_count, s);
+        if (ga.resident) {
+            if constexpr (LPR == 32) return launch_persistent(resident_kernel<T, LPR, 8, SS, 8, SEGS>(), a, items, sm_count, s);
+            return launch_persistent(resident_kernel<T, LPR, 4, SS, 8, SEGS>(), a, items, sm_count, s);
         }
-        return launch_pdl(hagk::gather_sum_kernel<T, LPR, 4, SS, 10>, grid, a, s);
+        return launch_pdl(plain_kernel<T, LPR, 4, SS, 10, SEGS>(), grid, a, s);
     } else {
-        return launch_pdl(hagk::gather_sum_kernel<T, LPR, 2, SS, 12>, grid, a, s);
+        return launch_pdl(plain_kernel<T, LPR, 2, SS, 12, SEGS>(), grid, a, s);
     }
 }
 
+template <typename T, int LPR, bool SS>
+cudaError_t launch_gather_lpr(const hagk::GatherArgs &a, const hagk::SegArgs &sg, int sm_count, cudaStream_t s) {
+    return sg.seg_count > 0 ? launch_gather_shape<T, LPR, SS, true>(a, sg, sm_count, s)
+                            : launch_gather_shape<T, LPR, SS, false>(a, sg, sm_count, s);
+}
+
 template <typename T>
-cudaError_t launch_gather(const hag *h, hagk::GatherArgs a, int64_t edges, int n_chunks, cudaStream_t s) {
+cudaError_t launch_gather(const hag *h, hagk::GatherArgs a, const seg_set &set, float *partial, int64_t edges,
+                          int n_chunks, cudaStream_t s) {
     if (a.row_count <= 0) return cudaSuccess;
+    const int gran = seg_gran_for_rows(a.row_count);
+    const seg_table &table = set.g[gran];
+    hagk::SegArgs sg{};
+    sg.long_row = kSegLongRow[gran];
+    // the segments of this launch's long rows: a contiguous run of the table (segments are sorted by row)
+    if (!table.segs.empty()) {
+        const int64_t total = table.count();
+        auto first_at_or_after = [&](int64_t row) {
+            int64_t lo = 0, hi = total;
+            while (lo < hi) {
+                const int64_t mid = (lo + hi) / 2;
+                if (table.segs[4 * mid] < row) lo = mid + 1; else hi = mid;
+            }
+            return lo;
+        };
+        const int64_t lo = first_at_or_after(a.row_begin), hi = first_at_or_after(int64_t(a.row_begin) + a.row_count);
+        sg.segs = reinterpret_cast<const int4 *>(table.d_segs) + lo;
+        sg.slots = reinterpret_cast<const int2 *>(table.d_slots);
+        sg.seg_done = table.d_done;
+        sg.partial = partial;
+        sg.seg_first = int32_t(lo);
+        sg.seg_count = int32_t(hi - lo);
+    }
     a.resident = (a.row_count >= kManyRows || edges >= kManyEdges) ? 1 : 0;
     hag *hm = const_cast<hag *>(h);
     a.sched = h->d.sched + 2 * (hm->sched_seq++ % kSchedSlots);
     const int lpr = lanes_per_row(n_chunks);
     const bool ss = a.src_scale != nullptr;
     switch (lpr) {
-        case 4: return ss ? launch_gather_lpr<T, 4, true>(a, h->sm_count, s) : launch_gather_lpr<T, 4, false>(a, h->sm_count, s);
-        case 8: return ss ? launch_gather_lpr<T, 8, true>(a, h->sm_count, s) : launch_gather_lpr<T, 8, false>(a, h->sm_count, s);
-        case 16: return ss ? launch_gather_lpr<T, 16, true>(a, h->sm_count, s) : launch_gather_lpr<T, 16, false>(a, h->sm_count, s);
-        default: return ss ? launch_gather_lpr<T, 32, true>(a, h->sm_count, s) : launch_gather_lpr<T, 32, false>(a, h->sm_count, s);
+        case 4: return ss ? launch_gather_lpr<T, 4, true>(a, sg, h->sm_count, s) : launch_gather_lpr<T, 4, false>(a, sg, h->sm_count, s);
+        case 8: return ss ? launch_gather_lpr<T, 8, true>(a, sg, h->sm_count, s) : launch_gather_lpr<T, 8, false>(a, sg, h->sm_count, s);
+        case 16: return ss ? launch_gather_lpr<T, 16, true>(a, sg, h->sm_count, s) : launch_gather_lpr<T, 16, false>(a, sg, h->sm_count, s);
+        default: return ss ? launch_gather_lpr<T, 32, true>(a, sg, h->sm_count, s) : launch_gather_lpr<T, 32, false>(a, sg, h->sm_count, s);
     }
 }
 
@@ -217,7 +272,7 @@ hag_status check_call(const hag *h, hag_dtype dtype, int32_t D, const void *in, 
 // level by level with the pair kernel, every deeper node in one gather launch
 // from its expansion.  rec may be null (no bookkeeping).
 template <typename T>
-hag_status enqueue_fwd_agg(const hag *h, int32_t D, const void *x, float *ws, cudaStream_t s, Recorder *rec) {
+hag_status enqueue_fwd_agg(const hag *h, int32_t D, const void *x, float *ws, float *partial, cudaStream_t s, Recorder *rec) {
     const int n_chunks = D / hagk::Chunk<T>::kElems;
     const hag_device_arrays &d = h->d;
     for (int32_t l = 1; l <= h->fwd_cut; ++l) {
@@ -249,7 +304,7 @@ hag_status enqueue_fwd_agg(const hag *h, int32_t D, const void *x, float *ws, cu
         a.out_is_f32 = 1;
         a.D = D;
         if (rec) rec->begin(1, a.row_count, int64_t(h->ftail_idx.size()));
-        if (launch_gather<T>(h, a, int64_t(h->ftail_idx.size()), n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+        if (launch_gather<T>(h, a, h->seg_ftail, partial, int64_t(h->ftail_idx.size()), n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
         if (rec) rec->end();
     }
     return HAG_OK;
@@ -269,9 +324,11 @@ hag_status fwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
     a.out = out;
     a.D = D;
     a.n_prim = std::numeric_limits<int32_t>::max();
+    // workspace layout: rows of the aggregation nodes (HAG calls only), then the partial rows of long-row segments
+    float *partial = static_cast<float *>(ws) + (use_hag ? size_t(h->num_agg) * D : 0);
     if (use_hag) {
         if (h->num_agg > 0) {
-            hag_status st = enqueue_fwd_agg<T>(h, D, x, static_cast<float *>(ws), s, rec);
+            hag_status st = enqueue_fwd_agg<T>(h, D, x, static_cast<float *>(ws), partial, s, rec);
             if (st != HAG_OK) return st;
             a.sec = static_cast<const float *>(ws);
             a.n_prim = h->n;
@@ -284,7 +341,7 @@ hag_status fwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
     }
     if (h->n > 0) {
         if (rec) rec->begin(2, h->n, use_hag ? h->e_res : h->e);
-        if (launch_gather<T>(h, a, use_hag ? h->e_res : h->e, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+        if (launch_gather<T>(h, a, use_hag ? h->seg_res : h->seg_csr, partial, use_hag ? h->e_res : h->e, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
         if (rec) rec->end();
     }
     return HAG_OK;
@@ -306,6 +363,7 @@ hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
     a.src_scale = (reduce == HAG_MEAN) ? d.inv_degree : nullptr;
     a.D = D;
     a.n_prim = std::numeric_limits<int32_t>::max();
+    float *partial = static_cast<float *>(ws) + (use_hag ? size_t(h->num_agg) * D : 0);
     if (use_hag && h->num_agg > 0) {
         const int32_t j0 = int32_t(h->level_ptr[h->bwd_cut]);
         if (j0 < h->num_agg) {
@@ -318,7 +376,7 @@ hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
             t.out_row_offset = h->n;
             t.out_is_f32 = 1;
             if (rec) rec->begin(1, t.row_count, int64_t(h->btail_idx.size()));
-            if (launch_gather<T>(h, t, int64_t(h->btail_idx.size()), n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+            if (launch_gather<T>(h, t, h->seg_btail, partial, int64_t(h->btail_idx.size()), n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
             if (rec) rec->end();
         }
         a.row_ptr = d.t_ptr;
@@ -335,7 +393,7 @@ hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
             if (lv.row_count <= 0) continue;
             const int64_t lv_edges = h->t_ptr[size_t(lv.row_begin) + lv.row_count] - h->t_ptr[lv.row_begin];
             if (rec) rec->begin(1, lv.row_count, lv_edges);
-            if (launch_gather<T>(h, lv, lv_edges, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+            if (launch_gather<T>(h, lv, h->seg_t, partial, lv_edges, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
             if (rec) rec->end();
         }
     } else if (use_hag) {
@@ -350,7 +408,7 @@ hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
     a.out = gx;
     if (h->n > 0) {
         if (rec) rec->begin(2, h->n, use_hag ? h->t_ptr[h->n] : h->e);
-        if (launch_gather<T>(h, a, use_hag ? h->t_ptr[h->n] : h->e, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+        if (launch_gather<T>(h, a, use_hag ? h->seg_t : h->seg_csr_t, partial, use_hag ? h->t_ptr[h->n] : h->e, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
         if (rec) rec->end();
     }
     return HAG_OK;
@@ -361,7 +419,8 @@ hag_status run(const hag *h, bool backward, bool use_hag, hag_reduce reduce, hag
     hag_status st = check_call(h, dtype, D, in, out);
     if (st != HAG_OK) return st;
     if (reduce != HAG_SUM && reduce != HAG_MEAN) return HAG_ERR_ARG;
-    if (use_hag && h->num_agg > 0) {
+    const bool needs_ws = use_hag ? (h->num_agg > 0 || h->max_segs_hag > 0) : (h->max_segs_csr > 0);
+    if (needs_ws) {
         if (!ws) return HAG_ERR_WORKSPACE;
         if (!aligned16(ws)) return HAG_ERR_ALIGN;
     }
@@ -441,6 +500,19 @@ extern "C" hag_status hag_to_device(hag_t *h, int device) {
             st = HAG_ERR_CUDA;
         }
     }
+    for (seg_set *set : {&h->seg_res, &h->seg_t, &h->seg_csr, &h->seg_csr_t, &h->seg_ftail, &h->seg_btail})
+    for (seg_table *t = set->g; t != set->g + kSegGrans; ++t) {
+        if (st != HAG_OK || t->segs.empty()) continue;
+        st = upload_i32(&t->d_segs, t->segs.data(), t->segs.size());
+        if (st == HAG_OK) st = upload_i32(&t->d_slots, t->slots.data(), t->slots.size());
+        if (st == HAG_OK) {
+            const size_t bytes = (t->slots.size() / 2) * sizeof(unsigned int);
+            if (cudaMalloc(reinterpret_cast<void **>(&t->d_done), bytes) != cudaSuccess || cudaMemset(t->d_done, 0, bytes) != cudaSuccess) {
+                cudaGetLastError();
+                st = HAG_ERR_CUDA;
+            }
+        }
+    }
     if (st == HAG_OK) {
         const size_t bytes = size_t(2) * kSchedSlots * sizeof(unsigned int);
         if (cudaMalloc(reinterpret_cast<void **>(&d.sched), bytes) != cudaSuccess || cudaMemset(d.sched, 0, bytes) != cudaSuccess ||
@@ -459,7 +531,12 @@ extern "C" hag_status hag_to_device(hag_t *h, int device) {
 
 extern "C" size_t hag_workspace_bytes(const hag_t *h, int32_t D) {
     if (!h || D <= 0) return 0;
-    return size_t(h->num_agg) * size_t(D) * sizeof(float);
+    return (size_t(h->num_agg) + size_t(h->max_segs_hag)) * size_t(D) * sizeof(float);
+}
+
+extern "C" size_t csr_workspace_bytes(const hag_t *h, int32_t D) {
+    if (!h || D <= 0) return 0;
+    return size_t(h->max_segs_csr) * size_t(D) * sizeof(float);
 }
 
 extern "C" hag_status hag_aggregate_fwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D, const void *x,
@@ -473,13 +550,13 @@ extern "C" hag_status hag_aggregate_bwd(const hag_t *h, hag_reduce reduce, hag_d
 }
 
 extern "C" hag_status csr_aggregate_fwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D, const void *x,
-                                        void *out, void *cuda_stream) {
-    return run(h, false, false, reduce, dtype, D, x, out, nullptr, cuda_stream);
+                                        void *out, void *workspace, void *cuda_stream) {
+    return run(h, false, false, reduce, dtype, D, x, out, workspace, cuda_stream);
 }
 
 extern "C" hag_status csr_aggregate_bwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D,
-                                        const void *grad_out, void *grad_x, void *cuda_stream) {
-    return run(h, true, false, reduce, dtype, D, grad_out, grad_x, nullptr, cuda_stream);
+                                        const void *grad_out, void *grad_x, void *workspace, void *cuda_stream) {
+    return run(h, true, false, reduce, dtype, D, grad_out, grad_x, workspace, cuda_stream);
 }
 
 extern "C" hag_status hag_aggregate_host(hag_t *h, int backward, int use_hag, hag_reduce reduce, hag_dtype dtype,
@@ -494,7 +571,8 @@ extern "C" hag_status hag_aggregate_host(hag_t *h, int backward, int use_hag, ha
     hag_device_arrays &d = h->d;
     hag_status st = grow(&d.stage_in, &d.stage_in_bytes, std::max<size_t>(bytes, 16));
     if (st == HAG_OK) st = grow(&d.stage_out, &d.stage_out_bytes, std::max<size_t>(bytes, 16));
-    if (st == HAG_OK) st = grow(&d.stage_ws, &d.stage_ws_bytes, std::max<size_t>(hag_workspace_bytes(h, D), 16));
+    if (st == HAG_OK)
+        st = grow(&d.stage_ws, &d.stage_ws_bytes, std::max<size_t>(std::max(hag_workspace_bytes(h, D), csr_workspace_bytes(h, D)), 16));
     if (st != HAG_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     if (bytes && cudaMemcpyAsync(d.stage_in, in_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
@@ -582,7 +660,7 @@ extern "C" hag_status hag_aggregate_fwd_static(const hag_t *h, hag_reduce reduce
     hag_status st = check_call(h, dtype, D, x, out);
     if (st != HAG_OK) return st;
     if (reduce != HAG_SUM && reduce != HAG_MEAN) return HAG_ERR_ARG;
-    if (size_t(h->num_agg) * size_t(D) * sizeof(float) > size_t(HAG_STATIC_SCRATCH_BYTES)) return HAG_ERR_TOO_LARGE;
+    if (hag_workspace_bytes(h, D) > size_t(HAG_STATIC_SCRATCH_BYTES)) return HAG_ERR_TOO_LARGE;
     DeviceGuard guard(h->device);
     if (!guard.ok) { cudaGetLastError(); return HAG_ERR_CUDA; }
     void *scratch = nullptr;

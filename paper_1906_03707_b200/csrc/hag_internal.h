@@ -8,6 +8,33 @@
 
 #include "hag.h"
 
+// Segments of the long rows of one CSR-like table (see hag_kernels.cuh): host copy and device copy.
+struct seg_table {
+    std::vector<int32_t> segs;    // 4 per segment: row id, first entry, end entry, slot
+    std::vector<int32_t> slots;   // 2 per long row: first segment, number of segments
+    int32_t *d_segs = nullptr;
+    int32_t *d_slots = nullptr;
+    unsigned int *d_done = nullptr;
+    int64_t count() const { return int64_t(segs.size() / 4); }
+};
+
+// Three granularities of splitting, chosen per launch by its number of rows: a launch that cannot fill the
+// machine with whole rows is split finely (more parallel work, at the price of a partial row and a completion
+// count per segment); a launch with rows to spare only splits what would otherwise stick out as a tail.
+constexpr int kSegGrans = 3;
+constexpr int32_t kSegLongRow[kSegGrans] = {64, 256, 1024};   // rows with more entries are split ...
+constexpr int32_t kSegLength[kSegGrans] = {32, 128, 512};     // ... into segments of this many entries
+inline int seg_gran_for_rows(int64_t rows) { return rows < 8192 ? 0 : (rows < 65536 ? 1 : 2); }
+
+struct seg_set {
+    seg_table g[kSegGrans];
+    int64_t max_count() const {
+        int64_t m = 0;
+        for (const seg_table &t : g) m = m > t.count() ? m : t.count();
+        return m;
+    }
+};
+
 constexpr int kSchedSlots = 64;      // far more than the kernels that can overlap on one stream
 
 struct hag_device_arrays {
@@ -52,6 +79,8 @@ struct hag {
     int32_t fwd_cut = 0, bwd_cut = 0;
     std::vector<int64_t> ftail_ptr, btail_ptr;
     std::vector<int32_t> ftail_idx, btail_idx;
+    seg_set seg_res, seg_t, seg_csr, seg_csr_t, seg_ftail, seg_btail;
+    int64_t max_segs_hag = 0, max_segs_csr = 0;   // partial rows the HAG / plain calls need in the workspace
     hag_info info{};
     int device = -1;
     hag_device_arrays d;

@@ -51,6 +51,23 @@ struct GatherArgs {
     int32_t resident;         // host-side choice of the launch form; the kernels ignore it
 };
 
+// Long rows (more than long_row entries) are not walked by one warp: they are cut into segments that
+// different warps sum into fp32 partial rows; whoever finishes a row's last segment adds them up.
+// Passed to the kernels as a parameter of its own, and only to the instantiations that handle long
+// rows: growing GatherArgs itself costs the plain row kernels registers.
+struct SegArgs {
+    int32_t long_row;
+    int32_t seg_first;        // index (in the table) of this launch's first segment
+    int32_t seg_count;        // segments of this launch
+    const int4 *segs;         // this launch's segments: {row, first entry, end entry, slot of the row}
+    const int2 *slots;        // per long row of the table: {index of its first segment, number of segments}
+    unsigned int *seg_done;   // per long row: finished segments (zero between launches)
+    float *partial;           // fp32 partial rows, indexed by the segment's index in its table
+};
+
+template <bool HAS_SEGS> struct KernelArgs { GatherArgs a; };
+template <> struct KernelArgs<true> { GatherArgs a; SegArgs sg; };
+
 template <typename T> struct Chunk;
 template <> struct Chunk<float> { static constexpr int kElems = 4; };
 template <> struct Chunk<__nv_bfloat16> { static constexpr int kElems = 8; };
@@ -253,29 +270,107 @@ __device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int
     }
 }
 
+// One segment of a long row: partial sum into a.partial, then, if this was the row's last open
+// segment, the fixed-order sum of all its partials into the output.  The completion count is an
+// integer atomic; the order of the floating-point additions never depends on who finishes when.
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE>
+__device__ __forceinline__ void gather_segment(const GatherArgs &a, const SegArgs &sa, int32_t seg_local, int lane) {
+    constexpr int E = Chunk<T>::kElems;
+    const int4 sg = __ldg(sa.segs + seg_local);
+    const int32_t row = sg.x, b = sg.y, e = sg.z, slot = sg.w;
+    GatherArgs part = a;
+    part.out = sa.partial;
+    part.out_is_f32 = 1;
+    part.out_row_offset = 0;
+    RowHead head = load_head<SRC_SCALE>(a, row, b, e, lane);
+    head.dst_scale = 1.0f;
+    gather_row<T, LPR, UNROLL, SRC_SCALE>(part, sa.seg_first + seg_local, b, e, head, lane);
+    __threadfence();                                   // partial row visible before the count moves
+    __syncwarp();
+    const int2 sl = __ldg(sa.slots + slot);
+    unsigned done = 0;
+    if (lane == 0) done = atomicAdd(sa.seg_done + slot, 1u);
+    done = __shfl_sync(0xffffffffu, done, 0);
+    if (done != unsigned(sl.y) - 1u) return;
+    __threadfence();
+    if (lane == 0) sa.seg_done[slot] = 0;              // ready for the next launch
+    const float dscale = a.dst_scale ? __ldg(a.dst_scale + row) : 1.0f;
+    const int n_chunks = a.D / E;
+    for (int chunk = lane; chunk < n_chunks; chunk += 32) {
+        float acc[E];
+#pragma unroll
+        for (int j = 0; j < E; ++j) acc[j] = 0.0f;
+        for (int k = 0; k < sl.y; ++k) {
+            const float *p = sa.partial + size_t(sl.x + k) * a.D + chunk * E;
+#pragma unroll
+            for (int j = 0; j < E; j += 4) {
+                const float4 q = __ldcg(reinterpret_cast<const float4 *>(p + j));   // written by other SMs: read at L2
+                acc[j] += q.x; acc[j + 1] += q.y; acc[j + 2] += q.z; acc[j + 3] += q.w;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < E; ++j) acc[j] *= dscale;
+        store_chunk<T>(a.out, a.out_is_f32, a.D, row - a.out_row_offset, chunk, acc);
+    }
+}
+
+// Out of line on purpose: the row path of the kernels keeps its registers and code.
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE>
+__device__ __noinline__ void gather_segment_call(const GatherArgs &a, const SegArgs &sa, int32_t seg_local, int lane) {
+    gather_segment<T, LPR, UNROLL, SRC_SCALE>(a, sa, seg_local, lane);
+}
+
 // out[row] = (dst_scale[row]) * sum_{e in row} (src_scale[id_e]) * table[id_e]
-// One warp per row, one launch-time row per warp.
-template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS>
-__global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_kernel(const GatherArgs a) {
+// One warp per work item, one item per launched warp.  HAS_SEGS: the launch has long rows; their
+// segments are the first items, and rows longer than a.long_row are left to them.  Without long
+// rows the kernel is compiled without any of that.
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, bool HAS_SEGS>
+__device__ __forceinline__ void gather_sum_body(const KernelArgs<HAS_SEGS> &k) {
+    const GatherArgs &a = k.a;
     pdl_launch_dependents();
     const int lane = threadIdx.x & 31;
-    const int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if constexpr (HAS_SEGS) {
+        if (r_local < k.sg.seg_count) {
+            pdl_wait();
+            gather_segment_call<T, LPR, UNROLL, SRC_SCALE>(a, k.sg, r_local, lane);
+            return;
+        }
+        r_local -= k.sg.seg_count;
+    }
     if (r_local >= a.row_count) return;
     const int32_t row = a.row_begin + r_local;
     const int32_t b = __ldg(a.row_ptr + row), e = __ldg(a.row_ptr + row + 1);
+    if constexpr (HAS_SEGS) {
+        if (e - b > k.sg.long_row) return;
+    }
     const RowHead head = load_head<SRC_SCALE>(a, row, b, e, lane);
     pdl_wait();        // structure arrays are static; features may come from the previous kernel
     gather_row<T, LPR, UNROLL, SRC_SCALE>(a, row, b, e, head, lane);
 }
 
-// The same, with resident warps that take rows four at a time from a shared
-// counter (a.sched[0]) and fetch the next row's pointers and first ids while the
-// current row is summed, so the pointer -> ids -> rows latency chain is paid once
-// per warp instead of once per row.  The last warp to finish zeroes the counters
-// (a.sched[1] counts finished warps) for the slot's next use.  No warp waits on
-// another: there is no spin anywhere.
+// Two entry points per form: the parameter block of the variant with long rows is declared
+// __grid_constant__ (its address is handed to the out-of-line segment function without a local
+// copy); the variant without long rows takes plain parameters, which costs it fewer registers.
 template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS>
-__global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_persistent_kernel(const GatherArgs a) {
+__global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_kernel(const KernelArgs<false> k) {
+    gather_sum_body<T, LPR, UNROLL, SRC_SCALE, false>(k);
+}
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS>
+__global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_long_kernel(const __grid_constant__ KernelArgs<true> k) {
+    gather_sum_body<T, LPR, UNROLL, SRC_SCALE, true>(k);
+}
+
+// The same, with resident warps that take items four at a time from a shared
+// counter (a.sched[0]): first the segments of the long rows if there are any (the
+// longest work goes first), then the rows, for which the next row's pointers and
+// first ids are fetched while the current row is summed, so the pointer -> ids ->
+// rows latency chain is paid once per warp instead of once per row.  The last warp
+// to finish zeroes the counters (a.sched[1] counts finished warps) for the slot's
+// next use.  No warp waits on another: there is no spin anywhere.
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, bool HAS_SEGS>
+__device__ __forceinline__ void gather_sum_persistent_body(const KernelArgs<HAS_SEGS> &k) {
+    const GatherArgs &a = k.a;
     pdl_launch_dependents();
     constexpr int CH = 4;
     constexpr unsigned FULL = 0xffffffffu;
@@ -290,11 +385,23 @@ __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_persistent_ke
     auto load_rp = [&](int32_t base) -> int32_t {   // lane i <= CH: pointer of row base + i (clamped to the end)
         return (lane <= CH && base < count) ? __ldg(rp_base + min(base + lane, count)) : 0;
     };
+    int32_t seg_items = 0;
     int32_t base = __shfl_sync(FULL, grab(), 0);
+    if constexpr (HAS_SEGS) {
+        seg_items = (k.sg.seg_count + CH - 1) / CH * CH;    // segments occupy whole grabs
+        pdl_wait();
+        while (base < seg_items) {                          // each segment is long: no pipelining needed
+#pragma unroll 1
+            for (int i = 0; i < CH; ++i)
+                if (base + i < k.sg.seg_count) gather_segment_call<T, LPR, UNROLL, SRC_SCALE>(a, k.sg, base + i, lane);
+            base = __shfl_sync(FULL, grab(), 0);
+        }
+        base -= seg_items;
+    }
     int32_t rp = load_rp(base);
     RowHead head{-1, 1.0f, 1.0f};
     if (base < count) head = load_head<SRC_SCALE>(a, a.row_begin + base, __shfl_sync(FULL, rp, 0), __shfl_sync(FULL, rp, 1), lane);
-    pdl_wait();
+    if constexpr (!HAS_SEGS) pdl_wait();
     while (base < count) {
         const int32_t grabbed = grab();     // the next four rows; consumed after the first row below
         const int nrows = min(CH, count - base);
@@ -306,15 +413,17 @@ __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_persistent_ke
                 head = load_head<SRC_SCALE>(a, a.row_begin + base + i + 1, e, __shfl_sync(FULL, rp, i + 2), lane);
             } else {
                 if (nrows == 1) {
-                    nbase = __shfl_sync(FULL, grabbed, 0);
+                    nbase = __shfl_sync(FULL, grabbed, 0) - seg_items;
                     rp_next = load_rp(nbase);
                 }
                 const int32_t nb = __shfl_sync(FULL, rp_next, 0), ne = __shfl_sync(FULL, rp_next, 1);
                 if (nbase < count) head = load_head<SRC_SCALE>(a, a.row_begin + nbase, nb, ne, lane);
             }
-            gather_row<T, LPR, UNROLL, SRC_SCALE>(a, a.row_begin + base + i, b, e, cur, lane);
+            bool whole = true;
+            if constexpr (HAS_SEGS) whole = e - b <= k.sg.long_row;
+            if (whole) gather_row<T, LPR, UNROLL, SRC_SCALE>(a, a.row_begin + base + i, b, e, cur, lane);
             if (i == 0 && nrows > 1) {
-                nbase = __shfl_sync(FULL, grabbed, 0);
+                nbase = __shfl_sync(FULL, grabbed, 0) - seg_items;
                 rp_next = load_rp(nbase);
             }
         }
@@ -328,6 +437,15 @@ __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_persistent_ke
             a.sched[1] = 0;
         }
     }
+}
+
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS>
+__global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_persistent_kernel(const KernelArgs<false> k) {
+    gather_sum_persistent_body<T, LPR, UNROLL, SRC_SCALE, false>(k);
+}
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS>
+__global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_persistent_long_kernel(const __grid_constant__ KernelArgs<true> k) {
+    gather_sum_persistent_body<T, LPR, UNROLL, SRC_SCALE, true>(k);
 }
 
 // Level kernel of Algorithm 2 (lines 5-6): every aggregation node of one level is

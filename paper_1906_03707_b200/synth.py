@@ -376,7 +376,7 @@ def upstream_grad(seed: int, n: int, d: int, dist: str, dtype: str = "f32") -> n
 # the named workloads (full size by default, ``scale`` < 1 shrinks them)
 # --------------------------------------------------------------------------- #
 def workload(index: int, scale: float = 1.0, capacity_frac: float = 0.25) -> Workload:
-    """Workload ``index`` (1-5).  ``scale`` shrinks the node count while keeping the
+    """Workload ``index`` (1-5 are the named shapes, 6 a clique-union graph).  ``scale`` shrinks the node count while keeping the
     generator, degree law, community size and feature shape."""
     if index == 1:
         n = max(200, int(round(1000 * scale)) // 100 * 100)
@@ -399,4 +399,11 @@ def workload(index: int, scale: float = 1.0, capacity_frac: float = 0.25) -> Wor
         g = config5_graph(seed=4, n=n, n_comm=max(2, int(round(2000 * scale))),
                           s_hi=max(120, min(20_000, n // 4)))
         return Workload(g, 256, "bf16", "sum", int(g.n * capacity_frac), "normal", 4, name="cfg5")
+    if index == 6:
+        # beyond the five named shapes: a union of cliques (co-authorship / shared-commenter projection), the regime
+        # of the paper's collaboration datasets: a deep hierarchy and a several-fold reduction of reads
+        n = max(2000, int(round(100_000 * scale)))
+        g = clique_union_graph(seed=5, n=n, n_groups=max(20, int(round(30_000 * scale))), g_lo=2,
+                               g_hi=max(20, min(400, n // 50)), g_alpha=2.3)
+        return Workload(g, 64, "f32", "sum", int(g.n * capacity_frac), "normal", 5, name="clique-union")
     raise ValueError(index)

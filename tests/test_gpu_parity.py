@@ -63,6 +63,7 @@ CASES = {
     "cfg3-small": lambda: synth.workload(3, scale=0.04),
     "cfg4-small": lambda: synth.workload(4, scale=0.01),
     "cfg5-small": lambda: synth.workload(5, scale=0.02),
+    "clique-union-small": lambda: synth.workload(6, scale=0.05),     # deep hierarchy (10+ levels)
 }
 _built = {}
 
@@ -128,7 +129,7 @@ def test_integer_features_are_bit_exact_for_sum(name):
 def test_capacity_zero_is_the_plain_path_bit_for_bit():
     g = synth.workload(2, scale=0.05).graph
     h = hb.Hag.build(g.row_ptr, g.col_idx, 0).to_device(0)
-    assert h.info()["num_agg"] == 0 and h.workspace_bytes(64) == 0
+    assert h.info()["num_agg"] == 0 and h.workspace_bytes(64) == h.csr_workspace_bytes(64)   # long-row partials only
     x = _dev(synth.features(3, g.n, 64, "normal"), "f32")
     for reduce in ("sum", "mean"):
         assert torch.equal(h.aggregate_fwd(x, reduce), h.csr_fwd(x, reduce))
@@ -187,6 +188,36 @@ def test_rows_without_neighbours_and_hubs():
         _check_all_paths(g, h, x, gr, reduce, "f32")
     out = h.aggregate_fwd(_dev(x, "f32"), "mean")
     assert not out[1:5].any()
+
+
+@pytest.mark.parametrize("dtype,d", [("f32", 16), ("f32", 64), ("f32", 128), ("f32", 516), ("bf16", 256)])
+def test_long_rows_are_split_and_still_exact(dtype, d):
+    # rows beyond a threshold are cut into segments summed by several warps and combined by whoever finishes
+    # last (64/32 entries for a launch this small; 256/128 and 1024/512 are met by the full-size shapes):
+    # lengths around the thresholds, and hubs far beyond them
+    n = 6000
+    lengths = {0: 256, 1: 257, 2: 384, 3: 385, 4: 1000, 5: 5999, 6: 129, 7: 3, 8: 64, 9: 65, 10: 96, 11: 97, 12: 33}
+    rng = np.random.default_rng(3)
+    rows = []
+    for v in range(n):
+        k = lengths.get(v, int(rng.integers(0, 12)))
+        rows.append(np.sort(rng.choice(n, size=k, replace=False)).tolist())
+    g = synth.csr_from_rows(rows)
+    h = hb.Hag.build(g.row_ptr, g.col_idx, n // 4).to_device(0)
+    assert h.csr_workspace_bytes(d) > 0 and h.workspace_bytes(d) > 0
+    x = synth.features(11, n, d, "normal", dtype)
+    gr = synth.upstream_grad(11, n, d, "normal", dtype)
+    for reduce in ("sum", "mean"):
+        _check_all_paths(g, h, x, gr, reduce, dtype)
+    if dtype == "f32":
+        xi = synth.features(12, n, d, "int")
+        a, _ = O.direct_forward(g.row_ptr, g.col_idx, xi.astype(np.float64), "sum")
+        b, _ = O.direct_backward(g.row_ptr, g.col_idx, xi.astype(np.float64), "sum")
+        for _ in range(2):      # twice: the completion counters must come back to zero
+            assert np.array_equal(_host(h.aggregate_fwd(_dev(xi, "f32"), "sum")), a)
+            assert np.array_equal(_host(h.csr_fwd(_dev(xi, "f32"), "sum")), a)
+            assert np.array_equal(_host(h.aggregate_bwd(_dev(xi, "f32"), "sum")), b)
+            assert np.array_equal(_host(h.csr_bwd(_dev(xi, "f32"), "sum")), b)
 
 
 def test_empty_graph_launches_nothing():

@@ -63,7 +63,8 @@ def test_static_scratch_rejects_what_does_not_fit_and_bad_arguments():
     w = synth.workload(2, scale=0.1)
     g = w.graph
     h = hb.Hag.build(g.row_ptr, g.col_idx, w.capacity).to_device(0)
-    k = h.info()["num_agg"]
+    k = h.workspace_bytes(4) // 16                                  # scratch rows: aggregation nodes + long-row partials
+    assert k >= h.info()["num_agg"] > 0
     d_big = 4 * (STATIC_SCRATCH_BYTES // (4 * k) // 4 + 1)          # smallest multiple of 4 that no longer fits
     assert k * d_big * 4 > STATIC_SCRATCH_BYTES
     x = torch.zeros((g.n, d_big), device="cuda")
