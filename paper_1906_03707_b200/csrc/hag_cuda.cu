@@ -93,7 +93,7 @@ cudaError_t launch_pdl(void (*kernel)(Args), unsigned grid, const Args &args, cu
 // B200 over the five workload shapes:
 //   fp32, large launch, 512-byte rows   : resident warps, 8 loads, 32 warps/SM
 //   fp32, large launch, narrower rows   : resident warps, 4 loads, 32 warps/SM
-//   fp32, small launch                  : one row per warp, 4 loads, 40 warps/SM
+//   fp32, small launch                  : one row per warp, 4 loads, 40 warps/SM (32 with per-source factors)
 // (large = at least 131072 rows or 4 Mi source entries)
 //   bf16                                : one row per warp, 2 loads, 48 warps/SM
 // Resident warps hide the pointer -> ids latency of the next row behind the
@@ -159,6 +159,8 @@ cudaError_t launch_gather_shape(const hagk::GatherArgs &ga, const hagk::SegArgs 
             if constexpr (LPR == 32) return launch_persistent(resident_kernel<T, LPR, 8, SS, 8, SEGS>(), a, items, sm_count, s);
             return launch_persistent(resident_kernel<T, LPR, 4, SS, 8, SEGS>(), a, items, sm_count, s);
         }
+        // the variant with per-source factors needs the registers of 8 CTAs per SM, or it spills
+        if constexpr (SS) return launch_pdl(plain_kernel<T, LPR, 4, SS, 8, SEGS>(), grid, a, s);
         return launch_pdl(plain_kernel<T, LPR, 4, SS, 10, SEGS>(), grid, a, s);
     } else {
         return launch_pdl(plain_kernel<T, LPR, 2, SS, 12, SEGS>(), grid, a, s);

@@ -98,6 +98,25 @@ __device__ __forceinline__ uint4 f32x8_to_bf16(const float *f) {
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
+// a[0..E) += b[0..E) as packed fp32x2 adds (one instruction per two sums on sm_100; each half is an
+// ordinary round-to-nearest add, so the bits are those of E scalar adds).
+// Used for fp32 storage (4 sums per chunk); with 8 sums per chunk (bf16 storage) the register pairs
+// it needs cost more in spills than the halved add count saves, so that path adds scalars.
+template <int E>
+__device__ __forceinline__ void add_rows(float *a, const float *b) {
+    if constexpr (E == 4) {
+#pragma unroll
+        for (int j = 0; j < E; j += 2) {
+            const float2 r = __fadd2_rn(make_float2(a[j], a[j + 1]), make_float2(b[j], b[j + 1]));
+            a[j] = r.x;
+            a[j + 1] = r.y;
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < E; ++j) a[j] += b[j];
+    }
+}
+
 // Per-lane view of the two source tables: byte pointers already offset to the
 // lane's chunk, so a row address is one multiply-add.
 template <typename T>
@@ -240,22 +259,12 @@ __device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int
 #pragma unroll
                     for (int w = U / 2; w >= 1; w /= 2)
 #pragma unroll
-                        for (int u = 0; u < w; ++u)
-#pragma unroll
-                            for (int j = 0; j < E; ++j) v[u][j] += v[u + w][j];
-                    if constexpr (E == 4) {
-#pragma unroll
-                        for (int j = 0; j < E; ++j) part[j] += v[0][j];
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < E; ++j) acc[j] += v[0][j];
-                    }
+                        for (int u = 0; u < w; ++u) add_rows<E>(v[u], v[u + w]);
+                    if constexpr (E == 4) add_rows<E>(part, v[0]);
+                    else add_rows<E>(acc, v[0]);
                 }
             }
-            if constexpr (E == 4) {
-#pragma unroll
-                for (int j = 0; j < E; ++j) acc[j] += part[j];
-            }
+            if constexpr (E == 4) add_rows<E>(acc, part);
         }
         // combine the slices (fixed butterfly), then slice 0 stores
 #pragma unroll
