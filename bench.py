@@ -191,6 +191,8 @@ def main():
     ap.add_argument("--workload", type=int, default=2, help="1-5: the named shapes (2 = the 50 000-node clustered power-law graph); 6: clique-union graph")
     ap.add_argument("--scale", type=float, default=1.0)
     ap.add_argument("--capacity-frac", type=float, default=0.25)
+    ap.add_argument("--min-redundancy", type=int, default=2,
+                    help="stop the search below this redundancy (2 = the paper's rule; 4 = no merge that loses bytes)")
     ap.add_argument("--capacity-sweep", action="store_true",
                     help="also time capacities 0, N/8, N/4, N/2 from ONE search (hag_truncate); reported under capacity_sweep")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -235,7 +237,7 @@ def main():
     w = synth.workload(args.workload, scale=args.scale, capacity_frac=args.capacity_frac)
     g = w.graph
     t0 = time.perf_counter()
-    h = hb.Hag.build(g.row_ptr, g.col_idx, w.capacity).to_device(local_rank)
+    h = hb.Hag.build(g.row_ptr, g.col_idx, w.capacity, min_redundancy=args.min_redundancy).to_device(local_rank)
     build_s = time.perf_counter() - t0
     info = h.info()
     arr = h.arrays()
@@ -417,7 +419,8 @@ def main():
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {
                 "workload": f"{w.name}: {g.name}, N={g.n}, E={info['e']}, D={w.d}, {w.dtype} storage, {w.reduce}, "
-                            f"|V_A|={info['num_agg']} (capacity {w.capacity}), {w.layers} layer(s), fwd+bwd",
+                            f"|V_A|={info['num_agg']} (capacity {w.capacity}, stop below redundancy "
+                            f"{args.min_redundancy}), {w.layers} layer(s), fwd+bwd",
                 "l2": "flushed between timed steps (256 MiB write outside the per-step events)",
                 "timing": "sum of per-step CUDA-event intervals on the launching stream, max over ranks",
                 "clocks": "nvidia-smi sampled every 100 ms across the GPU arms (HAG/plain x cold/warm, per-kernel pass)",

@@ -134,6 +134,15 @@ typedef struct hag_arrays {
  * 2^31); HAG_ERR_GRAPH; HAG_ERR_OOM_HOST.  On error *out is NULL. */
 hag_status hag_build(int32_t n, const int64_t *row_ptr, const int32_t *col_idx, int32_t capacity, hag_t **out);
 
+/* hag_build with a different stop value (an extension: the paper stops at redundancy 1).
+ * Merging a pair shared by r rows removes r - 2 row reads but adds one row write and, later,
+ * re-reads of the new row: it saves aggregations for every r >= 2 (the paper's cost function) but
+ * bytes only from r >= 4 on.  The search stops as soon as the best redundancy is below
+ * min_redundancy (>= 2; 2 reproduces hag_build exactly) or `capacity` nodes exist.
+ * HAG_ERR_ARG if min_redundancy < 2; otherwise as hag_build. */
+hag_status hag_build_ex(int32_t n, const int64_t *row_ptr, const int32_t *col_idx, int32_t capacity,
+                        int32_t min_redundancy, hag_t **out);
+
 /* Host threads hag_build may use for recounting pair redundancies (process-wide).
  * 0 = as many as the host has, at most 16 (the default); 1 = single-threaded;
  * a negative value only queries.  Returns the previous setting.  The merge

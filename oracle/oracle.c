@@ -285,8 +285,10 @@ typedef struct { int32_t *v; int32_t len; } ilist;
  *                  v1 < v2) and its redundancy, in creation order;
  *   cur_len[n], cur_idx[E]: on return row u's remaining in-neighbours (creation
  *                  ids, ascending) are cur_idx[row_ptr[u] .. row_ptr[u]+cur_len[u]).
+ *   min_redundancy: 2 is Algorithm 3 as printed; larger values stop the loop earlier (an
+ *                  option of the library, not of the paper);
  *   final_max_redundancy: the largest redundancy left when the loop stopped.  */
-int64_t o3b_greedy(int64_t n, const int64_t *row_ptr, const int32_t *col, int64_t capacity,
+int64_t o3b_greedy(int64_t n, const int64_t *row_ptr, const int32_t *col, int64_t capacity, int32_t min_redundancy,
                    int32_t *trace_v1, int32_t *trace_v2, int32_t *trace_r,
                    int32_t *cur_len, int32_t *cur_idx, int32_t *final_max_redundancy)
 {
@@ -344,7 +346,10 @@ int64_t o3b_greedy(int64_t n, const int64_t *row_ptr, const int32_t *col, int64_
             if (!c) { rc = -1; goto done; }
             if (*c == top.cnt) { found = 1; break; }
         }
-        if (!found || top.cnt <= 1) break;                     /* "if Redundancy > 1" */
+        if (!found || top.cnt < min_redundancy) {              /* "if Redundancy > 1" when min_redundancy is 2 */
+            if (found) h_push(&hp, top);                       /* keep it for the final maximum below */
+            break;
+        }
         int32_t v1 = top.a, v2 = top.b, w = (int32_t)(n + num_agg);
 
         /* R = { u : (v1,u) and (v2,u) are edges } */

@@ -73,7 +73,7 @@ def _c():
         lib.o_count_pair.restype = i64
         lib.o_max_pair_recount.argtypes = [i64, p, p, p, i64, i32, p, p]
         lib.o_max_pair_recount.restype = i64
-        lib.o3b_greedy.argtypes = [i64, p, p, i64, p, p, p, p, p, p]
+        lib.o3b_greedy.argtypes = [i64, p, p, i64, i32, p, p, p, p, p, p]
         lib.o3b_greedy.restype = i64
         _lib = lib
     return _lib
@@ -147,7 +147,7 @@ class SearchResult:
         return int(self.trace.shape[0])
 
 
-def greedy_bruteforce(row_ptr, col_idx, capacity) -> SearchResult:
+def greedy_bruteforce(row_ptr, col_idx, capacity, min_redundancy=2) -> SearchResult:
     """Algorithm 3 exactly as stated: every iteration recounts, for every
     unordered pair, how many graph nodes aggregate both; takes the largest
     (ties: smallest v1, then smallest v2); stops at redundancy <= 1."""
@@ -169,7 +169,7 @@ def greedy_bruteforce(row_ptr, col_idx, capacity) -> SearchResult:
             if c > best or (c == best and key < best_pair):
                 best_pair, best = key, c
         last_max = best
-        if len(trace) >= capacity or best <= 1:
+        if len(trace) >= capacity or best < min_redundancy:     # 2: the paper's "Redundancy > 1"
             break
         v1, v2 = best_pair
         w = n + len(trace)
@@ -183,7 +183,7 @@ def greedy_bruteforce(row_ptr, col_idx, capacity) -> SearchResult:
     return SearchResult(n, tr, [np.asarray(sorted(r), dtype=np.int32) for r in rows], int(last_max))
 
 
-def greedy_pairmap(row_ptr, col_idx, capacity) -> SearchResult:
+def greedy_pairmap(row_ptr, col_idx, capacity, min_redundancy=2) -> SearchResult:
     """Algorithm 3 with the pair-count map and heap of the complexity appendix (C)."""
     rp, ci = _csr(row_ptr, col_idx)
     n = rp.shape[0] - 1
@@ -194,7 +194,7 @@ def greedy_pairmap(row_ptr, col_idx, capacity) -> SearchResult:
     cur_len = np.zeros(max(n, 1), dtype=np.int32)
     cur_idx = np.zeros(max(ci.shape[0], 1), dtype=np.int32)
     fin = np.zeros(1, dtype=np.int32)
-    k = _c().o3b_greedy(n, _ptr(rp), _ptr(ci), cap, _ptr(t1), _ptr(t2), _ptr(tr), _ptr(cur_len), _ptr(cur_idx), _ptr(fin))
+    k = _c().o3b_greedy(n, _ptr(rp), _ptr(ci), cap, int(min_redundancy), _ptr(t1), _ptr(t2), _ptr(tr), _ptr(cur_len), _ptr(cur_idx), _ptr(fin))
     if k < 0:
         raise MemoryError(f"o3b_greedy failed with code {k}")
     trace = np.stack([t1[:k], t2[:k], tr[:k]], axis=1).astype(np.int32).reshape(-1, 3)

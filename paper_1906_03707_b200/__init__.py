@@ -24,7 +24,7 @@ HAG_SUM, HAG_MEAN = 0, 1
 HAG_F32, HAG_BF16 = 0, 1
 
 EXPORTED_SYMBOLS = [
-    "hag_build", "hag_build_threads", "hag_truncate", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes", "csr_workspace_bytes",
+    "hag_build", "hag_build_ex", "hag_build_threads", "hag_truncate", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes", "csr_workspace_bytes",
     "hag_aggregate_fwd", "hag_aggregate_bwd", "csr_aggregate_fwd", "csr_aggregate_bwd",
     "hag_aggregate_host", "hag_aggregate_fwd_static", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
 ]
@@ -75,6 +75,8 @@ def load_library():
     vp, i32 = ctypes.c_void_p, ctypes.c_int32
     lib.hag_build.argtypes = [i32, vp, vp, i32, ctypes.POINTER(vp)]
     lib.hag_build.restype = ctypes.c_int
+    lib.hag_build_ex.argtypes = [i32, vp, vp, i32, i32, ctypes.POINTER(vp)]
+    lib.hag_build_ex.restype = ctypes.c_int
     lib.hag_build_threads.argtypes = [i32]
     lib.hag_build_threads.restype = i32
     lib.hag_truncate.argtypes = [vp, i32, ctypes.POINTER(vp)]
@@ -149,14 +151,15 @@ class Hag:
 
     # -- construction ------------------------------------------------------- #
     @classmethod
-    def build(cls, row_ptr, col_idx, capacity: int) -> "Hag":
-        """``hag_build``: CSR of in-neighbours on the host (int64 row_ptr, int32 col_idx)."""
+    def build(cls, row_ptr, col_idx, capacity: int, min_redundancy: int = 2) -> "Hag":
+        """``hag_build`` / ``hag_build_ex``: CSR of in-neighbours on the host (int64 row_ptr, int32 col_idx)."""
         lib = load_library()
         rp = np.ascontiguousarray(row_ptr, dtype=np.int64)
         ci = np.ascontiguousarray(col_idx, dtype=np.int32)
         handle = ctypes.c_void_p()
         n = rp.shape[0] - 1
-        st = lib.hag_build(n, rp.ctypes.data, ci.ctypes.data if ci.size else None, int(capacity), ctypes.byref(handle))
+        st = lib.hag_build_ex(n, rp.ctypes.data, ci.ctypes.data if ci.size else None, int(capacity),
+                              int(min_redundancy), ctypes.byref(handle))
         _check(st, "hag_build")
         return cls(handle)
 

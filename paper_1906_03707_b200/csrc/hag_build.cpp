@@ -239,7 +239,7 @@ struct Searcher {
     }
     ~Searcher() { stop_pool(); }
 
-    hag_status run(std::vector<int32_t> &trace, int threads) {
+    hag_status run(std::vector<int32_t> &trace, int threads, int32_t min_redundancy) {
         init_lists();
         start_pool(threads);
         const size_t max_batch = size_t(4) * n_threads;
@@ -256,7 +256,7 @@ struct Searcher {
             const int32_t k = int32_t(top >> 32);
             const int32_t x = int32_t(0x7fffffff - uint32_t(top & 0xffffffffu));
             if (k != key[x]) continue;              // superseded entry
-            if (k < 2) break;
+            if (k < min_redundancy) break;           // every bound is below the stop value: so is every pair
             if (dirty[x]) {
                 // gather the run of stale nodes at the top of the queue and recount them together
                 batch.clear();
@@ -321,7 +321,7 @@ hag_status hag_search(hag *h, std::vector<int32_t> &rows_store, std::vector<int3
         Searcher s(h->n, h->capacity, h->csr_ptr.data(), rows_store, rows_len);
         int threads = g_build_threads.load();
         if (threads <= 0) threads = int(std::min<unsigned>(std::max<unsigned>(std::thread::hardware_concurrency(), 1u), 16u));
-        hag_status st = s.run(h->trace, threads);
+        hag_status st = s.run(h->trace, threads, h->min_redundancy);
         if (st != HAG_OK) return st;
     } catch (const std::bad_alloc &) {
         return HAG_ERR_OOM_HOST;
@@ -557,8 +557,14 @@ hag_status hag_layout(hag *h, const std::vector<int32_t> &rows_store, const std:
 }
 
 extern "C" hag_status hag_build(int32_t n, const int64_t *row_ptr, const int32_t *col_idx, int32_t capacity, hag_t **out) {
+    return hag_build_ex(n, row_ptr, col_idx, capacity, 2, out);
+}
+
+extern "C" hag_status hag_build_ex(int32_t n, const int64_t *row_ptr, const int32_t *col_idx, int32_t capacity,
+                                   int32_t min_redundancy, hag_t **out) {
     if (!out) return HAG_ERR_NULL;
     *out = nullptr;
+    if (min_redundancy < 2) return HAG_ERR_ARG;
     if (!row_ptr || (!col_idx && n > 0 && row_ptr[n] > 0)) return HAG_ERR_NULL;
     if (n < 0 || capacity < 0) return HAG_ERR_ARG;
     if (int64_t(n) + int64_t(capacity) >= (int64_t(1) << 31)) return HAG_ERR_ARG;
@@ -583,6 +589,7 @@ extern "C" hag_status hag_build(int32_t n, const int64_t *row_ptr, const int32_t
     try {
         h->n = n;
         h->capacity = capacity;
+        h->min_redundancy = min_redundancy;
         h->e = e;
         h->csr_ptr.assign(row_ptr, row_ptr + n + 1);
         h->csr_idx.assign(col_idx, col_idx + e);
@@ -624,6 +631,7 @@ extern "C" hag_status hag_truncate(const hag_t *src, int32_t capacity, hag_t **o
         const int32_t k = std::min(capacity, src->num_agg);
         h->n = src->n;
         h->capacity = capacity;
+        h->min_redundancy = src->min_redundancy;
         h->e = src->e;
         h->csr_ptr = src->csr_ptr;
         h->csr_idx = src->csr_idx;

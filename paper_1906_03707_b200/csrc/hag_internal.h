@@ -62,6 +62,7 @@ struct hag_device_arrays {
 
 struct hag {
     int32_t n = 0, capacity = 0, num_agg = 0, num_levels = 0;
+    int32_t min_redundancy = 2;      // the search stops below this redundancy (2 = the paper's "> 1")
     int64_t e = 0, e_res = 0, e_hat = 0;
     std::vector<int64_t> csr_ptr;
     std::vector<int32_t> csr_idx;

@@ -214,3 +214,27 @@ def test_build_does_not_depend_on_the_thread_count():
         assert hb.build_threads(-1) == 0
     finally:
         hb.build_threads(prev)
+
+
+def test_min_redundancy_stops_the_search_earlier():
+    g = synth.config2_graph(seed=19, n=2500, n_comm=25)
+    for min_r in (2, 4, 9):
+        h = hb.Hag.build(g.row_ptr, g.col_idx, 10 * g.n, min_redundancy=min_r)
+        ref = O.greedy_pairmap(g.row_ptr, g.col_idx, 10 * g.n, min_redundancy=min_r)
+        arr = h.arrays()
+        assert arr["trace"].tolist() == ref.trace.tolist()
+        assert (arr["trace"][:, 2] >= min_r).all() and ref.final_max_redundancy < min_r
+        layout = O.canonical_hag(g.row_ptr, ref)
+        for key in ("level_ptr", "agg_in", "res_ptr", "res_idx", "t_ptr", "t_idx"):
+            assert np.array_equal(arr[key], getattr(layout, key)), key
+    small = synth.random_digraph(77, 24, 0.4, True, True)
+    for min_r in (2, 3, 5):
+        a = O.greedy_bruteforce(small.row_ptr, small.col_idx, 100, min_redundancy=min_r)
+        b = hb.Hag.build(small.row_ptr, small.col_idx, 100, min_redundancy=min_r).arrays()
+        assert a.trace.tolist() == b["trace"].tolist()
+    # with the default the extended entry point is hag_build
+    assert hb.Hag.build(g.row_ptr, g.col_idx, 100).arrays()["trace"].tolist() == \
+        hb.Hag.build(g.row_ptr, g.col_idx, 100, min_redundancy=2).arrays()["trace"].tolist()
+    lib = hb.load_library()
+    out = ctypes.c_void_p()
+    assert lib.hag_build_ex(g.n, g.row_ptr.ctypes.data, g.col_idx.ctypes.data, 10, 1, ctypes.byref(out)) == 2
