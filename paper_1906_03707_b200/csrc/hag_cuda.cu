@@ -217,7 +217,7 @@ template <typename T>
 cudaError_t launch_pairs(const hagk::PairArgs &p, int n_chunks, cudaStream_t s) {
     if (p.count <= 0) return cudaSuccess;
     const int lpr = lanes_per_row(n_chunks);
-    const int rows_per_cta = hagk::kWarps * (32 / lpr);
+    const int rows_per_cta = hagk::kWarps * (32 / lpr) * hagk::kPairBatch;
     const unsigned grid = unsigned((p.count + rows_per_cta - 1) / rows_per_cta);
     switch (lpr) {
         case 4: return launch_pdl(hagk::pair_sum_kernel<T, 4>, grid, p, s);

@@ -469,32 +469,47 @@ struct PairArgs {
     int32_t D;
 };
 
-template <typename T, int LPR>
-__device__ __forceinline__ void pair_row(const PairArgs &p, int32_t j, int gl, bool first_of_kernel) {
-    constexpr int E = Chunk<T>::kElems;
-    const int2 in = __ldg(reinterpret_cast<const int2 *>(p.agg_in) + j);
-    if (first_of_kernel) pdl_wait();
-    const int n_chunks = p.D / E;
-    for (int chunk = gl; chunk < n_chunks; chunk += LPR) {
-        const Tables<T> tab(p.x, p.ahat, p.n, p.D, chunk);
-        float u[E], v[E];
-        tab.load(in.x, u);
-        tab.load(in.y, v);
-        float *o = p.ahat + size_t(j) * p.D + chunk * E;
-#pragma unroll
-        for (int i = 0; i < E; i += 4)
-            *reinterpret_cast<float4 *>(o + i) = make_float4(u[i] + v[i], u[i + 1] + v[i + 1], u[i + 2] + v[i + 2], u[i + 3] + v[i + 3]);
-    }
-}
+// Nodes per lane group: their input pairs are fetched together and all their row loads are in
+// flight before the first add, so a group pays the pointer -> rows latency once for kPairBatch nodes.
+constexpr int kPairBatch = 4;
 
 template <typename T, int LPR>
 __global__ void __launch_bounds__(kThreads) pair_sum_kernel(const PairArgs p) {
     pdl_launch_dependents();
+    constexpr int E = Chunk<T>::kElems;
     constexpr int GROUPS = 32 / LPR;
     const int lane = threadIdx.x & 31;
-    const int j_local = (blockIdx.x * kWarps + (threadIdx.x >> 5)) * GROUPS + lane / LPR;
-    if (j_local >= p.count) return;
-    pair_row<T, LPR>(p, p.first + j_local, lane % LPR, true);
+    const int gl = lane % LPR;
+    const int64_t group = (int64_t(blockIdx.x) * kWarps + (threadIdx.x >> 5)) * GROUPS + lane / LPR;
+    const int32_t j0 = int32_t(group * kPairBatch);
+    if (j0 >= p.count) return;
+    int2 in[kPairBatch];
+#pragma unroll
+    for (int t = 0; t < kPairBatch; ++t)
+        in[t] = (j0 + t < p.count) ? __ldg(reinterpret_cast<const int2 *>(p.agg_in) + p.first + j0 + t) : make_int2(-1, -1);
+    pdl_wait();
+    const int n_chunks = p.D / E;
+    for (int chunk = gl; chunk < n_chunks; chunk += LPR) {
+        const Tables<T> tab(p.x, p.ahat, p.n, p.D, chunk);
+        float u[kPairBatch][E], v[kPairBatch][E];
+#pragma unroll
+        for (int t = 0; t < kPairBatch; ++t) {
+            if (in[t].x >= 0) {
+                tab.load(in[t].x, u[t]);
+                tab.load(in[t].y, v[t]);
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < kPairBatch; ++t) {
+            if (in[t].x >= 0) {
+                float *o = p.ahat + size_t(p.first + j0 + t) * p.D + chunk * E;
+#pragma unroll
+                for (int i = 0; i < E; i += 4)
+                    *reinterpret_cast<float4 *>(o + i) = make_float4(u[t][i] + v[t][i], u[t][i + 1] + v[t][i + 1],
+                                                                     u[t][i + 2] + v[t][i + 2], u[t][i + 3] + v[t][i + 3]);
+            }
+        }
+    }
 }
 
 }  // namespace hagk
