@@ -66,7 +66,12 @@ typedef enum {
     HAG_ERR_TOO_LARGE = 12     /* the problem needs more than the built-in scratch array holds */
 } hag_status;
 
-typedef enum { HAG_SUM = 0, HAG_MEAN = 1 } hag_reduce;
+/* HAG_SUM: a_v = sum of h_u over N(v) (GCN's Aggregate, Table 1).  HAG_MEAN: that sum / |N(v)|.
+ * HAG_GCN: the argument of GCN's Update in Table 1, (a_v + h_v) / (|N(v)| + 1), i.e. the sum with the
+ * node's own row added and the normalisation fused into the gather's epilogue (the weight matrix and the
+ * non-linearity stay with the caller).  Its gradient is gx_u = sum over v with u in N(v) of
+ * g_v / (|N(v)| + 1), plus g_u / (|N(u)| + 1). */
+typedef enum { HAG_SUM = 0, HAG_MEAN = 1, HAG_GCN = 2 } hag_reduce;
 typedef enum { HAG_F32 = 0, HAG_BF16 = 1 } hag_dtype;
 
 /* Counters of one built HAG.  "aggregations" are binary aggregations as counted

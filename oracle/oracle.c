@@ -7,7 +7,8 @@
  *
  * What each function follows in the paper (arxiv 1906.03707):
  *   o1_direct_forward   Algorithm 1 line 4 with the GCN row of Table 1:
- *                       a_v = sum over u in N(v) of h_u   (mean: divided by |N(v)|)
+ *                       a_v = sum over u in N(v) of h_u   (mode 1, mean: divided by |N(v)|;
+ *                       mode 2: the argument of GCN's Update, (a_v + h_v) / (|N(v)| + 1))
  *   o2_direct_backward  equivalence clause (2) of Section 3.2 ("the same
  *                       gradients"): gx_u = sum over v with u in N(v) of s_v g_v
  *   o4_hag_forward      Algorithm 2 lines 3-8, evaluated over a given HAG
@@ -46,9 +47,14 @@ void o1_direct_forward(int64_t n, const int64_t *row_ptr, const int32_t *col, in
             if (ao) for (int64_t k = 0; k < d; ++k) ao[k] += fabs(xu[k]);
         }
         int64_t deg = row_ptr[v + 1] - row_ptr[v];
-        if (mean && deg > 0) {
+        if (mean == 1 && deg > 0) {
             for (int64_t k = 0; k < d; ++k) o[k] /= (double)deg;
             if (ao) for (int64_t k = 0; k < d; ++k) ao[k] /= (double)deg;
+        }
+        if (mean == 2) {                 /* Table 1, GCN: (a_v + h_v) / (|N(v)| + 1) */
+            const double *xv = x + v * d;
+            for (int64_t k = 0; k < d; ++k) o[k] = (o[k] + xv[k]) / (double)(deg + 1);
+            if (ao) for (int64_t k = 0; k < d; ++k) ao[k] = (ao[k] + fabs(xv[k])) / (double)(deg + 1);
         }
     }
 }
@@ -65,8 +71,17 @@ void o2_direct_backward(int64_t n, const int64_t *row_ptr, const int32_t *col, i
     if (abs_gx) memset(abs_gx, 0, sizeof(double) * (size_t)(out_rows * d));
     for (int64_t v = 0; v < n; ++v) {
         int64_t deg = row_ptr[v + 1] - row_ptr[v];
-        double s = (mean && deg > 0) ? 1.0 / (double)deg : 1.0;
+        double s = (mean == 1 && deg > 0) ? 1.0 / (double)deg : 1.0;
+        if (mean == 2) s = 1.0 / (double)(deg + 1);
         const double *gv = g + v * d;
+        if (mean == 2) {                 /* the h_v term of (a_v + h_v) / (|N(v)| + 1) sends s_v g_v back to v itself */
+            int64_t r = slot ? slot[v] : v;
+            if (r >= 0) {
+                double *o = gx + r * d;
+                for (int64_t k = 0; k < d; ++k) o[k] += s * gv[k];
+                if (abs_gx) { double *ao = abs_gx + r * d; for (int64_t k = 0; k < d; ++k) ao[k] += fabs(s * gv[k]); }
+            }
+        }
         for (int64_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) {
             int64_t u = col[e];
             int64_t r = slot ? slot[u] : u;

@@ -79,6 +79,10 @@ def _c():
     return _lib
 
 
+def _mode(reduce) -> int:
+    return {"sum": 0, "mean": 1, "gcn": 2}[reduce]
+
+
 def _ptr(a):
     return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
 
@@ -104,7 +108,7 @@ def direct_forward(row_ptr, col_idx, x, reduce="sum", rows=None):
     m = n if sel is None else sel.shape[0]
     out = np.empty((m, d), dtype=np.float64)
     ab = np.empty((m, d), dtype=np.float64)
-    _c().o1_direct_forward(n, _ptr(rp), _ptr(ci), d, _ptr(x), int(reduce == "mean"), _ptr(sel), m, _ptr(out), _ptr(ab))
+    _c().o1_direct_forward(n, _ptr(rp), _ptr(ci), d, _ptr(x), _mode(reduce), _ptr(sel), m, _ptr(out), _ptr(ab))
     return out, ab
 
 
@@ -126,7 +130,7 @@ def direct_backward(row_ptr, col_idx, g, reduce="sum", rows=None):
             raise ValueError("rows must be distinct")
     out = np.empty((m, d), dtype=np.float64)
     ab = np.empty((m, d), dtype=np.float64)
-    _c().o2_direct_backward(n, _ptr(rp), _ptr(ci), d, _ptr(g), int(reduce == "mean"), _ptr(slot), m, _ptr(out), _ptr(ab))
+    _c().o2_direct_backward(n, _ptr(rp), _ptr(ci), d, _ptr(g), _mode(reduce), _ptr(slot), m, _ptr(out), _ptr(ab))
     return out, ab
 
 

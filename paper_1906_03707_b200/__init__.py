@@ -20,7 +20,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhag_b200.so")
 
-HAG_SUM, HAG_MEAN = 0, 1
+HAG_SUM, HAG_MEAN, HAG_GCN = 0, 1, 2
 HAG_F32, HAG_BF16 = 0, 1
 
 EXPORTED_SYMBOLS = [
@@ -132,7 +132,9 @@ def _reduce_code(reduce) -> int:
         return HAG_SUM
     if reduce in ("mean", HAG_MEAN):
         return HAG_MEAN
-    raise ValueError(f"reduce must be 'sum' or 'mean', got {reduce!r}")
+    if reduce in ("gcn", HAG_GCN):
+        return HAG_GCN
+    raise ValueError(f"reduce must be 'sum', 'mean' or 'gcn', got {reduce!r}")
 
 
 def _view(ptr, count, dtype):

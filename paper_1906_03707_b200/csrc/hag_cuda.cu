@@ -7,6 +7,7 @@
 #include <cstdlib>
 #include <limits>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "hag_internal.h"
@@ -59,7 +60,7 @@ void free_device(hag *h) {
         t->d_done = nullptr;
     }
     void *ptrs[] = {d.agg_in, d.res_ptr, d.res_idx, d.t_ptr, d.t_idx, d.csr_ptr, d.csr_idx, d.csr_t_ptr,
-                    d.csr_t_idx, d.inv_degree, d.stage_in, d.stage_out, d.stage_ws,
+                    d.csr_t_idx, d.inv_degree, d.inv_degree1, d.stage_in, d.stage_out, d.stage_ws,
                     d.ftail_ptr, d.ftail_idx, d.btail_ptr, d.btail_idx, d.sched};
     for (void *p : ptrs)
         if (p) cudaFree(p);
@@ -126,51 +127,54 @@ hagk::KernelArgs<SEGS> pack_args(const hagk::GatherArgs &a, const hagk::SegArgs 
 }
 
 // The kernel entry for a shape: plain parameters without long rows, grid-constant ones with.
-template <typename T, int LPR, int U, bool SS, int MINB, bool SEGS>
+template <typename T, int LPR, int U, bool SS, int MINB, bool SEGS, bool SELF>
 auto plain_kernel() {
-    if constexpr (SEGS) return hagk::gather_sum_long_kernel<T, LPR, U, SS, MINB>;
-    else return hagk::gather_sum_kernel<T, LPR, U, SS, MINB>;
+    if constexpr (SEGS) return hagk::gather_sum_long_kernel<T, LPR, U, SS, MINB, SELF>;
+    else return hagk::gather_sum_kernel<T, LPR, U, SS, MINB, SELF>;
 }
-template <typename T, int LPR, int U, bool SS, int MINB, bool SEGS>
+template <typename T, int LPR, int U, bool SS, int MINB, bool SEGS, bool SELF>
 auto resident_kernel() {
-    if constexpr (SEGS) return hagk::gather_sum_persistent_long_kernel<T, LPR, U, SS, MINB>;
-    else return hagk::gather_sum_persistent_kernel<T, LPR, U, SS, MINB>;
+    if constexpr (SEGS) return hagk::gather_sum_persistent_long_kernel<T, LPR, U, SS, MINB, SELF>;
+    else return hagk::gather_sum_persistent_kernel<T, LPR, U, SS, MINB, SELF>;
 }
 
-template <typename T, int LPR, bool SS, bool SEGS>
+template <typename T, int LPR, bool SS, bool SEGS, bool SELF>
 cudaError_t launch_gather_shape(const hagk::GatherArgs &ga, const hagk::SegArgs &sg, int sm_count, cudaStream_t s) {
     const hagk::KernelArgs<SEGS> a = pack_args<SEGS>(ga, sg);
     const int64_t items = int64_t(ga.row_count) + (SEGS ? sg.seg_count : 0);
     const unsigned grid = unsigned((items + hagk::kWarps - 1) / hagk::kWarps);
 #ifdef HAG_TUNING
     switch (g_tune) {
-        case 0: return launch_pdl(plain_kernel<T, LPR, 8, SS, 8, SEGS>(), grid, a, s);
-        case 2: return launch_pdl(plain_kernel<T, LPR, 4, SS, 12, SEGS>(), grid, a, s);
-        case 4: return launch_pdl(plain_kernel<T, LPR, 2, SS, 16, SEGS>(), grid, a, s);
-        case 5: return launch_pdl(plain_kernel<T, LPR, 4, SS, 10, SEGS>(), grid, a, s);
-        case 9: return launch_persistent(resident_kernel<T, LPR, 4, SS, 10, SEGS>(), a, items, sm_count, s);
-        case 10: return launch_persistent(resident_kernel<T, LPR, 4, SS, 8, SEGS>(), a, items, sm_count, s);
-        case 11: return launch_persistent(resident_kernel<T, LPR, 8, SS, 8, SEGS>(), a, items, sm_count, s);
+        case 0: return launch_pdl(plain_kernel<T, LPR, 8, SS, 8, SEGS, SELF>(), grid, a, s);
+        case 2: return launch_pdl(plain_kernel<T, LPR, 4, SS, 12, SEGS, SELF>(), grid, a, s);
+        case 4: return launch_pdl(plain_kernel<T, LPR, 2, SS, 16, SEGS, SELF>(), grid, a, s);
+        case 5: return launch_pdl(plain_kernel<T, LPR, 4, SS, 10, SEGS, SELF>(), grid, a, s);
+        case 9: return launch_persistent(resident_kernel<T, LPR, 4, SS, 10, SEGS, SELF>(), a, items, sm_count, s);
+        case 10: return launch_persistent(resident_kernel<T, LPR, 4, SS, 8, SEGS, SELF>(), a, items, sm_count, s);
+        case 11: return launch_persistent(resident_kernel<T, LPR, 8, SS, 8, SEGS, SELF>(), a, items, sm_count, s);
         default: break;
     }
 #endif
     if constexpr (sizeof(T) == 4) {
         if (ga.resident) {
-            if constexpr (LPR == 32) return launch_persistent(resident_kernel<T, LPR, 8, SS, 8, SEGS>(), a, items, sm_count, s);
-            return launch_persistent(resident_kernel<T, LPR, 4, SS, 8, SEGS>(), a, items, sm_count, s);
+            if constexpr (LPR == 32) return launch_persistent(resident_kernel<T, LPR, 8, SS, 8, SEGS, SELF>(), a, items, sm_count, s);
+            return launch_persistent(resident_kernel<T, LPR, 4, SS, 8, SEGS, SELF>(), a, items, sm_count, s);
         }
         // the variant with per-source factors needs the registers of 8 CTAs per SM, or it spills
-        if constexpr (SS) return launch_pdl(plain_kernel<T, LPR, 4, SS, 8, SEGS>(), grid, a, s);
-        return launch_pdl(plain_kernel<T, LPR, 4, SS, 10, SEGS>(), grid, a, s);
+        if constexpr (SS) return launch_pdl(plain_kernel<T, LPR, 4, SS, 8, SEGS, SELF>(), grid, a, s);
+        return launch_pdl(plain_kernel<T, LPR, 4, SS, 10, SEGS, SELF>(), grid, a, s);
     } else {
-        return launch_pdl(plain_kernel<T, LPR, 2, SS, 12, SEGS>(), grid, a, s);
+        return launch_pdl(plain_kernel<T, LPR, 2, SS, 12, SEGS, SELF>(), grid, a, s);
     }
 }
 
 template <typename T, int LPR, bool SS>
 cudaError_t launch_gather_lpr(const hagk::GatherArgs &a, const hagk::SegArgs &sg, int sm_count, cudaStream_t s) {
-    return sg.seg_count > 0 ? launch_gather_shape<T, LPR, SS, true>(a, sg, sm_count, s)
-                            : launch_gather_shape<T, LPR, SS, false>(a, sg, sm_count, s);
+    if (a.out_is_f32 & 2)   // GCN's own-row term: its own instantiations, so the others stay as they are
+        return sg.seg_count > 0 ? launch_gather_shape<T, LPR, SS, true, true>(a, sg, sm_count, s)
+                                : launch_gather_shape<T, LPR, SS, false, true>(a, sg, sm_count, s);
+    return sg.seg_count > 0 ? launch_gather_shape<T, LPR, SS, true, false>(a, sg, sm_count, s)
+                            : launch_gather_shape<T, LPR, SS, false, false>(a, sg, sm_count, s);
 }
 
 template <typename T>
@@ -322,7 +326,8 @@ hag_status fwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
     a.row_begin = 0;
     a.row_count = h->n;
     a.prim = x;
-    a.dst_scale = (reduce == HAG_MEAN) ? d.inv_degree : nullptr;
+    a.dst_scale = (reduce == HAG_MEAN) ? d.inv_degree : (reduce == HAG_GCN ? d.inv_degree1 : nullptr);
+    a.out_is_f32 = (reduce == HAG_GCN) ? 2 : 0;      // GCN: add the node's own row before normalising
     a.out = out;
     a.D = D;
     a.n_prim = std::numeric_limits<int32_t>::max();
@@ -362,7 +367,7 @@ hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
     const hag_device_arrays &d = h->d;
     hagk::GatherArgs a{};
     a.prim = g;
-    a.src_scale = (reduce == HAG_MEAN) ? d.inv_degree : nullptr;
+    a.src_scale = (reduce == HAG_MEAN) ? d.inv_degree : (reduce == HAG_GCN ? d.inv_degree1 : nullptr);
     a.D = D;
     a.n_prim = std::numeric_limits<int32_t>::max();
     float *partial = static_cast<float *>(ws) + (use_hag ? size_t(h->num_agg) * D : 0);
@@ -408,6 +413,7 @@ hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
     a.row_begin = 0;
     a.row_count = h->n;
     a.out = gx;
+    a.out_is_f32 = (reduce == HAG_GCN) ? 2 : 0;      // GCN: plus the node's own scaled gradient row
     if (h->n > 0) {
         if (rec) rec->begin(2, h->n, use_hag ? h->t_ptr[h->n] : h->e);
         if (launch_gather<T>(h, a, use_hag ? h->seg_t : h->seg_csr_t, partial, use_hag ? h->t_ptr[h->n] : h->e, n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
@@ -420,7 +426,7 @@ hag_status run(const hag *h, bool backward, bool use_hag, hag_reduce reduce, hag
                void *out, void *ws, void *stream) {
     hag_status st = check_call(h, dtype, D, in, out);
     if (st != HAG_OK) return st;
-    if (reduce != HAG_SUM && reduce != HAG_MEAN) return HAG_ERR_ARG;
+    if (reduce != HAG_SUM && reduce != HAG_MEAN && reduce != HAG_GCN) return HAG_ERR_ARG;
     const bool needs_ws = use_hag ? (h->num_agg > 0 || h->max_segs_hag > 0) : (h->max_segs_csr > 0);
     if (needs_ws) {
         if (!ws) return HAG_ERR_WORKSPACE;
@@ -491,15 +497,21 @@ extern "C" hag_status hag_to_device(hag_t *h, int device) {
     if (st == HAG_OK) st = upload_i32(&d.btail_ptr, h->btail_ptr.data(), h->btail_ptr.size());
     if (st == HAG_OK) st = upload_i32(&d.btail_idx, h->btail_idx.data(), h->btail_idx.size());
     if (st == HAG_OK) {
-        std::vector<float> inv(std::max<size_t>(n, 1), 1.0f);
-        for (size_t v = 0; v < n; ++v) inv[v] = h->in_degree[v] > 0 ? 1.0f / float(h->in_degree[v]) : 1.0f;
-        cudaError_t err = cudaMalloc(reinterpret_cast<void **>(&d.inv_degree), inv.size() * sizeof(float));
-        if (err != cudaSuccess) {
-            cudaGetLastError();
-            st = err == cudaErrorMemoryAllocation ? HAG_ERR_OOM_DEVICE : HAG_ERR_CUDA;
-        } else if (cudaMemcpy(d.inv_degree, inv.data(), inv.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) {
-            cudaGetLastError();
-            st = HAG_ERR_CUDA;
+        std::vector<float> inv(std::max<size_t>(n, 1), 1.0f), inv1(std::max<size_t>(n, 1), 1.0f);
+        for (size_t v = 0; v < n; ++v) {
+            inv[v] = h->in_degree[v] > 0 ? 1.0f / float(h->in_degree[v]) : 1.0f;
+            inv1[v] = 1.0f / float(h->in_degree[v] + 1);
+        }
+        for (auto pr : {std::make_pair(&d.inv_degree, &inv), std::make_pair(&d.inv_degree1, &inv1)}) {
+            if (st != HAG_OK) break;
+            cudaError_t err = cudaMalloc(reinterpret_cast<void **>(pr.first), pr.second->size() * sizeof(float));
+            if (err != cudaSuccess) {
+                cudaGetLastError();
+                st = err == cudaErrorMemoryAllocation ? HAG_ERR_OOM_DEVICE : HAG_ERR_CUDA;
+            } else if (cudaMemcpy(*pr.first, pr.second->data(), pr.second->size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) {
+                cudaGetLastError();
+                st = HAG_ERR_CUDA;
+            }
         }
     }
     for (seg_set *set : {&h->seg_res, &h->seg_t, &h->seg_csr, &h->seg_csr_t, &h->seg_ftail, &h->seg_btail})
@@ -661,7 +673,7 @@ extern "C" hag_status hag_aggregate_fwd_static(const hag_t *h, hag_reduce reduce
                                                const void *x, void *out, void *cuda_stream) {
     hag_status st = check_call(h, dtype, D, x, out);
     if (st != HAG_OK) return st;
-    if (reduce != HAG_SUM && reduce != HAG_MEAN) return HAG_ERR_ARG;
+    if (reduce != HAG_SUM && reduce != HAG_MEAN && reduce != HAG_GCN) return HAG_ERR_ARG;
     if (hag_workspace_bytes(h, D) > size_t(HAG_STATIC_SCRATCH_BYTES)) return HAG_ERR_TOO_LARGE;
     DeviceGuard guard(h->device);
     if (!guard.ok) { cudaGetLastError(); return HAG_ERR_CUDA; }

@@ -52,6 +52,7 @@ struct hag_device_arrays {
     int32_t *ftail_ptr = nullptr, *ftail_idx = nullptr;   // forward expansion of the deep levels
     int32_t *btail_ptr = nullptr, *btail_idx = nullptr;   // backward expansion
     float *inv_degree = nullptr;   // [n] 1/|N(v)| (1 for empty rows)
+    float *inv_degree1 = nullptr;  // [n] 1/(|N(v)| + 1): the GCN normalisation
     unsigned int *sched = nullptr; // ring of kSchedSlots (next row, finished warps) pairs, zero between launches
     // staging for the host-buffer entry point
     void *stage_in = nullptr;

@@ -44,7 +44,9 @@ struct GatherArgs {
     const float *src_scale;   // optional per-source factor for primary rows (backward of mean)
     const float *dst_scale;   // optional per-destination factor, indexed by absolute row id
     unsigned int *sched;      // persistent kernel only: [0] next row to hand out, [1] finished warps (both zero at launch)
-    void *out;                // T rows (out_is_f32 == 0) or fp32 rows (out_is_f32 == 1)
+    void *out;                // T rows or fp32 rows; out_is_f32: bit 0 = fp32 rows; bit 1 (host side: selects the SELF
+                              // instantiations) = add the row's own primary-table row (times its src_scale)
+                              // before scaling: GCN's (a_v + h_v) term
     int32_t out_row_offset;   // absolute row r is written to output row r - out_row_offset
     int32_t out_is_f32;
     int32_t D;
@@ -192,7 +194,7 @@ __device__ __forceinline__ RowHead load_head(const GatherArgs &a, int32_t row, i
 }
 
 // Gather-sum of one row [b, e) by one warp.  Returns with the result stored.
-template <typename T, int LPR, int UNROLL, bool SRC_SCALE>
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, bool SELF>
 __device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int32_t b, int32_t e, const RowHead &head, int lane) {
     constexpr int E = Chunk<T>::kElems;
     constexpr int G = 32 / LPR;                 // slices per warp
@@ -272,9 +274,17 @@ __device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int
 #pragma unroll
             for (int j = 0; j < E; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], off);
         if (live && slice == 0) {
+            if constexpr (SELF) {         // GCN: the row's own term, compiled only into the variants that need it
+                float self[E];
+                tab.load(row, self);
+                float sc = 1.0f;
+                if constexpr (SRC_SCALE) sc = __ldg(a.src_scale + row);
+#pragma unroll
+                for (int j = 0; j < E; ++j) acc[j] = fmaf(self[j], sc, acc[j]);
+            }
 #pragma unroll
             for (int j = 0; j < E; ++j) acc[j] *= dscale;
-            store_chunk<T>(a.out, a.out_is_f32, a.D, row - a.out_row_offset, chunk, acc);
+            store_chunk<T>(a.out, a.out_is_f32 & 1, a.D, row - a.out_row_offset, chunk, acc);
         }
     }
 }
@@ -282,7 +292,7 @@ __device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int
 // One segment of a long row: partial sum into a.partial, then, if this was the row's last open
 // segment, the fixed-order sum of all its partials into the output.  The completion count is an
 // integer atomic; the order of the floating-point additions never depends on who finishes when.
-template <typename T, int LPR, int UNROLL, bool SRC_SCALE>
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, bool SELF>
 __device__ __forceinline__ void gather_segment(const GatherArgs &a, const SegArgs &sa, int32_t seg_local, int lane) {
     constexpr int E = Chunk<T>::kElems;
     const int4 sg = __ldg(sa.segs + seg_local);
@@ -293,7 +303,7 @@ __device__ __forceinline__ void gather_segment(const GatherArgs &a, const SegArg
     part.out_row_offset = 0;
     RowHead head = load_head<SRC_SCALE>(a, row, b, e, lane);
     head.dst_scale = 1.0f;
-    gather_row<T, LPR, UNROLL, SRC_SCALE>(part, sa.seg_first + seg_local, b, e, head, lane);
+    gather_row<T, LPR, UNROLL, SRC_SCALE, false>(part, sa.seg_first + seg_local, b, e, head, lane);
     __threadfence();                                   // partial row visible before the count moves
     __syncwarp();
     const int2 sl = __ldg(sa.slots + slot);
@@ -317,23 +327,32 @@ __device__ __forceinline__ void gather_segment(const GatherArgs &a, const SegArg
                 acc[j] += q.x; acc[j + 1] += q.y; acc[j + 2] += q.z; acc[j + 3] += q.w;
             }
         }
+        if constexpr (SELF) {
+            const Tables<T> tab(a.prim, a.sec, a.n_prim, a.D, chunk);
+            float self[E];
+            tab.load(row, self);
+            float sc = 1.0f;
+            if constexpr (SRC_SCALE) sc = __ldg(a.src_scale + row);
+#pragma unroll
+            for (int j = 0; j < E; ++j) acc[j] = fmaf(self[j], sc, acc[j]);
+        }
 #pragma unroll
         for (int j = 0; j < E; ++j) acc[j] *= dscale;
-        store_chunk<T>(a.out, a.out_is_f32, a.D, row - a.out_row_offset, chunk, acc);
+        store_chunk<T>(a.out, a.out_is_f32 & 1, a.D, row - a.out_row_offset, chunk, acc);
     }
 }
 
 // Out of line on purpose: the row path of the kernels keeps its registers and code.
-template <typename T, int LPR, int UNROLL, bool SRC_SCALE>
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, bool SELF>
 __device__ __noinline__ void gather_segment_call(const GatherArgs &a, const SegArgs &sa, int32_t seg_local, int lane) {
-    gather_segment<T, LPR, UNROLL, SRC_SCALE>(a, sa, seg_local, lane);
+    gather_segment<T, LPR, UNROLL, SRC_SCALE, SELF>(a, sa, seg_local, lane);
 }
 
 // out[row] = (dst_scale[row]) * sum_{e in row} (src_scale[id_e]) * table[id_e]
 // One warp per work item, one item per launched warp.  HAS_SEGS: the launch has long rows; their
 // segments are the first items, and rows longer than a.long_row are left to them.  Without long
 // rows the kernel is compiled without any of that.
-template <typename T, int LPR, int UNROLL, bool SRC_SCALE, bool HAS_SEGS>
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, bool HAS_SEGS, bool SELF>
 __device__ __forceinline__ void gather_sum_body(const KernelArgs<HAS_SEGS> &k) {
     const GatherArgs &a = k.a;
     pdl_launch_dependents();
@@ -342,7 +361,7 @@ __device__ __forceinline__ void gather_sum_body(const KernelArgs<HAS_SEGS> &k) {
     if constexpr (HAS_SEGS) {
         if (r_local < k.sg.seg_count) {
             pdl_wait();
-            gather_segment_call<T, LPR, UNROLL, SRC_SCALE>(a, k.sg, r_local, lane);
+            gather_segment_call<T, LPR, UNROLL, SRC_SCALE, SELF>(a, k.sg, r_local, lane);
             return;
         }
         r_local -= k.sg.seg_count;
@@ -355,19 +374,19 @@ __device__ __forceinline__ void gather_sum_body(const KernelArgs<HAS_SEGS> &k) {
     }
     const RowHead head = load_head<SRC_SCALE>(a, row, b, e, lane);
     pdl_wait();        // structure arrays are static; features may come from the previous kernel
-    gather_row<T, LPR, UNROLL, SRC_SCALE>(a, row, b, e, head, lane);
+    gather_row<T, LPR, UNROLL, SRC_SCALE, SELF>(a, row, b, e, head, lane);
 }
 
 // Two entry points per form: the parameter block of the variant with long rows is declared
 // __grid_constant__ (its address is handed to the out-of-line segment function without a local
 // copy); the variant without long rows takes plain parameters, which costs it fewer registers.
-template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS>
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS, bool SELF>
 __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_kernel(const KernelArgs<false> k) {
-    gather_sum_body<T, LPR, UNROLL, SRC_SCALE, false>(k);
+    gather_sum_body<T, LPR, UNROLL, SRC_SCALE, false, SELF>(k);
 }
-template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS>
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS, bool SELF>
 __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_long_kernel(const __grid_constant__ KernelArgs<true> k) {
-    gather_sum_body<T, LPR, UNROLL, SRC_SCALE, true>(k);
+    gather_sum_body<T, LPR, UNROLL, SRC_SCALE, true, SELF>(k);
 }
 
 // The same, with resident warps that take items four at a time from a shared
@@ -377,7 +396,7 @@ __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_long_kernel(c
 // rows latency chain is paid once per warp instead of once per row.  The last warp
 // to finish zeroes the counters (a.sched[1] counts finished warps) for the slot's
 // next use.  No warp waits on another: there is no spin anywhere.
-template <typename T, int LPR, int UNROLL, bool SRC_SCALE, bool HAS_SEGS>
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, bool HAS_SEGS, bool SELF>
 __device__ __forceinline__ void gather_sum_persistent_body(const KernelArgs<HAS_SEGS> &k) {
     const GatherArgs &a = k.a;
     pdl_launch_dependents();
@@ -402,7 +421,7 @@ __device__ __forceinline__ void gather_sum_persistent_body(const KernelArgs<HAS_
         while (base < seg_items) {                          // each segment is long: no pipelining needed
 #pragma unroll 1
             for (int i = 0; i < CH; ++i)
-                if (base + i < k.sg.seg_count) gather_segment_call<T, LPR, UNROLL, SRC_SCALE>(a, k.sg, base + i, lane);
+                if (base + i < k.sg.seg_count) gather_segment_call<T, LPR, UNROLL, SRC_SCALE, SELF>(a, k.sg, base + i, lane);
             base = __shfl_sync(FULL, grab(), 0);
         }
         base -= seg_items;
@@ -430,7 +449,7 @@ __device__ __forceinline__ void gather_sum_persistent_body(const KernelArgs<HAS_
             }
             bool whole = true;
             if constexpr (HAS_SEGS) whole = e - b <= k.sg.long_row;
-            if (whole) gather_row<T, LPR, UNROLL, SRC_SCALE>(a, a.row_begin + base + i, b, e, cur, lane);
+            if (whole) gather_row<T, LPR, UNROLL, SRC_SCALE, SELF>(a, a.row_begin + base + i, b, e, cur, lane);
             if (i == 0 && nrows > 1) {
                 nbase = __shfl_sync(FULL, grabbed, 0) - seg_items;
                 rp_next = load_rp(nbase);
@@ -448,13 +467,13 @@ __device__ __forceinline__ void gather_sum_persistent_body(const KernelArgs<HAS_
     }
 }
 
-template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS>
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS, bool SELF>
 __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_persistent_kernel(const KernelArgs<false> k) {
-    gather_sum_persistent_body<T, LPR, UNROLL, SRC_SCALE, false>(k);
+    gather_sum_persistent_body<T, LPR, UNROLL, SRC_SCALE, false, SELF>(k);
 }
-template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS>
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS, bool SELF>
 __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_persistent_long_kernel(const __grid_constant__ KernelArgs<true> k) {
-    gather_sum_persistent_body<T, LPR, UNROLL, SRC_SCALE, true>(k);
+    gather_sum_persistent_body<T, LPR, UNROLL, SRC_SCALE, true, SELF>(k);
 }
 
 // Level kernel of Algorithm 2 (lines 5-6): every aggregation node of one level is

@@ -77,7 +77,7 @@ def _case(name):
 
 
 @pytest.mark.parametrize("name", list(CASES))
-@pytest.mark.parametrize("reduce", ["sum", "mean"])
+@pytest.mark.parametrize("reduce", ["sum", "mean", "gcn"])
 def test_workload_shapes_match_oracle(name, reduce):
     w, h = _case(name)
     g = w.graph
@@ -207,7 +207,7 @@ def test_long_rows_are_split_and_still_exact(dtype, d):
     assert h.csr_workspace_bytes(d) > 0 and h.workspace_bytes(d) > 0
     x = synth.features(11, n, d, "normal", dtype)
     gr = synth.upstream_grad(11, n, d, "normal", dtype)
-    for reduce in ("sum", "mean"):
+    for reduce in ("sum", "mean", "gcn"):
         _check_all_paths(g, h, x, gr, reduce, dtype)
     if dtype == "f32":
         xi = synth.features(12, n, d, "int")

@@ -277,6 +277,26 @@ def test_direct_aggregation_is_spmm(undirected):
     np.testing.assert_allclose(gx, dense.T @ gr, rtol=1e-13, atol=1e-13)
 
 
+def test_gcn_mode_is_the_normalised_sum_with_the_own_row():
+    # Table 1, GCN: the argument of Update is (a_v + h_v) / (|N(v)| + 1) = D^-1 (A + I) x with D = deg + 1
+    g = synth.random_digraph(23, 50, 0.2, undirected=False, self_loops=False)
+    x = synth.features(2, g.n, 4, "normal").astype(np.float64)
+    gr = synth.upstream_grad(2, g.n, 4, "normal").astype(np.float64)
+    a_mat = sp.csr_matrix((np.ones(g.e), g.col_idx, g.row_ptr), shape=(g.n, g.n)) + sp.identity(g.n)
+    inv = 1.0 / (np.diff(g.row_ptr) + 1.0)
+    out, t = O.direct_forward(g.row_ptr, g.col_idx, x, "gcn")
+    np.testing.assert_allclose(out, (a_mat @ x) * inv[:, None], rtol=1e-13, atol=1e-13)
+    np.testing.assert_allclose(t, (a_mat @ np.abs(x)) * inv[:, None], rtol=1e-13, atol=1e-13)
+    gx, _ = O.direct_backward(g.row_ptr, g.col_idx, gr, "gcn")
+    np.testing.assert_allclose(gx, a_mat.T @ (gr * inv[:, None]), rtol=1e-13, atol=1e-13)
+    rows = np.asarray([3, 0, 49, 17])
+    part, _ = O.direct_backward(g.row_ptr, g.col_idx, gr, "gcn", rows=rows)
+    assert np.array_equal(part, gx[rows])
+    lhs = float((out * gr).sum())
+    rhs = float((x * gx).sum())
+    assert abs(lhs - rhs) < 1e-10
+
+
 def test_direct_aggregation_on_a_star_is_not_its_transpose():
     # node 0 aggregates 1..4; nobody else aggregates anything
     g = _graph_from_rows([[1, 2, 3, 4], [], [], [], []])
