@@ -230,8 +230,10 @@ hag_status hag_aggregate_host(hag_t *h, int backward, int use_hag, hag_reduce re
  * with cudaEventCreate and kept by the handle).  hag_profile_read synchronises
  * on the events of the LAST call and returns how many launches it made; for the
  * first `max` of them it fills ms[i] (device time), kind[i] (0 = level pair-sum,
- * 1 = gather over the aggregation nodes of one level (backward), 2 = gather over
- * the graph nodes), rows[i] (rows written) and edges[i] (source rows read).
+ * 1 = gather over aggregation nodes: one level of the backward pass, or the
+ * expanded deep levels of either pass, 2 = gather over the graph nodes), rows[i]
+ * (rows written) and edges[i] (source rows read).  A gather over a table with
+ * split long rows is still one launch: segments and rows share it.
  * Arrays may be NULL.  Returns -1 on error. */
 hag_status hag_profile_enable(hag_t *h, int enable);
 int32_t hag_profile_read(hag_t *h, int32_t max, float *ms, int32_t *kind, int64_t *rows, int64_t *edges);

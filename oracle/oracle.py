@@ -22,7 +22,7 @@ What it computes, and where the paper (arxiv 1906.03707) defines it:
   the cost function of Section 4.1 in both forms, f = |E| - |E-hat| + |V_A| of
   the Theorem 4 proof, and a from-the-definition replay of a merge trace.
 
-Readings of points the paper leaves open (each also listed in the design notes):
+Readings of points the paper leaves open:
 redundancy counts graph nodes u in V only (the rewrite loop of Algorithm 3 runs
 over V); pairs are unordered over V and V_A; ties go to the lexicographically
 smallest (v1, v2), v1 < v2, aggregation nodes numbered N, N+1, ... as created;
