@@ -220,6 +220,40 @@ def test_long_rows_are_split_and_still_exact(dtype, d):
             assert np.array_equal(_host(h.csr_bwd(_dev(xi, "f32"), "sum")), b)
 
 
+@pytest.mark.parametrize("seed", range(24))
+def test_random_graphs_every_path_exact_on_integers(seed):
+    """Small random graphs of many shapes: integer features make every fp32 partial sum exact, so sum results of
+    all four paths must equal the oracle bit for bit whatever the structure (empty rows, hubs, deep or no
+    hierarchy, any capacity, odd widths)."""
+    rng = np.random.default_rng(100 + seed)
+    n = int(rng.integers(40, 2500))
+    kind = seed % 4
+    if kind == 0:
+        g = synth.random_digraph(200 + seed, min(n, 400), float(rng.uniform(0.02, 0.5)), bool(seed % 2), bool(seed % 3 == 0))
+    elif kind == 1:
+        g = synth.clique_union_graph(200 + seed, n, max(5, n // 8), 2, max(4, n // 10), 2.0, self_loops=bool(seed % 2))
+    elif kind == 2:
+        g = synth.config2_graph(seed=200 + seed, n=max(n, 300), n_comm=max(3, n // 100), d_lo=3, d_hi=max(8, n // 4))
+    else:
+        g = synth.config4_graph(seed=200 + seed, n_graphs=max(2, n // 60), graph_size=int(rng.integers(8, 80)),
+                                p=float(rng.uniform(0.2, 0.9)))
+    cap = int(g.n * float(rng.choice([0.0, 0.1, 0.25, 1.0, 4.0])))
+    min_r = int(rng.choice([2, 2, 3, 5]))
+    h = hb.Hag.build(g.row_ptr, g.col_idx, cap, min_redundancy=min_r).to_device(0)
+    d = int(rng.choice([4, 12, 32, 68, 128]))
+    x = synth.features(300 + seed, g.n, d, "int")
+    a, _ = O.direct_forward(g.row_ptr, g.col_idx, x.astype(np.float64), "sum")
+    b, _ = O.direct_backward(g.row_ptr, g.col_idx, x.astype(np.float64), "sum")
+    xd = _dev(x, "f32")
+    assert np.array_equal(_host(h.aggregate_fwd(xd, "sum")), a)
+    assert np.array_equal(_host(h.csr_fwd(xd, "sum")), a)
+    assert np.array_equal(_host(h.aggregate_bwd(xd, "sum")), b)
+    assert np.array_equal(_host(h.csr_bwd(xd, "sum")), b)
+    xf = synth.features(400 + seed, g.n, d, "normal")
+    gf = synth.upstream_grad(400 + seed, g.n, d, "normal")
+    _check_all_paths(g, h, xf, gf, ["mean", "gcn"][seed % 2], "f32")
+
+
 def test_empty_graph_launches_nothing():
     h = hb.Hag.build(np.zeros(1, np.int64), np.zeros(0, np.int32), 4).to_device(0)
     x = torch.empty((0, 64), device="cuda")
