@@ -95,8 +95,8 @@ cudaError_t launch_pdl(void (*kernel)(Args), unsigned grid, const Args &args, cu
 //   fp32, large launch, 512-byte rows   : resident warps, 8 loads, 32 warps/SM
 //   fp32, large launch, narrower rows   : resident warps, 4 loads, 32 warps/SM
 //   fp32, small launch                  : one row per warp, 4 loads, 40 warps/SM (32 with per-source factors)
-// (large = at least 131072 rows or 4 Mi source entries)
 //   bf16                                : one row per warp, 2 loads, 48 warps/SM
+// (large = at least 131072 rows or 4 Mi source entries)
 // Resident warps hide the pointer -> ids latency of the next row behind the
 // current one, which pays once there are many rows per warp; with few rows the
 // hardware's own block scheduling balances better.
