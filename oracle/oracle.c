@@ -454,3 +454,179 @@ done:
     free(out); free(out_store); free(delta); free(touched); free(users); free(hp.e); pm_free(&map);
     return rc < 0 ? rc : num_agg;
 }
+
+/* ------------------------------------------------------------------------- */
+/* O3c: Algorithm 3 (set Aggregate) without a count per pair, for graphs whose
+ * pair map does not fit in memory.  Exact, by this argument:
+ *   - a merge of (v1, v2) only removes v1 and v2 from the rows that held both and
+ *     adds the new node w there, so the redundancy of every existing pair can only
+ *     fall, and a new pair (w, y) is held by a subset of the merged pair's rows;
+ *   - hence bound[x] >= max over b of Redundancy(x, b) stays valid if it is set
+ *     once to a true value (or to |out(x)| at the start, or to the merged pair's
+ *     redundancy for a new node) and never raised;
+ *   - the node x with the largest bound (ties: smallest id) is recounted from the
+ *     definition; if its true maximum equals its bound, no pair anywhere has a
+ *     larger redundancy, x is the smaller member of the lexicographically smallest
+ *     pair attaining it (a smaller member would carry the same bound and a smaller
+ *     id), and its partner is the smallest id attaining the count.  Otherwise the
+ *     bound is lowered to the true maximum and the search goes on.
+ * Same outputs as o3b_greedy.                                                 */
+typedef struct { int32_t key, id; } lent;
+static int l_before(const lent *x, const lent *y) {
+    if (x->key != y->key) return x->key > y->key;
+    return x->id < y->id;
+}
+typedef struct { lent *e; int64_t n, cap; } lheap;
+static int l_push(lheap *h, lent v) {
+    if (h->n == h->cap) {
+        int64_t nc = h->cap ? h->cap * 2 : 1024;
+        lent *ne = (lent *)realloc(h->e, sizeof(lent) * (size_t)nc);
+        if (!ne) return -1;
+        h->e = ne; h->cap = nc;
+    }
+    int64_t i = h->n++;
+    while (i > 0) {
+        int64_t p = (i - 1) / 2;
+        if (!l_before(&v, &h->e[p])) break;
+        h->e[i] = h->e[p]; i = p;
+    }
+    h->e[i] = v;
+    return 0;
+}
+static lent l_pop(lheap *h) {
+    lent top = h->e[0];
+    lent last = h->e[--h->n];
+    int64_t i = 0;
+    for (;;) {
+        int64_t l = 2 * i + 1, r = l + 1, c;
+        if (l >= h->n) break;
+        c = (r < h->n && l_before(&h->e[r], &h->e[l])) ? r : l;
+        if (!l_before(&h->e[c], &last)) break;
+        h->e[i] = h->e[c]; i = c;
+    }
+    if (h->n > 0) h->e[i] = last;
+    return top;
+}
+
+int64_t o3c_greedy(int64_t n, const int64_t *row_ptr, const int32_t *col, int64_t capacity, int32_t min_redundancy,
+                   int32_t *trace_v1, int32_t *trace_v2, int32_t *trace_r,
+                   int32_t *cur_len, int32_t *cur_idx, int32_t *final_max_redundancy)
+{
+    int64_t E = row_ptr[n];
+    int64_t n_ids = n + capacity;
+    int64_t num_agg = 0, rc = 0;
+    lheap hp = {0, 0, 0};
+    ilist *out = (ilist *)calloc((size_t)(n_ids > 0 ? n_ids : 1), sizeof(ilist));
+    int32_t *out_store = (int32_t *)malloc(sizeof(int32_t) * (size_t)(E > 0 ? E : 1));
+    int32_t *bound = (int32_t *)calloc((size_t)(n_ids > 0 ? n_ids : 1), sizeof(int32_t));
+    int32_t *count = (int32_t *)calloc((size_t)(n_ids > 0 ? n_ids : 1), sizeof(int32_t));
+    int32_t *touched = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n_ids > 0 ? n_ids : 1));
+    int32_t *users = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n > 0 ? n : 1));
+    *final_max_redundancy = 0;
+    if (!out || !out_store || !bound || !count || !touched || !users) return -1;
+
+    memcpy(cur_idx, col, sizeof(int32_t) * (size_t)E);
+    for (int64_t u = 0; u < n; ++u) cur_len[u] = (int32_t)(row_ptr[u + 1] - row_ptr[u]);
+    {
+        int64_t *fill = (int64_t *)calloc((size_t)n + 1, sizeof(int64_t));
+        if (!fill) return -1;
+        for (int64_t e = 0; e < E; ++e) fill[col[e] + 1]++;
+        for (int64_t s = 0; s < n; ++s) fill[s + 1] += fill[s];
+        for (int64_t s = 0; s < n; ++s) { out[s].v = out_store + fill[s]; out[s].len = 0; }
+        for (int64_t u = 0; u < n; ++u)
+            for (int64_t e = row_ptr[u]; e < row_ptr[u + 1]; ++e) { ilist *l = &out[col[e]]; l->v[l->len++] = (int32_t)u; }
+        free(fill);
+    }
+    /* a pair cannot be held by more rows than hold either member */
+    for (int64_t s = 0; s < n; ++s) {
+        bound[s] = out[s].len;
+        if (bound[s] >= 2) { lent v = { bound[s], (int32_t)s }; if (l_push(&hp, v)) { rc = -1; goto done; } }
+    }
+    for (;;) {
+        /* the node with the largest bound whose recount confirms the bound */
+        int32_t x = -1, best = 0, arg = -1;
+        while (hp.n > 0) {
+            lent top = l_pop(&hp);
+            if (top.key != bound[top.id]) continue;             /* an older, higher bound of this node */
+            int32_t cand = top.id, nt = 0;
+            for (int32_t k = 0; k < out[cand].len; ++k) {       /* Redundancy(cand, y) for every y, from the definition */
+                int32_t u = out[cand].v[k];
+                const int32_t *row = cur_idx + row_ptr[u];
+                for (int32_t i = 0; i < cur_len[u]; ++i) {
+                    int32_t y = row[i];
+                    if (y == cand) continue;
+                    if (count[y]++ == 0) touched[nt++] = y;
+                }
+            }
+            int32_t b = 0, a = -1;
+            for (int32_t t = 0; t < nt; ++t) {
+                int32_t y = touched[t], c = count[y];
+                count[y] = 0;
+                if (c > b || (c == b && y < a)) { b = c; a = y; }
+            }
+            if (b < top.key) {                                   /* stale: tighten and look again */
+                bound[cand] = b;
+                if (b >= 2) { lent v = { b, cand }; if (l_push(&hp, v)) { rc = -1; goto done; } }
+                continue;
+            }
+            x = cand; best = b; arg = a;
+            break;
+        }
+        if (x < 0) {                                             /* no pair is shared by two rows any more */
+            int any = 0;
+            for (int64_t u = 0; u < n && !any; ++u) any = cur_len[u] >= 2;
+            *final_max_redundancy = any ? 1 : 0;
+            break;
+        }
+        if (best < min_redundancy || num_agg >= capacity) {      /* "if Redundancy > 1" when min_redundancy is 2 */
+            *final_max_redundancy = best;
+            break;
+        }
+        if (arg <= x) { rc = -3; goto done; }                    /* would contradict the argument above */
+        int32_t v1 = x, v2 = arg, w = (int32_t)(n + num_agg);
+        int32_t nu = 0;
+        {
+            ilist *A = &out[v1], *B = &out[v2];
+            int32_t i = 0, j = 0;
+            while (i < A->len && j < B->len) {
+                if (A->v[i] < B->v[j]) ++i; else if (A->v[i] > B->v[j]) ++j;
+                else { users[nu++] = A->v[i]; ++i; ++j; }
+            }
+        }
+        if (nu != best) { rc = -2; goto done; }
+        trace_v1[num_agg] = v1; trace_v2[num_agg] = v2; trace_r[num_agg] = nu;
+        for (int32_t k = 0; k < nu; ++k) {                       /* E-hat <- E-hat - (v1,u) - (v2,u) + (w,u) */
+            int32_t u = users[k];
+            int32_t *row = cur_idx + row_ptr[u];
+            int32_t len = cur_len[u], o = 0;
+            for (int32_t i = 0; i < len; ++i) if (row[i] != v1 && row[i] != v2) row[o++] = row[i];
+            row[o++] = w;
+            cur_len[u] = o;
+        }
+        {
+            int32_t ends[2] = { v1, v2 };
+            for (int q = 0; q < 2; ++q) {
+                ilist *L = &out[ends[q]];
+                int32_t o = 0, k = 0;
+                for (int32_t i = 0; i < L->len; ++i) {
+                    while (k < nu && users[k] < L->v[i]) ++k;
+                    if (k < nu && users[k] == L->v[i]) continue;
+                    L->v[o++] = L->v[i];
+                }
+                L->len = o;
+            }
+            out[w].v = (int32_t *)malloc(sizeof(int32_t) * (size_t)nu);
+            if (!out[w].v) { rc = -1; goto done; }
+            memcpy(out[w].v, users, sizeof(int32_t) * (size_t)nu);
+            out[w].len = nu;
+        }
+        bound[w] = nu;                                           /* a pair with w is held by a subset of the nu rewritten rows */
+        { lent v = { nu, w }; if (nu >= 2 && l_push(&hp, v)) { rc = -1; goto done; } }
+        { lent v = { bound[v1], v1 }; if (l_push(&hp, v)) { rc = -1; goto done; } }   /* v1 left the heap when it was popped */
+        ++num_agg;
+    }
+done:
+    for (int64_t s = n; s < n_ids; ++s) free(out[s].v);
+    free(out); free(out_store); free(bound); free(count); free(touched); free(users); free(hp.e);
+    return rc < 0 ? rc : num_agg;
+}

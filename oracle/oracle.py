@@ -14,6 +14,8 @@ What it computes, and where the paper (arxiv 1906.03707) defines it:
   every pair from scratch in every iteration (tiny graphs only).
 * ``greedy_pairmap`` -- Algorithm 3 with the pair-count heap of the complexity
   appendix (plain C).
+* ``greedy_lazy`` -- Algorithm 3 with per-node bounds confirmed by recounts (plain
+  C, memory O(|E|)), for the shapes whose pair map does not fit in memory.
 * ``canonical_hag`` -- the run-time layout: levels (longest path from a source),
   level-sorted renumbering, input pairs, residual CSR, transposed HAG.
 * ``hag_forward`` / ``hag_backward`` -- Algorithm 2 and its adjoint over that
@@ -75,6 +77,8 @@ def _c():
         lib.o_max_pair_recount.restype = i64
         lib.o3b_greedy.argtypes = [i64, p, p, i64, i32, p, p, p, p, p, p]
         lib.o3b_greedy.restype = i64
+        lib.o3c_greedy.argtypes = [i64, p, p, i64, i32, p, p, p, p, p, p]
+        lib.o3c_greedy.restype = i64
         _lib = lib
     return _lib
 
@@ -187,8 +191,19 @@ def greedy_bruteforce(row_ptr, col_idx, capacity, min_redundancy=2) -> SearchRes
     return SearchResult(n, tr, [np.asarray(sorted(r), dtype=np.int32) for r in rows], int(last_max))
 
 
+def greedy_lazy(row_ptr, col_idx, capacity, min_redundancy=2) -> SearchResult:
+    """Algorithm 3 without a count per pair (C, memory O(|E|)): per-node upper bounds on the best
+    redundancy, confirmed by a recount from the definition before every merge.  For graphs whose
+    pair map does not fit in memory."""
+    return _greedy_c("o3c_greedy", row_ptr, col_idx, capacity, min_redundancy)
+
+
 def greedy_pairmap(row_ptr, col_idx, capacity, min_redundancy=2) -> SearchResult:
     """Algorithm 3 with the pair-count map and heap of the complexity appendix (C)."""
+    return _greedy_c("o3b_greedy", row_ptr, col_idx, capacity, min_redundancy)
+
+
+def _greedy_c(fn, row_ptr, col_idx, capacity, min_redundancy) -> SearchResult:
     rp, ci = _csr(row_ptr, col_idx)
     n = rp.shape[0] - 1
     cap = int(capacity)
@@ -198,9 +213,9 @@ def greedy_pairmap(row_ptr, col_idx, capacity, min_redundancy=2) -> SearchResult
     cur_len = np.zeros(max(n, 1), dtype=np.int32)
     cur_idx = np.zeros(max(ci.shape[0], 1), dtype=np.int32)
     fin = np.zeros(1, dtype=np.int32)
-    k = _c().o3b_greedy(n, _ptr(rp), _ptr(ci), cap, int(min_redundancy), _ptr(t1), _ptr(t2), _ptr(tr), _ptr(cur_len), _ptr(cur_idx), _ptr(fin))
+    k = getattr(_c(), fn)(n, _ptr(rp), _ptr(ci), cap, int(min_redundancy), _ptr(t1), _ptr(t2), _ptr(tr), _ptr(cur_len), _ptr(cur_idx), _ptr(fin))
     if k < 0:
-        raise MemoryError(f"o3b_greedy failed with code {k}")
+        raise MemoryError(f"{fn} failed with code {k}")
     trace = np.stack([t1[:k], t2[:k], tr[:k]], axis=1).astype(np.int32).reshape(-1, 3)
     rows = [cur_idx[rp[u]:rp[u] + cur_len[u]].copy() for u in range(n)]
     return SearchResult(n, trace, rows, int(fin[0]))

@@ -20,7 +20,7 @@ def _graph_from_rows(rows):
     return synth.csr_from_rows(rows)
 
 
-SEARCHES = [O.greedy_bruteforce, O.greedy_pairmap]
+SEARCHES = [O.greedy_bruteforce, O.greedy_pairmap, O.greedy_lazy]
 
 
 # --------------------------------------------------------------------------- #
@@ -164,7 +164,10 @@ def test_pairmap_equals_bruteforce_on_tiny_graphs(seed):
     for cap in (n // 4, 3 * n):
         a = O.greedy_bruteforce(g.row_ptr, g.col_idx, cap)
         b = O.greedy_pairmap(g.row_ptr, g.col_idx, cap)
-        assert a.trace.tolist() == b.trace.tolist()
+        c = O.greedy_lazy(g.row_ptr, g.col_idx, cap)
+        assert a.trace.tolist() == b.trace.tolist() == c.trace.tolist()
+        assert [r.tolist() for r in a.rows] == [r.tolist() for r in c.rows]
+        assert a.final_max_redundancy == c.final_max_redundancy
         assert [r.tolist() for r in a.rows] == [r.tolist() for r in b.rows]
         assert a.final_max_redundancy == b.final_max_redundancy
         # replay from the definition, with an arg-max recount at a few steps
@@ -220,6 +223,8 @@ def _invariants(g, res, h):
 def test_invariants_and_values_on_workload_shapes(maker):
     g = maker()
     res = O.greedy_pairmap(g.row_ptr, g.col_idx, g.n // 4)
+    lazy = O.greedy_lazy(g.row_ptr, g.col_idx, g.n // 4)
+    assert lazy.trace.tolist() == res.trace.tolist() and lazy.final_max_redundancy == res.final_max_redundancy
     h = O.canonical_hag(g.row_ptr, res)
     c = _invariants(g, res, h)
     assert c["num_agg"] > 0
