@@ -15,6 +15,8 @@
  *   o4_hag_backward     the adjoint of Algorithm 2 over the transposed HAG
  *   o3b_greedy          Algorithm 3, set-Aggregate branch, with the pair-count
  *                       heap the complexity appendix sketches
+ *   o3c_greedy          the same algorithm without a count per pair (memory O(|E|)):
+ *                       per-node upper bounds confirmed by recounts from the definition
  *   o_count_pair / o_max_pair_recount   the Redundancy function of Algorithm 3
  *                       evaluated from its definition
  *

@@ -31,9 +31,9 @@ smallest (v1, v2), v1 < v2, aggregation nodes numbered N, N+1, ... as created;
 the loop stops when the best redundancy is <= 1 or |V_A| = capacity; an empty
 neighbourhood yields a zero row; mean divides by the in-degree in the input graph.
 
-Parity pins: see tests/test_oracle_pins.py.  The search at the two largest
-workload shapes is pinned only by replay and sampled recounts ("parity unpinned"
-beyond that, as no worked example of that size exists).
+Parity pins: see tests/test_oracle_pins.py.  The three searches must agree
+merge for merge; the memory-light one is what reaches the two largest workload
+shapes, and it is pinned against brute force and against the pair-count heap.
 """
 from __future__ import annotations
 
