@@ -149,6 +149,10 @@ cudaError_t launch_gather_shape(const hagk::GatherArgs &ga, const hagk::SegArgs 
         case 2: return launch_pdl(plain_kernel<T, LPR, 4, SS, 12, SEGS, SELF>(), grid, a, s);
         case 4: return launch_pdl(plain_kernel<T, LPR, 2, SS, 16, SEGS, SELF>(), grid, a, s);
         case 5: return launch_pdl(plain_kernel<T, LPR, 4, SS, 10, SEGS, SELF>(), grid, a, s);
+        case 6: return launch_pdl(plain_kernel<T, LPR, 2, SS, 10, SEGS, SELF>(), grid, a, s);
+        case 7: return launch_pdl(plain_kernel<T, LPR, 4, SS, 8, SEGS, SELF>(), grid, a, s);
+        case 8: return launch_pdl(plain_kernel<T, LPR, 2, SS, 8, SEGS, SELF>(), grid, a, s);
+        case 3: return launch_pdl(plain_kernel<T, LPR, 2, SS, 12, SEGS, SELF>(), grid, a, s);
         case 9: return launch_persistent(resident_kernel<T, LPR, 4, SS, 10, SEGS, SELF>(), a, items, sm_count, s);
         case 10: return launch_persistent(resident_kernel<T, LPR, 4, SS, 8, SEGS, SELF>(), a, items, sm_count, s);
         case 11: return launch_persistent(resident_kernel<T, LPR, 8, SS, 8, SEGS, SELF>(), a, items, sm_count, s);

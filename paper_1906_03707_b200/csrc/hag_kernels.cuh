@@ -102,8 +102,9 @@ __device__ __forceinline__ uint4 f32x8_to_bf16(const float *f) {
 
 // a[0..E) += b[0..E) as packed fp32x2 adds (one instruction per two sums on sm_100; each half is an
 // ordinary round-to-nearest add, so the bits are those of E scalar adds).
-// Used for fp32 storage (4 sums per chunk); with 8 sums per chunk (bf16 storage) the register pairs
-// it needs cost more in spills than the halved add count saves, so that path adds scalars.
+// Used for fp32 storage (4 sums per chunk); with 8 sums per chunk (bf16 storage) it was measured at every
+// register budget from 40 to 64 and never beat scalar adds (spills at 40, too few warps above), so that
+// path adds scalars.
 template <int E>
 __device__ __forceinline__ void add_rows(float *a, const float *b) {
     if constexpr (E == 4) {
