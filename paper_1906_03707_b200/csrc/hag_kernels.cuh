@@ -240,14 +240,24 @@ __device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int
                 if (k * G < cnt) {
                     float v[U][E];
 #pragma unroll
-                    for (int u = 0; u < U; ++u) {
-                        const int src_lane = (k + u) * G + slice;
-                        const int32_t id = __shfl_sync(0xffffffffu, cur, src_lane);
-                        if (id >= 0 && live) {
-                            tab.load(id, v[u]);
-                        } else {
+                    // Measured on B200: the unchecked path is 4-18 % faster for fp32 storage without per-source
+                    // factors; with factors or bf16 storage the doubled loop body spills and loses 5-13 %.
+                    constexpr bool kFastGroups = (E == 4) && !SRC_SCALE;
+                    if (kFastGroups && (k + U) * G <= cnt) {
+                        // every entry of this group exists: no checks, no zero fill (lanes beyond the row
+                        // width read chunk 0 of a valid row and are never stored)
 #pragma unroll
-                            for (int j = 0; j < E; ++j) v[u][j] = 0.0f;
+                        for (int u = 0; u < U; ++u) tab.load(__shfl_sync(0xffffffffu, cur, (k + u) * G + slice), v[u]);
+                    } else {
+#pragma unroll
+                        for (int u = 0; u < U; ++u) {
+                            const int32_t id = __shfl_sync(0xffffffffu, cur, (k + u) * G + slice);
+                            if (id >= 0 && (kFastGroups || live)) {
+                                tab.load(id, v[u]);
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < E; ++j) v[u][j] = 0.0f;
+                            }
                         }
                     }
                     if constexpr (SRC_SCALE) {
