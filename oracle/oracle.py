@@ -24,6 +24,11 @@ What it computes, and where the paper (arxiv 1906.03707) defines it:
   the cost function of Section 4.1 in both forms, f = |E| - |E-hat| + |V_A| of
   the Theorem 4 proof, and a from-the-definition replay of a merge trace.
 
+* ``graph_pool_forward`` / ``graph_pool_backward`` -- the mean-pooling layer that the
+  experimental setup (Section 5.1) puts after the GNN layers for graph
+  classification: one output row per graph of a batch, the mean (or sum) of the
+  rows of its nodes, and the gradient of that; fp64, one slice sum per graph.
+
 Readings of points the paper leaves open:
 redundancy counts graph nodes u in V only (the rewrite loop of Algorithm 3 runs
 over V); pairs are unordered over V and V_A; ties go to the lexicographically
@@ -136,6 +141,42 @@ def direct_backward(row_ptr, col_idx, g, reduce="sum", rows=None):
     ab = np.empty((m, d), dtype=np.float64)
     _c().o2_direct_backward(n, _ptr(rp), _ptr(ci), d, _ptr(g), _mode(reduce), _ptr(slot), m, _ptr(out), _ptr(ab))
     return out, ab
+
+
+def graph_pool_forward(seg_ptr, x, reduce="mean"):
+    """Graph-level read-out of Section 5.1: graph i owns the node rows
+    seg_ptr[i] .. seg_ptr[i+1]-1; out_i = sum of those rows (mean: divided by their
+    number; a graph without nodes gives a zero row).  Returns (out, T), T = the same
+    with |x| (the scale of the comparison tolerance)."""
+    sp = np.ascontiguousarray(seg_ptr, dtype=np.int64)
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    m = sp.shape[0] - 1
+    out = np.zeros((m, x.shape[1]), dtype=np.float64)
+    ab = np.zeros((m, x.shape[1]), dtype=np.float64)
+    for i in range(m):
+        b, e = int(sp[i]), int(sp[i + 1])
+        if e <= b:
+            continue
+        w = 1.0 / (e - b) if reduce == "mean" else 1.0
+        out[i] = x[b:e].sum(axis=0) * w
+        ab[i] = np.abs(x[b:e]).sum(axis=0) * w
+    return out, ab
+
+
+def graph_pool_backward(seg_ptr, g, n_rows, reduce="mean"):
+    """Gradient of graph_pool_forward: every node row of graph i receives g_i
+    (mean: divided by the number of nodes of the graph); rows outside every graph
+    receive zero.  Returns (gx, T) with T = |gx|."""
+    sp = np.ascontiguousarray(seg_ptr, dtype=np.int64)
+    g = np.ascontiguousarray(g, dtype=np.float64)
+    gx = np.zeros((int(n_rows), g.shape[1]), dtype=np.float64)
+    for i in range(sp.shape[0] - 1):
+        b, e = int(sp[i]), int(sp[i + 1])
+        if e <= b:
+            continue
+        w = 1.0 / (e - b) if reduce == "mean" else 1.0
+        gx[b:e] = g[i] * w
+    return gx, np.abs(gx)
 
 
 # --------------------------------------------------------------------------- #

@@ -385,3 +385,76 @@ def test_expanded_deep_levels_are_covers_and_transitive_users():
         assert np.array_equal(gr[ids].sum(0), ghat[j0 + i])
     # a small graph never pays for a launch per level: everything deeper than the cut is expanded
     assert t["fwd_cut"] < h.num_levels and t["bwd_cut"] < h.num_levels
+
+
+# --------------------------------------------------------------------------- #
+# Graph read-out (mean-pooling layer of Section 5.1)
+# --------------------------------------------------------------------------- #
+def _ragged_segments(seed, m, max_len, with_empty=True):
+    rng = np.random.default_rng(seed)
+    lens = rng.integers(1, max_len + 1, size=m)
+    if with_empty:
+        lens[rng.integers(0, m, size=max(1, m // 7))] = 0
+    return np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+
+
+def test_graph_pool_closed_forms():
+    # x[v, j] = v + 1000 j: the sum over rows b..e-1 is an arithmetic series
+    sp_ = np.array([0, 3, 3, 10, 11, 40], dtype=np.int64)
+    n, d = 40, 5
+    x = np.arange(n, dtype=np.float64)[:, None] + 1000.0 * np.arange(d)[None, :]
+    s, _ = O.graph_pool_forward(sp_, x, "sum")
+    mean, t = O.graph_pool_forward(sp_, x, "mean")
+    for i in range(5):
+        b, e = int(sp_[i]), int(sp_[i + 1])
+        k = e - b
+        series = (b + e - 1) * k / 2.0
+        assert np.array_equal(s[i], series + 1000.0 * np.arange(d) * k)
+        if k:
+            assert np.allclose(mean[i], (b + e - 1) / 2.0 + 1000.0 * np.arange(d), rtol=1e-15)
+            assert np.allclose(t[i], mean[i], rtol=1e-15)          # all terms are positive
+        else:
+            assert not mean[i].any() and not s[i].any()            # a graph without nodes: zero row
+
+
+def test_graph_pool_mean_of_a_constant_is_the_constant():
+    sp_ = _ragged_segments(3, 50, 30, with_empty=False)
+    x = np.full((int(sp_[-1]), 7), -2.75)
+    out, t = O.graph_pool_forward(sp_, x, "mean")
+    assert np.allclose(out, -2.75, rtol=1e-15) and np.allclose(t, 2.75, rtol=1e-15)
+
+
+def test_graph_pool_matches_reduceat_and_a_dense_pooling_matrix():
+    sp_ = _ragged_segments(4, 60, 25, with_empty=False)
+    n = int(sp_[-1])
+    x = np.random.default_rng(5).standard_normal((n, 9))
+    s, _ = O.graph_pool_forward(sp_, x, "sum")
+    assert np.allclose(s, np.add.reduceat(x, sp_[:-1], axis=0), rtol=1e-13, atol=1e-13)
+    # P[i, v] = 1/|G_i| for v in G_i: forward is P x, backward is P^T g
+    sp2 = _ragged_segments(6, 40, 12)
+    n2 = int(sp2[-1])
+    p = np.zeros((40, n2))
+    for i in range(40):
+        if sp2[i + 1] > sp2[i]:
+            p[i, sp2[i]:sp2[i + 1]] = 1.0 / (sp2[i + 1] - sp2[i])
+    x2 = np.random.default_rng(7).standard_normal((n2, 6))
+    g2 = np.random.default_rng(8).standard_normal((40, 6))
+    out, _ = O.graph_pool_forward(sp2, x2, "mean")
+    gx, _ = O.graph_pool_backward(sp2, g2, n2, "mean")
+    assert np.allclose(out, p @ x2, rtol=1e-12, atol=1e-13)
+    assert np.allclose(gx, p.T @ g2, rtol=1e-12, atol=1e-13)
+    gs, _ = O.graph_pool_backward(sp2, g2, n2, "sum")
+    assert np.allclose(gs, (p != 0).T.astype(np.float64) @ g2, rtol=1e-12, atol=1e-13)
+
+
+@pytest.mark.parametrize("reduce", ["sum", "mean"])
+def test_graph_pool_adjoint_identity(reduce):
+    sp_ = _ragged_segments(9, 33, 17)
+    n = int(sp_[-1]) + 4                       # trailing rows that belong to no graph
+    rng = np.random.default_rng(10)
+    x = rng.standard_normal((n, 4))
+    g = rng.standard_normal((33, 4))
+    out, _ = O.graph_pool_forward(sp_, x, reduce)
+    gx, _ = O.graph_pool_backward(sp_, g, n, reduce)
+    assert abs((out * g).sum() - (x * gx).sum()) < 1e-10
+    assert not gx[int(sp_[-1]):].any()
