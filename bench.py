@@ -409,6 +409,35 @@ def main():
         for pt in sweep["points"]:
             pt["speedup_vs_capacity_0"] = base_ms / pt["ms_per_step"]
 
+    readout = None
+    meta = getattr(g, "meta", None) or {}
+    if rank == 0 and "graph_size" in meta and g.n % int(meta["graph_size"]) == 0:
+        # graph classification (Section 5.1): the mean-pooling layer after the GNN layers, one row per graph
+        size = int(meta["graph_size"])
+        seg = torch.arange(0, g.n + 1, size, dtype=torch.int32, device=dev)
+        pooled = torch.empty((g.n // size, w.d), dtype=x.dtype, device=dev)
+        gpool = torch.empty_like(x)
+        for _ in range(3):
+            hb.graph_pool_fwd(seg, x, "mean", out=pooled)
+            hb.graph_pool_bwd(seg, pooled, g.n, "mean", out=gpool)
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+        torch.cuda.synchronize(dev)
+        for e3 in ev:
+            flush.zero_()
+            e3[0].record(stream)
+            hb.graph_pool_fwd(seg, x, "mean", out=pooled)
+            e3[1].record(stream)
+            hb.graph_pool_bwd(seg, pooled, g.n, "mean", out=gpool)
+            e3[2].record(stream)
+        torch.cuda.synchronize(dev)
+        f_ms = float(np.mean([e3[0].elapsed_time(e3[1]) for e3 in ev]))
+        b_ms = float(np.mean([e3[1].elapsed_time(e3[2]) for e3 in ev]))
+        rb = (x.numel() + pooled.numel()) * x.element_size()        # each pass reads one matrix and writes the other
+        readout = {"what": f"mean-pooling read-out, {g.n // size} graphs of {size} nodes, cold L2", "fwd_ms": f_ms, "bwd_ms": b_ms,
+                   "fwd_gbps": rb / (f_ms * 1e-3) / 1e9, "bwd_gbps": rb / (b_ms * 1e-3) / 1e9,
+                   "fwd_frac_of_measured_hbm": rb / (f_ms * 1e-3) / 1e9 / measured_peak()[0],
+                   "bwd_frac_of_measured_hbm": rb / (b_ms * 1e-3) / 1e9 / measured_peak()[0]}
+
     if rank == 0:
         bytes_step = 2 * w.layers * nbytes["hag_pass"]
         value = world * bytes_step / (hag_ms * 1e-3) / 1e9
@@ -451,6 +480,8 @@ def main():
         }
         if sweep is not None:
             line["capacity_sweep"] = sweep
+        if readout is not None:
+            line["graph_readout"] = readout
         if w.dtype == "bf16":
             line["dtype"] = "f32 accumulate, bf16 storage"
         print(json.dumps(line))

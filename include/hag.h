@@ -238,6 +238,30 @@ hag_status hag_aggregate_host(hag_t *h, int backward, int use_hag, hag_reduce re
 hag_status hag_profile_enable(hag_t *h, int enable);
 int32_t hag_profile_read(hag_t *h, int32_t max, float *ms, int32_t *kind, int64_t *rows, int64_t *edges);
 
+/* Graph read-out for graph classification (Section 5.1: after the GNN layers "a
+ * mean-pooling layer" gathers graph-level activations).  A batch of graphs is laid
+ * out as in workload shapes of that kind: graph i owns the consecutive node rows
+ * seg_ptr[i] .. seg_ptr[i+1]-1 of x.
+ *   forward : out_i = sum of the rows of graph i, times 1/(number of rows) for
+ *             HAG_MEAN; a graph without rows gives a zero row.  HAG_SUM and HAG_MEAN only.
+ *   backward: grad_x_v = s_i * grad_out_i for every row v of graph i (s_i = 1 or
+ *             1/rows); rows of grad_x before seg_ptr[0] and from seg_ptr[n_graphs]
+ *             to n_rows are set to zero.
+ * seg_ptr: DEVICE pointer to n_graphs + 1 non-decreasing int32 row offsets (not
+ * checked: it lives on the device).  x / grad_x: n_rows x D, out / grad_out:
+ * n_graphs x D of `dtype`, DEVICE pointers, 16-byte aligned, D * sizeof(dtype) a
+ * multiple of 16; accumulation is fp32 on two levels (a row of the sum passes
+ * through at most about rows/64 + 12 roundings).  One kernel each, on the current
+ * device, no handle, no workspace, no allocation.  One warp reads the rows of one
+ * graph, so the launch suits batches of many small graphs.
+ * A matrix that has no rows (out / grad_out when n_graphs = 0, grad_x when n_rows = 0)
+ * may be NULL; x is not read when n_graphs = 0.
+ * Errors: NULL, ARG (D <= 0, n_graphs < 0, n_rows < 0, reduce), DTYPE, ALIGN, CUDA. */
+hag_status hag_graph_pool_fwd(const int32_t *seg_ptr, int32_t n_graphs, hag_reduce reduce, hag_dtype dtype,
+                              int32_t D, const void *x, void *out, void *cuda_stream);
+hag_status hag_graph_pool_bwd(const int32_t *seg_ptr, int32_t n_graphs, int32_t n_rows, hag_reduce reduce,
+                              hag_dtype dtype, int32_t D, const void *grad_out, void *grad_x, void *cuda_stream);
+
 /* hag_aggregate_fwd for callers that must not allocate device memory (the paper
  * has no counterpart: its operators take their buffers from the framework).
  *

@@ -22,11 +22,13 @@ LIB_PATH = os.path.join(_HERE, "libhag_b200.so")
 
 HAG_SUM, HAG_MEAN, HAG_GCN = 0, 1, 2
 HAG_F32, HAG_BF16 = 0, 1
+(HAG_OK, HAG_ERR_NULL, HAG_ERR_ARG, HAG_ERR_GRAPH, HAG_ERR_OOM_HOST, HAG_ERR_OOM_DEVICE, HAG_ERR_CUDA, HAG_ERR_DTYPE,
+ HAG_ERR_ALIGN, HAG_ERR_WORKSPACE, HAG_ERR_TIMEOUT, HAG_ERR_NOT_ON_DEVICE, HAG_ERR_TOO_LARGE) = range(13)
 
 EXPORTED_SYMBOLS = [
     "hag_build", "hag_build_ex", "hag_build_threads", "hag_truncate", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes", "csr_workspace_bytes",
     "hag_aggregate_fwd", "hag_aggregate_bwd", "csr_aggregate_fwd", "csr_aggregate_bwd",
-    "hag_aggregate_host", "hag_aggregate_fwd_static", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
+    "hag_aggregate_host", "hag_aggregate_fwd_static", "hag_graph_pool_fwd", "hag_graph_pool_bwd", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
 ]
 
 
@@ -101,6 +103,10 @@ def load_library():
     lib.hag_aggregate_host.restype = ctypes.c_int
     lib.hag_aggregate_fwd_static.argtypes = [vp, ctypes.c_int, ctypes.c_int, i32, vp, vp, vp]
     lib.hag_aggregate_fwd_static.restype = ctypes.c_int
+    lib.hag_graph_pool_fwd.argtypes = [vp, i32, ctypes.c_int, ctypes.c_int, i32, vp, vp, vp]
+    lib.hag_graph_pool_fwd.restype = ctypes.c_int
+    lib.hag_graph_pool_bwd.argtypes = [vp, i32, i32, ctypes.c_int, ctypes.c_int, i32, vp, vp, vp]
+    lib.hag_graph_pool_bwd.restype = ctypes.c_int
     lib.hag_profile_enable.argtypes = [vp, ctypes.c_int]
     lib.hag_profile_enable.restype = ctypes.c_int
     lib.hag_profile_read.argtypes = [vp, i32, vp, vp, vp, vp]
@@ -326,3 +332,39 @@ class Hag:
                                                self._dtype_code(inp), inp.shape[1], inp.data_ptr(), out.data_ptr(), s)
         _check(st, "hag_aggregate_host")
         return out
+
+
+def _pool_args(seg_ptr, t):
+    import torch
+    if not (seg_ptr.is_cuda and seg_ptr.dtype == torch.int32 and seg_ptr.is_contiguous() and seg_ptr.numel() >= 1):
+        raise ValueError("seg_ptr must be a contiguous int32 device tensor of n_graphs + 1 offsets")
+    if not (t.is_cuda and t.is_contiguous() and t.dim() == 2 and t.device == seg_ptr.device):
+        raise ValueError("features must be a contiguous 2-D tensor on seg_ptr's device")
+    return seg_ptr.numel() - 1, Hag._dtype_code(t)
+
+
+def graph_pool_fwd(seg_ptr, x, reduce="mean", out=None):
+    """``hag_graph_pool_fwd``: one row per graph of a batch (graph i = rows seg_ptr[i]..seg_ptr[i+1]-1 of x)."""
+    import torch
+    n_graphs, code = _pool_args(seg_ptr, x)
+    if out is None:
+        out = torch.empty((n_graphs, x.shape[1]), dtype=x.dtype, device=x.device)
+    with torch.cuda.device(x.device):
+        st = load_library().hag_graph_pool_fwd(seg_ptr.data_ptr(), n_graphs, _reduce_code(reduce), code, x.shape[1],
+                                               x.data_ptr(), out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    _check(st, "hag_graph_pool_fwd")
+    return out
+
+
+def graph_pool_bwd(seg_ptr, grad_out, n_rows: int, reduce="mean", out=None):
+    """``hag_graph_pool_bwd``: the gradient of ``graph_pool_fwd`` for an input of n_rows rows."""
+    import torch
+    n_graphs, code = _pool_args(seg_ptr, grad_out)
+    if out is None:
+        out = torch.empty((n_rows, grad_out.shape[1]), dtype=grad_out.dtype, device=grad_out.device)
+    with torch.cuda.device(grad_out.device):
+        st = load_library().hag_graph_pool_bwd(seg_ptr.data_ptr(), n_graphs, n_rows, _reduce_code(reduce), code,
+                                               grad_out.shape[1], grad_out.data_ptr(), out.data_ptr(),
+                                               torch.cuda.current_stream().cuda_stream)
+    _check(st, "hag_graph_pool_bwd")
+    return out
