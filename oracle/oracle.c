@@ -19,6 +19,12 @@
  *                       per-node upper bounds confirmed by recounts from the definition
  *   o_count_pair / o_max_pair_recount   the Redundancy function of Algorithm 3
  *                       evaluated from its definition
+ *   o6_max_forward / o6_max_backward    the element-wise max Aggregate of the GraphSAGE-P
+ *                       row of Table 1, a_v = max over u in N(v) of z_u, straight
+ *                       from the definition, and its gradient
+ *   o7_hag_max_forward / o7_hag_max_backward   Algorithm 2 with max as the (associative,
+ *                       commutative: Section 3.1, set Aggregate) operator, and its
+ *                       gradient over the transposed HAG
  *
  * All floating point is fp64.  Graph layout: CSR of in-neighbours, row v lists
  * the sources u of v, int64 row pointers, int32 sorted duplicate-free columns.
@@ -153,6 +159,94 @@ void o4_hag_backward(int64_t n, int64_t num_agg, const int64_t *t_ptr, const int
                 const double *gh = ghat + (dst - n) * d;
                 for (int64_t k = 0; k < d; ++k) o[k] += gh[k];
             }
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* O6: element-wise max aggregation (Table 1, GraphSAGE-P) from the definition.
+ * An empty neighbourhood gives a zero row (the reading used for sum as well).  */
+void o6_max_forward(int64_t n, const int64_t *row_ptr, const int32_t *col, int64_t d,
+                    const double *z, double *out)
+{
+    for (int64_t v = 0; v < n; ++v) {
+        double *o = out + v * d;
+        int64_t b = row_ptr[v], e = row_ptr[v + 1];
+        if (e == b) { for (int64_t k = 0; k < d; ++k) o[k] = 0.0; continue; }
+        const double *z0 = z + (int64_t)col[b] * d;
+        for (int64_t k = 0; k < d; ++k) o[k] = z0[k];
+        for (int64_t i = b + 1; i < e; ++i) {
+            const double *zu = z + (int64_t)col[i] * d;
+            for (int64_t k = 0; k < d; ++k) if (zu[k] > o[k]) o[k] = zu[k];
+        }
+    }
+}
+
+/* Gradient of the above for L = sum_v <g_v, a_v>: component k of g_v goes to the
+ * in-neighbours u of v that attain the maximum, z_u[k] == a_v[k].  Reading (the
+ * paper does not say what happens on ties): every such u receives it.  a is
+ * the forward result.  abs_gz receives the same sums over |g|.               */
+void o6_max_backward(int64_t n, const int64_t *row_ptr, const int32_t *col, int64_t d,
+                     const double *z, const double *a, const double *g, double *gz, double *abs_gz)
+{
+    memset(gz, 0, sizeof(double) * (size_t)(n * d));
+    memset(abs_gz, 0, sizeof(double) * (size_t)(n * d));
+    for (int64_t v = 0; v < n; ++v) {
+        const double *av = a + v * d, *gv = g + v * d;
+        for (int64_t i = row_ptr[v]; i < row_ptr[v + 1]; ++i) {
+            int64_t u = col[i];
+            const double *zu = z + u * d;
+            for (int64_t k = 0; k < d; ++k)
+                if (zu[k] == av[k]) { gz[u * d + k] += gv[k]; abs_gz[u * d + k] += fabs(gv[k]); }
+        }
+    }
+}
+
+/* O7: Algorithm 2 with max.  Layout as for o4_hag_forward.  ahat: (n + num_agg) x d
+ * doubles; on return rows n.. hold the maxima of the aggregation nodes (the
+ * backward pass needs them).                                                  */
+void o7_hag_max_forward(int64_t n, int64_t num_agg, const int32_t *agg_in,
+                        const int64_t *res_ptr, const int32_t *res_idx,
+                        int64_t d, const double *z, double *ahat, double *out)
+{
+    memcpy(ahat, z, sizeof(double) * (size_t)(n * d));                 /* lines 3-4 */
+    for (int64_t j = 0; j < num_agg; ++j) {                            /* lines 5-6 */
+        const double *p = ahat + (int64_t)agg_in[2 * j] * d;
+        const double *q = ahat + (int64_t)agg_in[2 * j + 1] * d;
+        double *w = ahat + (n + j) * d;
+        for (int64_t k = 0; k < d; ++k) w[k] = p[k] > q[k] ? p[k] : q[k];
+    }
+    for (int64_t v = 0; v < n; ++v) {                                  /* lines 7-8 */
+        double *o = out + v * d;
+        int64_t b = res_ptr[v], e = res_ptr[v + 1];
+        if (e == b) { for (int64_t k = 0; k < d; ++k) o[k] = 0.0; continue; }
+        const double *a0 = ahat + (int64_t)res_idx[b] * d;
+        for (int64_t k = 0; k < d; ++k) o[k] = a0[k];
+        for (int64_t i = b + 1; i < e; ++i) {
+            const double *a = ahat + (int64_t)res_idx[i] * d;
+            for (int64_t k = 0; k < d; ++k) if (a[k] > o[k]) o[k] = a[k];
+        }
+    }
+}
+
+/* Gradient over the transposed HAG (layout as for o4_hag_backward): a source s
+ * (graph node or aggregation node) receives component k from a destination t
+ * when its value equals the destination's maximum.  Values: ahat for sources and
+ * aggregation-node destinations, the forward output a for graph-node
+ * destinations.  ghat: num_agg x d doubles.                                  */
+void o7_hag_max_backward(int64_t n, int64_t num_agg, const int64_t *t_ptr, const int32_t *t_idx,
+                         int64_t d, const double *ahat, const double *a, const double *g,
+                         double *ghat, double *gz)
+{
+    for (int64_t s = n + num_agg - 1; s >= 0; --s) {
+        double *o = (s >= n) ? ghat + (s - n) * d : gz + s * d;
+        const double *val = ahat + s * d;
+        for (int64_t k = 0; k < d; ++k) o[k] = 0.0;
+        for (int64_t e = t_ptr[s]; e < t_ptr[s + 1]; ++e) {
+            int64_t t = t_idx[e];
+            const double *tv = (t < n) ? a + t * d : ahat + t * d;
+            const double *tg = (t < n) ? g + t * d : ghat + (t - n) * d;
+            for (int64_t k = 0; k < d; ++k) if (val[k] == tv[k]) o[k] += tg[k];
         }
     }
 }

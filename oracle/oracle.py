@@ -29,6 +29,14 @@ What it computes, and where the paper (arxiv 1906.03707) defines it:
   classification: one output row per graph of a batch, the mean (or sum) of the
   rows of its nodes, and the gradient of that; fp64, one slice sum per graph.
 
+* ``direct_max_forward`` / ``direct_max_backward`` -- the element-wise max Aggregate of
+  the GraphSAGE-P row of Table 1 from its definition, and its gradient;
+  ``hag_max_forward`` / ``hag_max_backward`` -- Algorithm 2 with max as the operator
+  (a set Aggregate in the sense of Section 3.1) and its gradient over the
+  transposed HAG.  Reading: on a tie every in-neighbour that attains the maximum
+  receives the gradient component (the paper does not say; ties have probability
+  zero for continuous activations).
+
 Readings of points the paper leaves open:
 redundancy counts graph nodes u in V only (the rewrite loop of Algorithm 3 runs
 over V); pairs are unordered over V and V_A; ties go to the lexicographically
@@ -76,6 +84,14 @@ def _c():
         lib.o4_hag_forward.restype = None
         lib.o4_hag_backward.argtypes = [i64, i64, p, p, p, i64, p, ctypes.c_int, p, p]
         lib.o4_hag_backward.restype = None
+        lib.o6_max_forward.argtypes = [i64, p, p, i64, p, p]
+        lib.o6_max_forward.restype = None
+        lib.o6_max_backward.argtypes = [i64, p, p, i64, p, p, p, p, p]
+        lib.o6_max_backward.restype = None
+        lib.o7_hag_max_forward.argtypes = [i64, i64, p, p, p, i64, p, p, p]
+        lib.o7_hag_max_forward.restype = None
+        lib.o7_hag_max_backward.argtypes = [i64, i64, p, p, i64, p, p, p, p, p]
+        lib.o7_hag_max_backward.restype = None
         lib.o_count_pair.argtypes = [i64, p, p, p, i32, i32]
         lib.o_count_pair.restype = i64
         lib.o_max_pair_recount.argtypes = [i64, p, p, p, i64, i32, p, p]
@@ -429,6 +445,52 @@ def hag_backward(h: CanonicalHag, g, reduce="sum"):
     _c().o4_hag_backward(h.n, h.num_agg, _ptr(np.ascontiguousarray(h.t_ptr)), _ptr(np.ascontiguousarray(h.t_idx)),
                          _ptr(np.ascontiguousarray(h.in_degree)), d, _ptr(g), int(reduce == "mean"), _ptr(scratch), _ptr(gx))
     return gx
+
+
+def direct_max_forward(row_ptr, col_idx, z):
+    """a_v = element-wise max over u in N(v) of z_u (zero row for an empty N(v)), fp64."""
+    rp, ci = _csr(row_ptr, col_idx)
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    out = np.empty_like(z)
+    _c().o6_max_forward(rp.shape[0] - 1, _ptr(rp), _ptr(ci), z.shape[1], _ptr(z), _ptr(out))
+    return out
+
+
+def direct_max_backward(row_ptr, col_idx, z, g):
+    """gz_u[k] = sum over v with u in N(v) and z_u[k] == a_v[k] of g_v[k].  Returns (gz, T),
+    T the same sum over |g| (the scale of the comparison tolerance)."""
+    rp, ci = _csr(row_ptr, col_idx)
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    g = np.ascontiguousarray(g, dtype=np.float64)
+    a = direct_max_forward(rp, ci, z)
+    gz = np.empty_like(z)
+    ab = np.empty_like(z)
+    _c().o6_max_backward(rp.shape[0] - 1, _ptr(rp), _ptr(ci), z.shape[1], _ptr(z), _ptr(a), _ptr(g), _ptr(gz), _ptr(ab))
+    return gz, ab
+
+
+def hag_max_forward(h: CanonicalHag, z):
+    """Algorithm 2 with max.  Returns (out, ahat): ahat has n + num_agg rows, the last
+    num_agg being the maxima held by the aggregation nodes."""
+    z = np.ascontiguousarray(z, dtype=np.float64)
+    d = z.shape[1]
+    ahat = np.empty((h.n + h.num_agg, d), dtype=np.float64)
+    out = np.empty((h.n, d), dtype=np.float64)
+    _c().o7_hag_max_forward(h.n, h.num_agg, _ptr(np.ascontiguousarray(h.agg_in)), _ptr(np.ascontiguousarray(h.res_ptr)),
+                            _ptr(np.ascontiguousarray(h.res_idx)), d, _ptr(z), _ptr(ahat), _ptr(out))
+    return out, ahat
+
+
+def hag_max_backward(h: CanonicalHag, z, g):
+    """Gradient of hag_max_forward over the transposed HAG."""
+    g = np.ascontiguousarray(g, dtype=np.float64)
+    out, ahat = hag_max_forward(h, z)
+    d = g.shape[1]
+    ghat = np.empty((max(h.num_agg, 1), d), dtype=np.float64)
+    gz = np.empty((h.n, d), dtype=np.float64)
+    _c().o7_hag_max_backward(h.n, h.num_agg, _ptr(np.ascontiguousarray(h.t_ptr)), _ptr(np.ascontiguousarray(h.t_idx)), d,
+                             _ptr(ahat), _ptr(out), _ptr(g), _ptr(ghat), _ptr(gz))
+    return gz
 
 
 # --------------------------------------------------------------------------- #

@@ -458,3 +458,110 @@ def test_graph_pool_adjoint_identity(reduce):
     gx, _ = O.graph_pool_backward(sp_, g, n, reduce)
     assert abs((out * g).sum() - (x * gx).sum()) < 1e-10
     assert not gx[int(sp_[-1]):].any()
+
+
+# --------------------------------------------------------------------------- #
+# Element-wise max aggregation (GraphSAGE-P row of Table 1)
+# --------------------------------------------------------------------------- #
+def _max_bruteforce(g, z, gr):
+    """Loops over the definition: a_v[k] = max_{u in N(v)} z_u[k]; each maximiser receives g_v[k]."""
+    n, d = z.shape
+    a = np.zeros((n, d))
+    gz = np.zeros((n, d))
+    for v in range(n):
+        nb = [int(u) for u in g.col_idx[g.row_ptr[v]:g.row_ptr[v + 1]]]
+        for k in range(d):
+            if not nb:
+                continue
+            m = max(z[u, k] for u in nb)
+            a[v, k] = m
+            for u in nb:
+                if z[u, k] == m:
+                    gz[u, k] += gr[v, k]
+    return a, gz
+
+
+@pytest.mark.parametrize("seed", range(6))
+@pytest.mark.parametrize("ties", [False, True])
+def test_max_matches_bruteforce_on_tiny_graphs(seed, ties):
+    rng = np.random.default_rng(100 + seed)
+    g = synth.random_digraph(seed=seed, n=int(rng.integers(5, 30)), p=0.3, undirected=bool(seed % 3 == 0), self_loops=bool(seed % 2))
+    d = 3
+    z = rng.integers(-2, 3, size=(g.n, d)).astype(np.float64) if ties else rng.standard_normal((g.n, d))
+    gr = rng.integers(-4, 5, size=(g.n, d)).astype(np.float64)
+    a, gz = _max_bruteforce(g, z, gr)
+    assert np.array_equal(O.direct_max_forward(g.row_ptr, g.col_idx, z), a)
+    got, t = O.direct_max_backward(g.row_ptr, g.col_idx, z, gr)
+    assert np.array_equal(got, gz)
+    assert (t >= np.abs(got)).all()
+
+
+def test_max_is_the_masked_dense_maximum_and_empty_rows_are_zero():
+    g = synth.random_digraph(seed=3, n=40, p=0.08, undirected=False, self_loops=False)
+    assert (np.diff(g.row_ptr) == 0).any()                     # the case has empty neighbourhoods
+    z = np.random.default_rng(4).standard_normal((g.n, 5))
+    adj = np.zeros((g.n, g.n), dtype=bool)
+    for v in range(g.n):
+        adj[v, g.col_idx[g.row_ptr[v]:g.row_ptr[v + 1]]] = True
+    dense = np.where(adj[:, :, None], z[None, :, :], -np.inf).max(axis=1)
+    dense[~adj.any(axis=1)] = 0.0
+    assert np.array_equal(O.direct_max_forward(g.row_ptr, g.col_idx, z), dense)
+
+
+def test_max_gradient_is_the_finite_difference_of_the_loss():
+    # without ties the aggregation is linear around z, so a small step gives the derivative exactly
+    g = synth.random_digraph(seed=5, n=9, p=0.45, undirected=False, self_loops=True)
+    rng = np.random.default_rng(6)
+    z = rng.permutation(g.n * 3).reshape(g.n, 3).astype(np.float64)        # all distinct, gaps of 1
+    gr = rng.standard_normal((g.n, 3))
+    gz, _ = O.direct_max_backward(g.row_ptr, g.col_idx, z, gr)
+    base = (gr * O.direct_max_forward(g.row_ptr, g.col_idx, z)).sum()
+    eps = 1.0 / 64.0
+    for u in range(g.n):
+        for k in range(3):
+            zp = z.copy()
+            zp[u, k] += eps
+            num = ((gr * O.direct_max_forward(g.row_ptr, g.col_idx, zp)).sum() - base) / eps
+            assert abs(num - gz[u, k]) < 1e-9
+
+
+def test_max_closed_forms():
+    g = synth.config1_graph()
+    n = g.n
+    rng = np.random.default_rng(7)
+    gr = rng.standard_normal((n, 4))
+    # constant features: every in-neighbour ties, so the gradient is that of the sum
+    gz, _ = O.direct_max_backward(g.row_ptr, g.col_idx, np.full((n, 4), 1.5), gr)
+    want, _ = O.direct_backward(g.row_ptr, g.col_idx, gr, "sum")
+    assert np.allclose(gz, want, rtol=1e-13, atol=1e-13)
+    # features that grow with the node id: the maximum sits at the last (largest) in-neighbour of the sorted row
+    z = np.arange(n, dtype=np.float64)[:, None] * np.ones((1, 4))
+    a = O.direct_max_forward(g.row_ptr, g.col_idx, z)
+    last = g.col_idx[g.row_ptr[1:] - 1]
+    assert np.array_equal(a[:, 0], last.astype(np.float64))
+    gz, _ = O.direct_max_backward(g.row_ptr, g.col_idx, z, gr)
+    want = np.zeros((n, 4))
+    np.add.at(want, last, gr)
+    assert np.allclose(gz, want, rtol=1e-13, atol=1e-13)
+
+
+@pytest.mark.parametrize("maker", [lambda: synth.config1_graph(), lambda: synth.workload(2, scale=0.05).graph,
+                                   lambda: synth.clique_union_graph(seed=2, n=600, n_groups=150, g_lo=2, g_hi=40, g_alpha=2.0)])
+def test_hag_max_equals_direct_max(maker):
+    """Theorem 2's cover condition makes Algorithm 2 with any associative, commutative operator reach
+    the GNN-graph's result; for max that holds bit for bit, and with integer gradients so does the backward
+    pass, ties included."""
+    g = maker()
+    res = O.greedy_pairmap(g.row_ptr, g.col_idx, g.n // 4)
+    h = O.canonical_hag(g.row_ptr, res)
+    assert h.num_agg > 0
+    rng = np.random.default_rng(8)
+    for z in (rng.standard_normal((g.n, 6)), rng.integers(-1, 2, size=(g.n, 6)).astype(np.float64)):
+        gr = rng.integers(-3, 4, size=(g.n, 6)).astype(np.float64)
+        out, ahat = O.hag_max_forward(h, z)
+        assert np.array_equal(out, O.direct_max_forward(g.row_ptr, g.col_idx, z))
+        for j in rng.integers(0, h.num_agg, size=20):          # an aggregation node holds the max over its inputs
+            p, q = h.agg_in[2 * j], h.agg_in[2 * j + 1]
+            assert np.array_equal(ahat[h.n + j], np.maximum(ahat[p], ahat[q]))
+        want, _ = O.direct_max_backward(g.row_ptr, g.col_idx, z, gr)
+        assert np.array_equal(O.hag_max_backward(h, z, gr), want)
