@@ -262,6 +262,42 @@ hag_status hag_graph_pool_fwd(const int32_t *seg_ptr, int32_t n_graphs, hag_redu
 hag_status hag_graph_pool_bwd(const int32_t *seg_ptr, int32_t n_graphs, int32_t n_rows, hag_reduce reduce,
                               hag_dtype dtype, int32_t D, const void *grad_out, void *grad_x, void *cuda_stream);
 
+/* Element-wise max aggregation over the same HAG (Table 1, GraphSAGE-P:
+ * a_v = max over u in N(v) of z_u, z = the activations the model feeds to the
+ * pooling).  Max is associative and commutative, i.e. a set Aggregate in the sense
+ * of Section 3.1, so Algorithm 2 applies with max in place of the sum and the HAG
+ * built by hag_build is reused as it is.
+ *   hag_max_fwd : a-hat_w = max(a-hat_in0, a-hat_in1) for aggregation nodes, then
+ *                 out_v = max over the residual in-neighbours of v; an empty
+ *                 neighbourhood gives a zero row.  Exact (no rounding): the result
+ *                 equals the direct evaluation bit for bit, for both dtypes.
+ *                 `workspace`: hag_max_workspace_bytes(h, D) bytes (|V_A| x D fp32);
+ *                 after the call it holds the maxima of the aggregation nodes,
+ *                 which hag_max_bwd needs: keep it until then.
+ *   hag_max_bwd : gradient for L = sum_v <grad_out_v, out_v>: component k of
+ *                 grad_out_v goes to the in-neighbours u with z_u[k] == out_v[k];
+ *                 on a tie every such u receives it (the paper does not say; ties
+ *                 have probability zero for continuous activations).  Computed as
+ *                 a gather over the transposed HAG, no atomics, fixed summation
+ *                 order.  Takes z and out of the forward call, `fwd_workspace` as
+ *                 hag_max_fwd left it (read only), and a second buffer `workspace`
+ *                 of the same size for the gradients of the aggregation nodes.
+ *   csr_max_fwd / csr_max_bwd : the same on the plain GNN-graph (no workspace).
+ * z, out, grad_out, grad_z: N x D of `dtype`, DEVICE pointers, 16-byte aligned, must not
+ * overlap one another; values must not be NaN.  Rows are not split: a row of a
+ * thousand entries is walked by one warp.
+ * Errors: NULL, ARG (D <= 0, overlapping buffers), DTYPE, ALIGN, WORKSPACE,
+ * NOT_ON_DEVICE, CUDA. */
+size_t hag_max_workspace_bytes(const hag_t *h, int32_t D);
+hag_status hag_max_fwd(const hag_t *h, hag_dtype dtype, int32_t D, const void *z, void *out, void *workspace,
+                       void *cuda_stream);
+hag_status hag_max_bwd(const hag_t *h, hag_dtype dtype, int32_t D, const void *z, const void *out,
+                       const void *fwd_workspace, const void *grad_out, void *grad_z, void *workspace,
+                       void *cuda_stream);
+hag_status csr_max_fwd(const hag_t *h, hag_dtype dtype, int32_t D, const void *z, void *out, void *cuda_stream);
+hag_status csr_max_bwd(const hag_t *h, hag_dtype dtype, int32_t D, const void *z, const void *out,
+                       const void *grad_out, void *grad_z, void *cuda_stream);
+
 /* hag_aggregate_fwd for callers that must not allocate device memory (the paper
  * has no counterpart: its operators take their buffers from the framework).
  *

@@ -28,7 +28,8 @@ HAG_F32, HAG_BF16 = 0, 1
 EXPORTED_SYMBOLS = [
     "hag_build", "hag_build_ex", "hag_build_threads", "hag_truncate", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes", "csr_workspace_bytes",
     "hag_aggregate_fwd", "hag_aggregate_bwd", "csr_aggregate_fwd", "csr_aggregate_bwd",
-    "hag_aggregate_host", "hag_aggregate_fwd_static", "hag_graph_pool_fwd", "hag_graph_pool_bwd", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
+    "hag_aggregate_host", "hag_aggregate_fwd_static", "hag_graph_pool_fwd", "hag_graph_pool_bwd",
+    "hag_max_workspace_bytes", "hag_max_fwd", "hag_max_bwd", "csr_max_fwd", "csr_max_bwd", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
 ]
 
 
@@ -107,6 +108,16 @@ def load_library():
     lib.hag_graph_pool_fwd.restype = ctypes.c_int
     lib.hag_graph_pool_bwd.argtypes = [vp, i32, i32, ctypes.c_int, ctypes.c_int, i32, vp, vp, vp]
     lib.hag_graph_pool_bwd.restype = ctypes.c_int
+    lib.hag_max_workspace_bytes.argtypes = [vp, i32]
+    lib.hag_max_workspace_bytes.restype = ctypes.c_size_t
+    lib.hag_max_fwd.argtypes = [vp, ctypes.c_int, i32, vp, vp, vp, vp]
+    lib.hag_max_fwd.restype = ctypes.c_int
+    lib.hag_max_bwd.argtypes = [vp, ctypes.c_int, i32, vp, vp, vp, vp, vp, vp, vp]
+    lib.hag_max_bwd.restype = ctypes.c_int
+    lib.csr_max_fwd.argtypes = [vp, ctypes.c_int, i32, vp, vp, vp]
+    lib.csr_max_fwd.restype = ctypes.c_int
+    lib.csr_max_bwd.argtypes = [vp, ctypes.c_int, i32, vp, vp, vp, vp, vp]
+    lib.csr_max_bwd.restype = ctypes.c_int
     lib.hag_profile_enable.argtypes = [vp, ctypes.c_int]
     lib.hag_profile_enable.restype = ctypes.c_int
     lib.hag_profile_read.argtypes = [vp, i32, vp, vp, vp, vp]
@@ -320,6 +331,46 @@ class Hag:
     def csr_bwd(self, grad_out, reduce="sum", out=None, workspace=None):
         """``csr_aggregate_bwd``."""
         return self._run("csr_aggregate_bwd", False, grad_out, reduce, out, workspace)
+
+    def max_workspace(self, d: int, device):
+        """A fresh buffer of ``hag_max_workspace_bytes`` (the forward pass leaves the aggregation nodes' maxima in it)."""
+        import torch
+        need = max(int(load_library().hag_max_workspace_bytes(self._h, d)), 16)
+        return torch.empty(need // 4, dtype=torch.float32, device=device)
+
+    def max_fwd(self, z, out=None, workspace=None, use_hag=True):
+        """``hag_max_fwd`` (or ``csr_max_fwd``).  Returns (out, workspace); keep both for ``max_bwd``."""
+        import torch
+        if out is None:
+            out = torch.empty_like(z)
+        s = torch.cuda.current_stream().cuda_stream
+        lib = load_library()
+        if use_hag:
+            if workspace is None:
+                workspace = self.max_workspace(z.shape[1], z.device)
+            st = lib.hag_max_fwd(self._h, self._dtype_code(z), z.shape[1], z.data_ptr(), out.data_ptr(), workspace.data_ptr(), s)
+        else:
+            st = lib.csr_max_fwd(self._h, self._dtype_code(z), z.shape[1], z.data_ptr(), out.data_ptr(), s)
+        _check(st, "hag_max_fwd" if use_hag else "csr_max_fwd")
+        return out, workspace
+
+    def max_bwd(self, z, fwd_out, fwd_workspace, grad_out, out=None, workspace=None, use_hag=True):
+        """``hag_max_bwd`` (or ``csr_max_bwd``): the gradient with respect to z."""
+        import torch
+        if out is None:
+            out = torch.empty_like(z)
+        s = torch.cuda.current_stream().cuda_stream
+        lib = load_library()
+        code = self._dtype_code(z)
+        if use_hag:
+            if workspace is None:
+                workspace = self.max_workspace(z.shape[1], z.device)
+            st = lib.hag_max_bwd(self._h, code, z.shape[1], z.data_ptr(), fwd_out.data_ptr(), fwd_workspace.data_ptr(),
+                                 grad_out.data_ptr(), out.data_ptr(), workspace.data_ptr(), s)
+        else:
+            st = lib.csr_max_bwd(self._h, code, z.shape[1], z.data_ptr(), fwd_out.data_ptr(), grad_out.data_ptr(), out.data_ptr(), s)
+        _check(st, "hag_max_bwd" if use_hag else "csr_max_bwd")
+        return out
 
     def aggregate_host(self, inp, out, reduce="sum", backward=False, use_hag=True, stream=None):
         """``hag_aggregate_host``: host tensors in and out (pinned for async copies);

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhag_b200.so")
-SOURCES = ["hag_build.cpp", "hag_cuda.cu", "hag_pool.cu"]
+SOURCES = ["hag_build.cpp", "hag_cuda.cu", "hag_pool.cu", "hag_max.cu"]
 HEADERS = [os.path.join(ROOT, "include", "hag.h"), os.path.join(CSRC, "hag_internal.h"),
            os.path.join(CSRC, "hag_kernels.cuh")]
 

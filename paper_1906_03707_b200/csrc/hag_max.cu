@@ -1,0 +1,459 @@
+// Element-wise max aggregation (the GraphSAGE-P row of Table 1) over the same HAG:
+// max is associative and commutative (a set Aggregate, Section 3.1), so Algorithm 2
+// holds with max in place of the sum, and by the cover condition of Theorem 2 every
+// in-neighbour reaches its node along exactly one path.  Forward: pair kernel for
+// the shallow levels, one gather for the expanded deep levels, one gather over the
+// residual rows.  Backward: a component of the gradient of a node goes to the sources
+// whose value equals the node's maximum; evaluated as a gather over the transposed
+// HAG (no atomics, fixed summation order), two row loads per entry: the
+// destination's maximum and its gradient.
+//
+// One warp per row, LPR lanes per row chunk of 16 bytes, 32/LPR lane groups on
+// alternate entries, ids read 32 at a time and handed round by shuffle.  Rows are
+// not split here (a row of a thousand entries is walked by one warp).
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <limits>
+
+#include "hag.h"
+#include "hag_internal.h"
+#include "hag_kernels.cuh"
+
+namespace {
+
+using hagk::Chunk;
+using hagk::kThreads;
+using hagk::kWarps;
+using hagk::Tables;
+
+struct MaxArgs {
+    const int32_t *row_ptr;   // indexed by absolute row id
+    const int32_t *idx;
+    int32_t row_begin, row_count;
+    int32_t n_prim;           // ids below: graph nodes (rows of T); from it on: aggregation nodes (fp32 rows)
+    int32_t D;
+    // forward: values of the sources.  backward: maxima of the destinations (forward output / kept a-hat rows)
+    const void *val_prim;
+    const float *val_sec;
+    // backward only: gradients of the destinations, and this row's own value
+    const void *grad_prim;
+    const float *grad_sec;
+    const void *own_prim;
+    const float *own_sec;
+    void *out;
+    int32_t out_is_f32;
+    int32_t out_row_offset;
+};
+
+struct PairMaxArgs {
+    const int32_t *agg_in;
+    int32_t first, count;
+    const void *z;
+    float *ahat;
+    int32_t n, D;
+};
+
+constexpr int kMaxLoads = 4;        // forward: row loads in flight per lane
+constexpr int kGradEntries = 2;     // backward: entries in flight per lane (two loads each)
+
+template <typename T, int LPR>
+__global__ void __launch_bounds__(kThreads) gather_max_kernel(const MaxArgs a) {
+    hagk::pdl_launch_dependents();
+    constexpr int E = Chunk<T>::kElems;
+    constexpr int G = 32 / LPR;
+    constexpr int U = kMaxLoads < LPR ? kMaxLoads : LPR;
+    const int lane = threadIdx.x & 31;
+    const int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (r_local >= a.row_count) return;
+    const int32_t row = a.row_begin + r_local;
+    const int32_t b = __ldg(a.row_ptr + row), e = __ldg(a.row_ptr + row + 1);
+    const int32_t first = (b + lane < e) ? __ldg(a.idx + b + lane) : -1;
+    hagk::pdl_wait();
+    const int slice = lane / LPR, gl = lane % LPR;
+    const int n_chunks = a.D / E;
+    const float ninf = __int_as_float(0xff800000);      // -infinity: the neutral element of max
+    for (int c0 = 0; c0 < n_chunks; c0 += LPR) {
+        const int chunk = c0 + gl;
+        const bool live = chunk < n_chunks;
+        const Tables<T> tab(a.val_prim, a.val_sec, a.n_prim, a.D, live ? chunk : 0);
+        float acc[E];
+#pragma unroll
+        for (int j = 0; j < E; ++j) acc[j] = ninf;
+        int32_t mine = (c0 == 0) ? first : ((b + lane < e) ? __ldg(a.idx + b + lane) : -1);
+        for (int32_t base = b; base < e; base += 32) {
+            const int32_t cur = mine;
+            const int32_t nb = base + 32;
+            mine = (nb + lane < e) ? __ldg(a.idx + nb + lane) : -1;
+            const int cnt = min(32, e - base);
+#pragma unroll
+            for (int k = 0; k < LPR; k += U) {
+                if (k * G < cnt) {
+                    float v[U][E];
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        const int32_t id = __shfl_sync(0xffffffffu, cur, (k + u) * G + slice);
+                        if (id >= 0 && live) {
+                            tab.load(id, v[u]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < E; ++j) v[u][j] = ninf;
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < U; ++u)
+#pragma unroll
+                        for (int j = 0; j < E; ++j) acc[j] = fmaxf(acc[j], v[u][j]);
+                }
+            }
+        }
+#pragma unroll
+        for (int off = LPR; off < 32; off <<= 1)
+#pragma unroll
+            for (int j = 0; j < E; ++j) acc[j] = fmaxf(acc[j], __shfl_xor_sync(0xffffffffu, acc[j], off));
+        if (live && slice == 0) {
+            if (e == b) {                 // empty neighbourhood: zero row
+#pragma unroll
+                for (int j = 0; j < E; ++j) acc[j] = 0.0f;
+            }
+            hagk::store_chunk<T>(a.out, a.out_is_f32, a.D, row - a.out_row_offset, chunk, acc);
+        }
+    }
+}
+
+// a-hat_w = max(a-hat_in0, a-hat_in1) for one level; one lane group per aggregation node.
+template <typename T, int LPR>
+__global__ void __launch_bounds__(kThreads) pair_max_kernel(const PairMaxArgs p) {
+    hagk::pdl_launch_dependents();
+    constexpr int E = Chunk<T>::kElems;
+    constexpr int G = 32 / LPR;
+    const int lane = threadIdx.x & 31;
+    const int slice = lane / LPR, gl = lane % LPR;
+    const int32_t j = (blockIdx.x * kWarps + (threadIdx.x >> 5)) * G + slice;
+    if (j >= p.count) return;
+    const int2 in = __ldg(reinterpret_cast<const int2 *>(p.agg_in) + p.first + j);
+    hagk::pdl_wait();
+    const int n_chunks = p.D / E;
+    for (int chunk = gl; chunk < n_chunks; chunk += LPR) {
+        const Tables<T> tab(p.z, p.ahat, p.n, p.D, chunk);
+        float u[E], v[E];
+        tab.load(in.x, u);
+        tab.load(in.y, v);
+#pragma unroll
+        for (int i = 0; i < E; ++i) u[i] = fmaxf(u[i], v[i]);
+        hagk::store_chunk<T>(p.ahat, 1, p.D, p.first + j, chunk, u);
+    }
+}
+
+// grad_s[k] = sum over the destinations t of row s with max_t[k] == value_s[k] of grad_t[k].
+template <typename T, int LPR>
+__global__ void __launch_bounds__(kThreads) gather_maxgrad_kernel(const MaxArgs a) {
+    hagk::pdl_launch_dependents();
+    constexpr int E = Chunk<T>::kElems;
+    constexpr int G = 32 / LPR;
+    constexpr int U = kGradEntries < LPR ? kGradEntries : LPR;
+    const int lane = threadIdx.x & 31;
+    const int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (r_local >= a.row_count) return;
+    const int32_t row = a.row_begin + r_local;
+    const int32_t b = __ldg(a.row_ptr + row), e = __ldg(a.row_ptr + row + 1);
+    const int32_t first = (b + lane < e) ? __ldg(a.idx + b + lane) : -1;
+    hagk::pdl_wait();
+    const int slice = lane / LPR, gl = lane % LPR;
+    const int n_chunks = a.D / E;
+    for (int c0 = 0; c0 < n_chunks; c0 += LPR) {
+        const int chunk = c0 + gl;
+        const bool live = chunk < n_chunks;
+        const Tables<T> vals(a.val_prim, a.val_sec, a.n_prim, a.D, live ? chunk : 0);
+        const Tables<T> grads(a.grad_prim, a.grad_sec, a.n_prim, a.D, live ? chunk : 0);
+        float own[E], acc[E];
+        {
+            const Tables<T> self(a.own_prim, a.own_sec, a.n_prim, a.D, live ? chunk : 0);
+            self.load(row, own);
+        }
+#pragma unroll
+        for (int j = 0; j < E; ++j) acc[j] = 0.0f;
+        int32_t mine = (c0 == 0) ? first : ((b + lane < e) ? __ldg(a.idx + b + lane) : -1);
+        for (int32_t base = b; base < e; base += 32) {
+            const int32_t cur = mine;
+            const int32_t nb = base + 32;
+            mine = (nb + lane < e) ? __ldg(a.idx + nb + lane) : -1;
+            const int cnt = min(32, e - base);
+            float part[E];            // two-level sum: one partial per batch of 32 ids
+#pragma unroll
+            for (int j = 0; j < E; ++j) part[j] = 0.0f;
+#pragma unroll
+            for (int k = 0; k < LPR; k += U) {
+                if (k * G < cnt) {
+                    float tv[U][E], tg[U][E];
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        const int32_t id = __shfl_sync(0xffffffffu, cur, (k + u) * G + slice);
+                        if (id >= 0 && live) {
+                            vals.load(id, tv[u]);
+                            grads.load(id, tg[u]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < E; ++j) { tv[u][j] = own[j]; tg[u][j] = 0.0f; }
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < U; ++u)
+#pragma unroll
+                        for (int j = 0; j < E; ++j) part[j] += (tv[u][j] == own[j]) ? tg[u][j] : 0.0f;
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < E; ++j) acc[j] += part[j];
+        }
+#pragma unroll
+        for (int off = LPR; off < 32; off <<= 1)
+#pragma unroll
+            for (int j = 0; j < E; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], off);
+        if (live && slice == 0) hagk::store_chunk<T>(a.out, a.out_is_f32, a.D, row - a.out_row_offset, chunk, acc);
+    }
+}
+
+struct DeviceScope {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceScope(int device) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != device && cudaSetDevice(device) != cudaSuccess) ok = false;
+    }
+    ~DeviceScope() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+template <typename Args>
+cudaError_t launch(void (*kernel)(Args), int64_t warps, const Args &args, cudaStream_t s) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(unsigned((warps + kWarps - 1) / kWarps));
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args);
+}
+
+int lanes_for(int n_chunks) {
+    int l = 4;
+    while (l < 32 && l < n_chunks) l *= 2;
+    return l;
+}
+
+template <typename T>
+cudaError_t launch_rows(bool grad, const MaxArgs &a, cudaStream_t s) {
+    if (a.row_count <= 0) return cudaSuccess;
+    switch (lanes_for(a.D / Chunk<T>::kElems)) {
+        case 4: return grad ? launch(gather_maxgrad_kernel<T, 4>, a.row_count, a, s) : launch(gather_max_kernel<T, 4>, a.row_count, a, s);
+        case 8: return grad ? launch(gather_maxgrad_kernel<T, 8>, a.row_count, a, s) : launch(gather_max_kernel<T, 8>, a.row_count, a, s);
+        case 16: return grad ? launch(gather_maxgrad_kernel<T, 16>, a.row_count, a, s) : launch(gather_max_kernel<T, 16>, a.row_count, a, s);
+        default: return grad ? launch(gather_maxgrad_kernel<T, 32>, a.row_count, a, s) : launch(gather_max_kernel<T, 32>, a.row_count, a, s);
+    }
+}
+
+template <typename T>
+cudaError_t launch_pair_level(const PairMaxArgs &p, cudaStream_t s) {
+    if (p.count <= 0) return cudaSuccess;
+    const int lpr = lanes_for(p.D / Chunk<T>::kElems);
+    const int64_t warps = (int64_t(p.count) + (32 / lpr) - 1) / (32 / lpr);
+    switch (lpr) {
+        case 4: return launch(pair_max_kernel<T, 4>, warps, p, s);
+        case 8: return launch(pair_max_kernel<T, 8>, warps, p, s);
+        case 16: return launch(pair_max_kernel<T, 16>, warps, p, s);
+        default: return launch(pair_max_kernel<T, 32>, warps, p, s);
+    }
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+hag_status check(const hag *h, hag_dtype dtype, int32_t D) {
+    if (!h) return HAG_ERR_NULL;
+    if (dtype != HAG_F32 && dtype != HAG_BF16) return HAG_ERR_DTYPE;
+    if (D <= 0) return HAG_ERR_ARG;
+    if ((size_t(D) * (dtype == HAG_F32 ? 4 : 2)) % 16 != 0) return HAG_ERR_ALIGN;
+    if (h->device < 0) return HAG_ERR_NOT_ON_DEVICE;
+    return HAG_OK;
+}
+
+constexpr int32_t kAllPrim = std::numeric_limits<int32_t>::max();
+
+template <typename T>
+hag_status max_fwd(hag *h, bool use_hag, int32_t D, const void *z, void *out, float *ahat, cudaStream_t s) {
+    const hag_device_arrays &d = h->d;
+    int32_t launches = 0;
+    MaxArgs a{};
+    a.D = D;
+    a.val_prim = z;
+    a.n_prim = kAllPrim;
+    if (use_hag && h->num_agg > 0) {
+        for (int32_t l = 1; l <= h->fwd_cut; ++l) {        // Algorithm 2 lines 5-6, level by level
+            PairMaxArgs p{d.agg_in, int32_t(h->level_ptr[l - 1]), int32_t(h->level_ptr[l] - h->level_ptr[l - 1]), z, ahat, h->n, D};
+            if (p.count <= 0) continue;
+            if (launch_pair_level<T>(p, s) != cudaSuccess) return HAG_ERR_CUDA;
+            ++launches;
+        }
+        const int32_t j0 = int32_t(h->level_ptr[h->fwd_cut]);
+        if (j0 < h->num_agg) {                             // the deeper nodes from their expansion: max over the cover
+            MaxArgs t = a;
+            t.row_ptr = d.ftail_ptr - (h->n + j0);
+            t.idx = d.ftail_idx;
+            t.row_begin = h->n + j0;
+            t.row_count = h->num_agg - j0;
+            t.val_sec = ahat;
+            t.n_prim = h->n;
+            t.out = ahat;
+            t.out_is_f32 = 1;
+            t.out_row_offset = h->n;
+            if (launch_rows<T>(false, t, s) != cudaSuccess) return HAG_ERR_CUDA;
+            ++launches;
+        }
+        a.val_sec = ahat;
+        a.n_prim = h->n;
+    }
+    a.row_ptr = use_hag ? d.res_ptr : d.csr_ptr;           // lines 7-8
+    a.idx = use_hag ? d.res_idx : d.csr_idx;
+    a.row_begin = 0;
+    a.row_count = h->n;
+    a.out = out;
+    if (h->n > 0) {
+        if (launch_rows<T>(false, a, s) != cudaSuccess) return HAG_ERR_CUDA;
+        ++launches;
+    }
+    h->last_launches = launches;
+    return HAG_OK;
+}
+
+template <typename T>
+hag_status max_bwd(hag *h, bool use_hag, int32_t D, const void *z, const void *out, const float *ahat, const void *g,
+                   void *gz, float *ghat, cudaStream_t s) {
+    const hag_device_arrays &d = h->d;
+    int32_t launches = 0;
+    MaxArgs a{};
+    a.D = D;
+    a.val_prim = out;         // a graph-node destination: its forward output and its incoming gradient
+    a.grad_prim = g;
+    a.own_prim = z;
+    a.n_prim = kAllPrim;
+    if (use_hag && h->num_agg > 0) {
+        a.val_sec = ahat;     // an aggregation-node destination: its kept maximum and its computed gradient
+        a.grad_sec = ghat;
+        a.own_sec = ahat;
+        a.n_prim = h->n;
+        const int32_t j0 = int32_t(h->level_ptr[h->bwd_cut]);
+        if (j0 < h->num_agg) {                             // deep nodes straight from the graph nodes that use them
+            MaxArgs t = a;
+            t.row_ptr = d.btail_ptr - (h->n + j0);
+            t.idx = d.btail_idx;
+            t.row_begin = h->n + j0;
+            t.row_count = h->num_agg - j0;
+            t.out = ghat;
+            t.out_is_f32 = 1;
+            t.out_row_offset = h->n;
+            if (launch_rows<T>(true, t, s) != cudaSuccess) return HAG_ERR_CUDA;
+            ++launches;
+        }
+        for (int32_t l = h->bwd_cut; l >= 1; --l) {
+            MaxArgs lv = a;
+            lv.row_ptr = d.t_ptr;
+            lv.idx = d.t_idx;
+            lv.row_begin = h->n + int32_t(h->level_ptr[l - 1]);
+            lv.row_count = int32_t(h->level_ptr[l] - h->level_ptr[l - 1]);
+            lv.out = ghat;
+            lv.out_is_f32 = 1;
+            lv.out_row_offset = h->n;
+            if (lv.row_count <= 0) continue;
+            if (launch_rows<T>(true, lv, s) != cudaSuccess) return HAG_ERR_CUDA;
+            ++launches;
+        }
+    }
+    a.row_ptr = use_hag ? d.t_ptr : d.csr_t_ptr;
+    a.idx = use_hag ? d.t_idx : d.csr_t_idx;
+    a.row_begin = 0;
+    a.row_count = h->n;
+    a.out = gz;
+    if (h->n > 0) {
+        if (launch_rows<T>(true, a, s) != cudaSuccess) return HAG_ERR_CUDA;
+        ++launches;
+    }
+    h->last_launches = launches;
+    return HAG_OK;
+}
+
+hag_status run_fwd(const hag_t *hc, bool use_hag, hag_dtype dtype, int32_t D, const void *z, void *out, void *ws, void *stream) {
+    hag_status st = check(hc, dtype, D);
+    if (st != HAG_OK) return st;
+    if (!z || !out) return HAG_ERR_NULL;
+    if (!aligned16(z) || !aligned16(out)) return HAG_ERR_ALIGN;
+    if (z == out) return HAG_ERR_ARG;
+    hag *h = const_cast<hag *>(hc);
+    if (use_hag && h->num_agg > 0) {
+        if (!ws) return HAG_ERR_WORKSPACE;
+        if (!aligned16(ws)) return HAG_ERR_ALIGN;
+    }
+    DeviceScope scope(h->device);
+    if (!scope.ok) { cudaGetLastError(); return HAG_ERR_CUDA; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = dtype == HAG_F32 ? max_fwd<float>(h, use_hag, D, z, out, static_cast<float *>(ws), s)
+                          : max_fwd<__nv_bfloat16>(h, use_hag, D, z, out, static_cast<float *>(ws), s);
+    if (st != HAG_OK) cudaGetLastError();
+    return st;
+}
+
+hag_status run_bwd(const hag_t *hc, bool use_hag, hag_dtype dtype, int32_t D, const void *z, const void *out, const void *fwd_ws,
+                   const void *g, void *gz, void *ws, void *stream) {
+    hag_status st = check(hc, dtype, D);
+    if (st != HAG_OK) return st;
+    if (!z || !out || !g || !gz) return HAG_ERR_NULL;
+    if (!aligned16(z) || !aligned16(out) || !aligned16(g) || !aligned16(gz)) return HAG_ERR_ALIGN;
+    if (gz == z || gz == out || gz == g) return HAG_ERR_ARG;
+    hag *h = const_cast<hag *>(hc);
+    if (use_hag && h->num_agg > 0) {
+        if (!ws || !fwd_ws) return HAG_ERR_WORKSPACE;
+        if (!aligned16(ws) || !aligned16(fwd_ws)) return HAG_ERR_ALIGN;
+        if (ws == fwd_ws) return HAG_ERR_ARG;
+    }
+    DeviceScope scope(h->device);
+    if (!scope.ok) { cudaGetLastError(); return HAG_ERR_CUDA; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = dtype == HAG_F32
+             ? max_bwd<float>(h, use_hag, D, z, out, static_cast<const float *>(fwd_ws), g, gz, static_cast<float *>(ws), s)
+             : max_bwd<__nv_bfloat16>(h, use_hag, D, z, out, static_cast<const float *>(fwd_ws), g, gz, static_cast<float *>(ws), s);
+    if (st != HAG_OK) cudaGetLastError();
+    return st;
+}
+
+}  // namespace
+
+extern "C" size_t hag_max_workspace_bytes(const hag_t *h, int32_t D) {
+    if (!h || D <= 0) return 0;
+    return size_t(h->num_agg) * size_t(D) * sizeof(float);
+}
+
+extern "C" hag_status hag_max_fwd(const hag_t *h, hag_dtype dtype, int32_t D, const void *z, void *out, void *workspace,
+                                  void *cuda_stream) {
+    return run_fwd(h, true, dtype, D, z, out, workspace, cuda_stream);
+}
+
+extern "C" hag_status hag_max_bwd(const hag_t *h, hag_dtype dtype, int32_t D, const void *z, const void *out,
+                                  const void *fwd_workspace, const void *grad_out, void *grad_z, void *workspace,
+                                  void *cuda_stream) {
+    return run_bwd(h, true, dtype, D, z, out, fwd_workspace, grad_out, grad_z, workspace, cuda_stream);
+}
+
+extern "C" hag_status csr_max_fwd(const hag_t *h, hag_dtype dtype, int32_t D, const void *z, void *out, void *cuda_stream) {
+    return run_fwd(h, false, dtype, D, z, out, nullptr, cuda_stream);
+}
+
+extern "C" hag_status csr_max_bwd(const hag_t *h, hag_dtype dtype, int32_t D, const void *z, const void *out,
+                                  const void *grad_out, void *grad_z, void *cuda_stream) {
+    return run_bwd(h, false, dtype, D, z, out, nullptr, grad_out, grad_z, nullptr, cuda_stream);
+}
