@@ -197,6 +197,8 @@ def main():
                     help="also time capacities 0, N/8, N/4, N/2 from ONE search (hag_truncate); reported under capacity_sweep")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--max-leg", action="store_true",
+                    help="also time the element-wise max aggregation (hag_max_fwd/bwd against csr_max_fwd/bwd); reported under max_aggregation")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -438,6 +440,42 @@ def main():
                    "fwd_frac_of_measured_hbm": rb / (f_ms * 1e-3) / 1e9 / measured_peak()[0],
                    "bwd_frac_of_measured_hbm": rb / (b_ms * 1e-3) / 1e9 / measured_peak()[0]}
 
+    maxagg = None
+    if rank == 0 and args.max_leg:
+        # the max Aggregate of Table 1 (GraphSAGE-P) over the same HAG, against the same kernels on the plain graph
+        mo = torch.empty_like(x)
+        mg = torch.empty_like(x)
+        mws = [h.max_workspace(w.d, dev), h.max_workspace(w.d, dev)]
+
+        def max_step(use_hag):
+            h.max_fwd(x, out=mo, workspace=mws[0], use_hag=use_hag)
+            n_l = h.last_launch_count
+            h.max_bwd(x, mo, mws[0], gr, out=mg, workspace=mws[1], use_hag=use_hag)
+            return n_l + h.last_launch_count
+
+        res = {}
+        for use_hag in (True, False):
+            for _ in range(3):
+                max_step(use_hag)
+            ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(max(args.steps // 4, 5))]
+            torch.cuda.synchronize(dev)
+            for e3 in ev:
+                flush.zero_()
+                e3[0].record(stream)
+                h.max_fwd(x, out=mo, workspace=mws[0], use_hag=use_hag)
+                e3[1].record(stream)
+                h.max_bwd(x, mo, mws[0], gr, out=mg, workspace=mws[1], use_hag=use_hag)
+                e3[2].record(stream)
+            torch.cuda.synchronize(dev)
+            res[use_hag] = (float(np.mean([e3[0].elapsed_time(e3[1]) for e3 in ev])),
+                            float(np.mean([e3[1].elapsed_time(e3[2]) for e3 in ev])))
+        maxagg = {"what": "element-wise max aggregation, fwd and bwd timed apart, cold L2; forward bytes counted like the sum's",
+                  "hag_fwd_ms": res[True][0], "hag_bwd_ms": res[True][1], "plain_fwd_ms": res[False][0], "plain_bwd_ms": res[False][1],
+                  "hag_fwd_gbps": nbytes["hag_pass"] / (res[True][0] * 1e-3) / 1e9,
+                  "plain_fwd_gbps": nbytes["plain_pass"] / (res[False][0] * 1e-3) / 1e9,
+                  "speedup_hag_vs_plain_fwd": res[False][0] / res[True][0],
+                  "speedup_hag_vs_plain_fwd_bwd": sum(res[False]) / sum(res[True])}
+
     if rank == 0:
         bytes_step = 2 * w.layers * nbytes["hag_pass"]
         value = world * bytes_step / (hag_ms * 1e-3) / 1e9
@@ -482,6 +520,8 @@ def main():
             line["capacity_sweep"] = sweep
         if readout is not None:
             line["graph_readout"] = readout
+        if maxagg is not None:
+            line["max_aggregation"] = maxagg
         if w.dtype == "bf16":
             line["dtype"] = "f32 accumulate, bf16 storage"
         print(json.dumps(line))

@@ -137,3 +137,10 @@ def test_argument_errors():
     host_only = hb.Hag.build(w.graph.row_ptr, w.graph.col_idx, w.capacity)
     assert lib.csr_max_fwd(host_only._h, 0, 16, vp(z.data_ptr()), vp(o.data_ptr()), None) == hb.HAG_ERR_NOT_ON_DEVICE
     torch.cuda.synchronize()
+
+
+def test_full_size_clustered_workload():
+    """The 50 000-node clustered workload at full size, fp32, D = 64: every element of the forward result
+    and of the gradient against the oracle."""
+    w = synth.workload(2)
+    _check(w.graph, w.capacity, w.d, "f32", seed=w.seed)
