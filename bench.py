@@ -197,6 +197,8 @@ def main():
                     help="also time capacities 0, N/8, N/4, N/2 from ONE search (hag_truncate); reported under capacity_sweep")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--permute-ids", action="store_true",
+                    help="relabel the nodes by a seeded random permutation first (locality stress: communities no longer contiguous)")
     ap.add_argument("--max-leg", action="store_true",
                     help="also time the element-wise max aggregation (hag_max_fwd/bwd against csr_max_fwd/bwd); reported under max_aggregation")
     args = ap.parse_args()
@@ -237,6 +239,8 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     w = synth.workload(args.workload, scale=args.scale, capacity_frac=args.capacity_frac)
+    if args.permute_ids:
+        w.graph = synth.permute_ids(w.graph, seed=w.seed + 77)
     g = w.graph
     t0 = time.perf_counter()
     h = hb.Hag.build(g.row_ptr, g.col_idx, w.capacity, min_redundancy=args.min_redundancy).to_device(local_rank)
@@ -512,7 +516,7 @@ def main():
             "roofline": {"bound": "hbm", "kernel": "gather_sum_kernel (forward gather over the residual rows)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_kind": f"{peak_kind} copy bandwidth",
-                         "traffic": NCU_DRAM_BYTES_FWD_GATHER.get(w.name) if args.scale == 1.0 else None,
+                         "traffic": NCU_DRAM_BYTES_FWD_GATHER.get(w.name) if (args.scale == 1.0 and not args.permute_ids) else None,
                          "algorithmic_bytes_per_launch": nbytes["fwd_gather"], "ms_per_launch": fg_ms},
             "cpu_baseline": cpu,
         }
