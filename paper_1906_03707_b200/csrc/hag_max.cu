@@ -56,15 +56,37 @@ struct PairMaxArgs {
     int32_t n, D;
 };
 
-constexpr int kMaxLoads = 4;        // forward: row loads in flight per lane
-constexpr int kGradEntries = 2;     // backward: entries in flight per lane (two loads each)
+// Launch shapes from a sweep on B200 (loads or entries in flight per lane, resident CTAs per SM):
+// more resident warps beat more loads per warp, as for the sum kernels.
+//   fp32: forward 4 loads x 10 CTAs, backward 2 entries x 10 CTAs; bf16: forward 2 x 10, backward 1 x 8.
+#ifndef HAG_MAX_SHAPES
+#define HAG_MAX_SHAPES 4, 10, 2, 10, 2, 10, 1, 8
+#endif
+#ifdef HAG_MS0      // tuning builds: the eight numbers one by one
+#undef HAG_MAX_SHAPES
+#define HAG_MAX_SHAPES HAG_MS0, HAG_MS1, HAG_MS2, HAG_MS3, HAG_MS4, HAG_MS5, HAG_MS6, HAG_MS7
+#endif
+template <typename T> struct MaxShape;
+template <int FL, int FB, int BE, int BB, int HFL, int HFB, int HBE, int HBB> struct MaxShapeTable {
+    static constexpr int f32[4] = {FL, FB, BE, BB};
+    static constexpr int bf16[4] = {HFL, HFB, HBE, HBB};
+};
+using MaxShapes = MaxShapeTable<HAG_MAX_SHAPES>;
+template <> struct MaxShape<float> {
+    static constexpr int kFwdLoads = MaxShapes::f32[0], kFwdBlocks = MaxShapes::f32[1];
+    static constexpr int kBwdEntries = MaxShapes::f32[2], kBwdBlocks = MaxShapes::f32[3];
+};
+template <> struct MaxShape<__nv_bfloat16> {
+    static constexpr int kFwdLoads = MaxShapes::bf16[0], kFwdBlocks = MaxShapes::bf16[1];
+    static constexpr int kBwdEntries = MaxShapes::bf16[2], kBwdBlocks = MaxShapes::bf16[3];
+};
 
 template <typename T, int LPR>
-__global__ void __launch_bounds__(kThreads) gather_max_kernel(const MaxArgs a) {
+__global__ void __launch_bounds__(kThreads, MaxShape<T>::kFwdBlocks) gather_max_kernel(const MaxArgs a) {
     hagk::pdl_launch_dependents();
     constexpr int E = Chunk<T>::kElems;
     constexpr int G = 32 / LPR;
-    constexpr int U = kMaxLoads < LPR ? kMaxLoads : LPR;
+    constexpr int U = MaxShape<T>::kFwdLoads < LPR ? MaxShape<T>::kFwdLoads : LPR;
     const int lane = threadIdx.x & 31;
     const int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
     if (r_local >= a.row_count) return;
@@ -149,11 +171,11 @@ __global__ void __launch_bounds__(kThreads) pair_max_kernel(const PairMaxArgs p)
 
 // grad_s[k] = sum over the destinations t of row s with max_t[k] == value_s[k] of grad_t[k].
 template <typename T, int LPR>
-__global__ void __launch_bounds__(kThreads) gather_maxgrad_kernel(const MaxArgs a) {
+__global__ void __launch_bounds__(kThreads, MaxShape<T>::kBwdBlocks) gather_maxgrad_kernel(const MaxArgs a) {
     hagk::pdl_launch_dependents();
     constexpr int E = Chunk<T>::kElems;
     constexpr int G = 32 / LPR;
-    constexpr int U = kGradEntries < LPR ? kGradEntries : LPR;
+    constexpr int U = MaxShape<T>::kBwdEntries < LPR ? MaxShape<T>::kBwdEntries : LPR;
     const int lane = threadIdx.x & 31;
     const int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
     if (r_local >= a.row_count) return;
