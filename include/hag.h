@@ -133,7 +133,8 @@ typedef struct hag_arrays {
  *   32768 * (launches) + sum over deep nodes of (expanded inputs - 1),
  * ties to the larger c; c = num_levels means no expansion.  The backward pass
  * has its own cut: nodes deeper than it gather straight from the graph-node
- * outputs that use them (transitively), cost term (expanded users - direct users).
+ * outputs that use them (transitively), 131072 per launch, cost term (expanded
+ * users - direct users).
  * Host only; the input arrays are read during the call and not kept.
  * Errors: HAG_ERR_NULL; HAG_ERR_ARG (n < 0, capacity < 0, n + capacity or |E| >=
  * 2^31); HAG_ERR_GRAPH; HAG_ERR_OOM_HOST.  On error *out is NULL. */

@@ -344,7 +344,8 @@ def canonical_hag(row_ptr, search: SearchResult) -> CanonicalHag:
     return CanonicalHag(n, k, num_levels, level_ptr, agg_in, res_ptr, res_idx, t_ptr, t_idx, in_degree, c2c)
 
 
-LAUNCH_ROWS = 32768  # what the layout rule charges for one kernel launch, in rows moved
+LAUNCH_ROWS = 32768       # what the layout rule charges for one forward kernel launch, in rows moved
+BWD_LAUNCH_ROWS = 131072  # the same for a backward launch
 
 
 def expanded_tails(h: CanonicalHag) -> dict:
@@ -355,7 +356,8 @@ def expanded_tails(h: CanonicalHag) -> dict:
     cover(v)); c minimises  LAUNCH_ROWS * (c + [some node is deeper than c])
     + sum over deep nodes of (expanded inputs - 1), ties to the larger c.
     Backward: a node deeper than the cut collects the gradient of every graph-node
-    output that uses it, directly or through deeper nodes; the cost term is
+    output that uses it, directly or through deeper nodes; a launch is charged
+    BWD_LAUNCH_ROWS there and the cost term is
     (transitive users - direct users)."""
     n, k, L = h.n, h.num_agg, h.num_levels
     level = np.zeros(n + k, dtype=np.int64)
@@ -388,10 +390,10 @@ def expanded_tails(h: CanonicalHag) -> dict:
             d = int(d)
             out.extend([d] if d < n else users[d])
         users[n + j] = sorted(out)
-    best = (LAUNCH_ROWS * L, L)
+    best = (BWD_LAUNCH_ROWS * L, L)
     for c in range(L - 1, -1, -1):
         extra = sum(len(users[n + j]) - int(h.t_ptr[n + j + 1] - h.t_ptr[n + j]) for j in range(int(h.level_ptr[c]), k))
-        cost = LAUNCH_ROWS * (c + 1) + extra
+        cost = BWD_LAUNCH_ROWS * (c + 1) + extra
         if cost < best[0]:
             best = (cost, c)
     bwd_cut = best[1]

@@ -406,7 +406,9 @@ hag_status hag_layout(hag *h, const std::vector<int32_t> &rows_store, const std:
         }
         // ---- deep levels in one launch: choose the cuts and expand ----
         {
-            const int64_t kLaunchRows = 32768;   // what one extra launch costs, in rows moved
+            // what one extra launch costs, in rows moved; measured on B200: the backward launches (rows of tens of
+            // users each) pay for a merge up to four times later than the forward ones (rows of two to eight inputs)
+            const int64_t kLaunchRows = 32768, kBwdLaunchRows = 131072;
             const int32_t L = max_level;
             std::vector<int32_t> clevel(k);      // level per canonical aggregation node
             for (int32_t l = 1; l <= L; ++l)
@@ -460,13 +462,13 @@ hag_status hag_layout(hag *h, const std::vector<int32_t> &rows_store, const std:
                 usz[j] = t;
             }
             int32_t best_b = L;
-            int64_t best_bcost = kLaunchRows * L;
+            int64_t best_bcost = kBwdLaunchRows * L;
             {
                 int64_t extra = 0;
                 for (int32_t c = L - 1; c >= 0; --c) {
                     for (int64_t j = h->level_ptr[c]; j < h->level_ptr[c + 1]; ++j)
                         extra += usz[j] - (h->t_ptr[n + j + 1] - h->t_ptr[n + j]);
-                    const int64_t cost = kLaunchRows * (c + 1) + extra;
+                    const int64_t cost = kBwdLaunchRows * (c + 1) + extra;
                     if (cost < best_bcost) { best_bcost = cost; best_b = c; }
                 }
             }
