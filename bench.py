@@ -171,7 +171,9 @@ def run_reference(args, w, bytes_per_step_fn):
         "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "sample": what},
+        "config": {"workload": f"{w.name}: {w.graph.name}, N={w.graph.n}, E={w.graph.e}, D={w.d}, {w.dtype} storage, {w.reduce}, "
+                               f"{w.layers} layer(s), fwd+bwd; the oracle evaluates the GNN-graph directly in fp64",
+                   "sample": what},
         "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": what},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
