@@ -34,7 +34,7 @@ if ROOT not in sys.path:
 METRIC = "HAG fwd+bwd aggregation GB/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE forward-gather launch, from ncu captures of this
 # program at the workload's full size (None: not captured)
-NCU_DRAM_BYTES_FWD_GATHER = {"cfg2": 23.36e6 + 0.04e6, "cfg4": 228.1e6 + 104.0e6}
+NCU_DRAM_BYTES_FWD_GATHER = {"cfg2": 23.40e6 + 0.02e6, "cfg4": 228.2e6 + 105.5e6}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 L2_FLUSH_BYTES = 256 << 20
