@@ -139,8 +139,9 @@ def test_argument_errors():
     torch.cuda.synchronize()
 
 
-def test_full_size_clustered_workload():
-    """The 50 000-node clustered workload at full size, fp32, D = 64: every element of the forward result
-    and of the gradient against the oracle."""
-    w = synth.workload(2)
+@pytest.mark.parametrize("index", [2, 4])
+def test_full_size_workloads(index):
+    """The 50 000-node clustered workload and the batch of 5 000 small graphs at full size, fp32, D = 64:
+    every element of the forward result and of the gradient against the oracle."""
+    w = synth.workload(index)
     _check(w.graph, w.capacity, w.d, "f32", seed=w.seed)
