@@ -8,7 +8,10 @@
  * (Section 5.1: graph_to_hag, hag_aggregate, hag_aggregate_grad) map to
  * hag_build, hag_aggregate_fwd and hag_aggregate_bwd; csr_aggregate_* evaluate
  * the plain GNN-graph (the special case V_A = {} of Section 3.1) with the same
- * kernels, as the comparison path.
+ * kernels, as the comparison path.  Beyond that core: hag_max_* / csr_max_* (the
+ * element-wise max Aggregate of Table 1's GraphSAGE-P row over the same HAG) and
+ * hag_graph_pool_* (the mean-pooling read-out of Section 5.1 over the graphs of
+ * a batch).
  *
  * Conventions
  *   ids        graph nodes 0..N-1; aggregation nodes N..N+|V_A|-1, sorted by level
