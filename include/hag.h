@@ -221,8 +221,15 @@ hag_status csr_aggregate_bwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype,
  * out_host are HOST pointers to N x D matrices (pinned memory makes the copies
  * asynchronous).  The call copies the input to device staging buffers owned by
  * the handle (grown on demand with cudaMalloc), runs the aggregation on
- * cuda_stream and copies the result back; it returns after enqueuing, so the
- * caller synchronises the stream before reading out_host.  `backward` != 0 runs
+ * cuda_stream and copies the result back on cuda_stream; it returns after
+ * enqueuing, so the caller synchronises the stream before reading out_host.
+ * The copy-in runs on a stream of the handle's own, into one of two buffers, so
+ * that the copy-in of a call overlaps the aggregation and the copy-out of the
+ * call before it (both directions of the host link are busy at once).  For that
+ * reason x_host must hold its data when the call is made (it is read without
+ * waiting for earlier work in cuda_stream) and must stay unchanged until the
+ * stream has been synchronised; consecutive calls on one handle must use the same
+ * cuda_stream or be separated by a synchronisation.  `backward` != 0 runs
  * hag_aggregate_bwd instead of hag_aggregate_fwd; `use_hag` == 0 runs the
  * csr_aggregate_* path. */
 hag_status hag_aggregate_host(hag_t *h, int backward, int use_hag, hag_reduce reduce, hag_dtype dtype, int32_t D,

@@ -59,8 +59,16 @@ void free_device(hag *h) {
         t->d_segs = t->d_slots = nullptr;
         t->d_done = nullptr;
     }
+    if (d.copy_in_stream) {
+        cudaStreamSynchronize(d.copy_in_stream);
+        cudaStreamDestroy(d.copy_in_stream);
+    }
+    for (int i = 0; i < 2; ++i) {
+        if (d.in_ready[i]) cudaEventDestroy(d.in_ready[i]);
+        if (d.in_free[i]) cudaEventDestroy(d.in_free[i]);
+    }
     void *ptrs[] = {d.agg_in, d.res_ptr, d.res_idx, d.t_ptr, d.t_idx, d.csr_ptr, d.csr_idx, d.csr_t_ptr,
-                    d.csr_t_idx, d.inv_degree, d.inv_degree1, d.stage_in, d.stage_out, d.stage_ws,
+                    d.csr_t_idx, d.inv_degree, d.inv_degree1, d.stage_in, d.stage_in2, d.stage_out, d.stage_ws,
                     d.ftail_ptr, d.ftail_idx, d.btail_ptr, d.btail_idx, d.sched};
     for (void *p : ptrs)
         if (p) cudaFree(p);
@@ -587,18 +595,36 @@ extern "C" hag_status hag_aggregate_host(hag_t *h, int backward, int use_hag, ha
     DeviceGuard guard(h->device);
     if (!guard.ok) { cudaGetLastError(); return HAG_ERR_CUDA; }
     hag_device_arrays &d = h->d;
-    hag_status st = grow(&d.stage_in, &d.stage_in_bytes, std::max<size_t>(bytes, 16));
+    // Pipeline over consecutive calls: the copy-in runs on a stream of the handle's own into one of two input
+    // buffers, so it overlaps the aggregation and the copy-out of the previous call (which stay on the caller's
+    // stream, where the caller waits for the result).  Events order the reuse of the two buffers.
+    if (!d.copy_in_stream) {
+        if (cudaStreamCreateWithFlags(&d.copy_in_stream, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); return HAG_ERR_CUDA; }
+        for (int i = 0; i < 2; ++i) {
+            if (cudaEventCreateWithFlags(&d.in_ready[i], cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&d.in_free[i], cudaEventDisableTiming) != cudaSuccess) { cudaGetLastError(); return HAG_ERR_CUDA; }
+        }
+    }
+    const uint32_t slot = d.host_calls & 1u;
+    void **in_buf = slot ? &d.stage_in2 : &d.stage_in;
+    size_t *in_have = slot ? &d.stage_in2_bytes : &d.stage_in_bytes;
+    hag_status st = grow(in_buf, in_have, std::max<size_t>(bytes, 16));
     if (st == HAG_OK) st = grow(&d.stage_out, &d.stage_out_bytes, std::max<size_t>(bytes, 16));
     if (st == HAG_OK)
         st = grow(&d.stage_ws, &d.stage_ws_bytes, std::max<size_t>(std::max(hag_workspace_bytes(h, D), csr_workspace_bytes(h, D)), 16));
     if (st != HAG_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    if (bytes && cudaMemcpyAsync(d.stage_in, in_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
-        cudaGetLastError();
-        return HAG_ERR_CUDA;
-    }
-    st = run(h, backward != 0, use_hag != 0, reduce, dtype, D, d.stage_in, d.stage_out, d.stage_ws, cuda_stream);
+    bool ok = true;
+    // the buffer is free once the aggregation of the call before last has read it
+    if (d.host_calls >= 2) ok = ok && cudaStreamWaitEvent(d.copy_in_stream, d.in_free[slot], 0) == cudaSuccess;
+    if (bytes) ok = ok && cudaMemcpyAsync(*in_buf, in_host, bytes, cudaMemcpyHostToDevice, d.copy_in_stream) == cudaSuccess;
+    ok = ok && cudaEventRecord(d.in_ready[slot], d.copy_in_stream) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(s, d.in_ready[slot], 0) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return HAG_ERR_CUDA; }
+    ++d.host_calls;
+    st = run(h, backward != 0, use_hag != 0, reduce, dtype, D, *in_buf, d.stage_out, d.stage_ws, cuda_stream);
     if (st != HAG_OK) return st;
+    if (cudaEventRecord(d.in_free[slot], s) != cudaSuccess) { cudaGetLastError(); return HAG_ERR_CUDA; }
     if (bytes && cudaMemcpyAsync(out_host, d.stage_out, bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) {
         cudaGetLastError();
         return HAG_ERR_CUDA;

@@ -54,11 +54,17 @@ struct hag_device_arrays {
     float *inv_degree = nullptr;   // [n] 1/|N(v)| (1 for empty rows)
     float *inv_degree1 = nullptr;  // [n] 1/(|N(v)| + 1): the GCN normalisation
     unsigned int *sched = nullptr; // ring of kSchedSlots (next row, finished warps) pairs, zero between launches
-    // staging for the host-buffer entry point
+    // staging for the host-buffer entry point: the input side is double-buffered and copied on a stream of its
+    // own, so that the copy-in of one call runs under the aggregation and the copy-out of the call before it
     void *stage_in = nullptr;
+    void *stage_in2 = nullptr;
     void *stage_out = nullptr;
     void *stage_ws = nullptr;
-    size_t stage_in_bytes = 0, stage_out_bytes = 0, stage_ws_bytes = 0;
+    size_t stage_in_bytes = 0, stage_in2_bytes = 0, stage_out_bytes = 0, stage_ws_bytes = 0;
+    cudaStream_t copy_in_stream = nullptr;
+    cudaEvent_t in_ready[2] = {nullptr, nullptr};   // copy-in into buffer i finished
+    cudaEvent_t in_free[2] = {nullptr, nullptr};    // the aggregation that read buffer i finished
+    uint32_t host_calls = 0;
 };
 
 struct hag {

@@ -279,6 +279,28 @@ def test_host_buffer_entry_point_matches_device_path():
             assert torch.equal(out.cuda(), fn(x.cuda(), "mean"))
 
 
+def test_host_buffer_calls_back_to_back_do_not_mix_their_buffers():
+    """Consecutive host-buffer calls overlap (the copy-in of one runs under the aggregation and the copy-out of
+    the one before, through two input buffers): a run of calls with different inputs, widths and directions,
+    synchronised only at the end, must give what the device entry points give for each of them."""
+    w, h = _case("cfg2-small")
+    n = w.graph.n
+    calls = []
+    for i in range(9):
+        d = (64, 32, 128)[i % 3]
+        x = torch.from_numpy(synth.features(20 + i, n, d, "normal")).pin_memory()
+        out = torch.full((n, d), float("nan")).pin_memory()
+        calls.append((x, out, bool(i % 2), i % 4 != 3))
+    for _ in range(3):
+        for x, out, backward, use_hag in calls:
+            h.aggregate_host(x, out, "mean", backward=backward, use_hag=use_hag)
+    torch.cuda.synchronize()
+    for x, out, backward, use_hag in calls:
+        fn = {(False, True): h.aggregate_fwd, (True, True): h.aggregate_bwd,
+              (False, False): h.csr_fwd, (True, False): h.csr_bwd}[(backward, use_hag)]
+        assert torch.equal(out.cuda(), fn(x.cuda(), "mean"))
+
+
 def test_device_call_errors_are_statuses():
     w, h = _case("cfg1")
     lib = hb.load_library()
