@@ -24,6 +24,18 @@ def shard_range(n_units: int, rank: int, world: int):
     return first, base + (1 if rank < extra else 0)
 
 
+def shard_columns(d: int, rank: int, world: int, elem_bytes: int = 4):
+    """Feature-column split of one graph over ranks: (first column, count) for ``rank``.
+    Aggregation treats every column alike, so each rank can hold the whole structure and
+    a slice of the columns of x and needs no exchange.  Slices are multiples of 16 bytes
+    (the kernels' row granularity); ranks at the end may get nothing when D is small."""
+    if d <= 0 or (d * elem_bytes) % 16:
+        raise ValueError("row size must be a positive multiple of 16 bytes")
+    per16 = 16 // elem_bytes if elem_bytes <= 16 else 1
+    first, count = shard_range(d // per16, rank, world)
+    return first * per16, count * per16
+
+
 def shard_block_diagonal(g: Graph, graph_size: int, rank: int, world: int) -> Graph:
     """The sub-batch of a block-diagonal batch of equal-size graphs owned by ``rank``,
     re-indexed from 0.  Raises if an edge leaves its block (the batch would not be

@@ -86,3 +86,23 @@ def test_two_gloo_ranks_tile_the_batch(tmp_path):
     got_b = np.concatenate([np.load(tmp_path / f"gx{r}.npy") for r in range(world)])
     np.testing.assert_allclose(got, want, rtol=0, atol=1e-12)
     np.testing.assert_allclose(got_b, want_b, rtol=0, atol=1e-12)
+
+
+def test_column_slices_tile_the_features_and_need_no_exchange():
+    for d, eb, world in ((64, 4, 2), (64, 4, 3), (20, 4, 8), (256, 2, 8), (8, 2, 4)):
+        parts = [sharding.shard_columns(d, r, world, eb) for r in range(world)]
+        assert parts[0][0] == 0 and sum(c for _, c in parts) == d
+        for (f0, c0), (f1, _) in zip(parts, parts[1:]):
+            assert f1 == f0 + c0
+        assert all((c * eb) % 16 == 0 and (f * eb) % 16 == 0 for f, c in parts)
+    with pytest.raises(ValueError):
+        sharding.shard_columns(6, 0, 2, 4)
+    # every rank aggregates its own columns over the whole graph; side by side they are the full result
+    g = synth.config1_graph()
+    x = synth.features(5, g.n, 24, "normal").astype(np.float64)
+    want, _ = O.direct_forward(g.row_ptr, g.col_idx, x, "mean")
+    got = []
+    for r in range(3):
+        f, c = sharding.shard_columns(24, r, 3, 4)
+        got.append(O.direct_forward(g.row_ptr, g.col_idx, np.ascontiguousarray(x[:, f:f + c]), "mean")[0])
+    np.testing.assert_array_equal(np.concatenate(got, axis=1), want)
