@@ -726,3 +726,189 @@ done:
     free(out); free(out_store); free(bound); free(count); free(touched); free(users); free(hp.e);
     return rc < 0 ? rc : num_agg;
 }
+
+/* ------------------------------------------------------------------------- */
+/* Replay of a recorded run of Algorithm 3 from the Redundancy definition, at any
+ * size.  Independent of how the trace was found: no bounds, no heap, no pair map.
+ *
+ * State: the current rows (the edge set E-hat of Algorithm 3, graph-node rows
+ * only, sorted) and, per node s, a candidate list cand(s) of rows that MAY hold s.
+ * The rows are the authority; cand(s) only narrows which rows are looked at.  It is
+ * a superset of the holders of s at all times: a graph node enters rows only in
+ * the input graph (cand = its out-neighbours there), an aggregation node w only at
+ * its creation (cand = the rows rewritten then), and entries are never added to
+ * a row otherwise.
+ *
+ * Before merge i (recorded v1 < v2, redundancy r):
+ *   - Redundancy(v1, v2) = number of rows that contain both, counted by testing
+ *     every row of cand(v1); it must equal r, and r must be >= min_redundancy;
+ *   - if i is one of check_steps: Redundancy of EVERY pair is recounted (for each
+ *     node a, over the rows that hold a, one count per larger member b) and the
+ *     recorded pair must be the largest, ties to the smallest v1 and then the
+ *     smallest v2 (aggregation nodes numbered n, n+1, ... in creation order).
+ * Then the rewrite of the algorithm's inner loop is applied: each such row loses v1
+ * and v2 and gains w = n + i.
+ * A check step equal to k (after the last merge) recounts every pair once more
+ * and reports the largest redundancy that is left.
+ *
+ * report[0] = -1 when everything held, else the step that failed;
+ * report[1] = what failed (1 bad pair ids, 2 redundancy differs, 3 below the stop
+ *             value, 4 another pair is larger or earlier, 5 out of memory);
+ * report[2] = largest redundancy left after the last merge (-1 if k was not a check step);
+ * report[3] = full recounts done; report[4] = pair-count updates they made;
+ * report[5], report[6], report[7] = on code 2: recount; on code 4: the arg-max pair and its redundancy.
+ * cur_len / cur_idx receive the final rows laid over row_ptr.                     */
+static int32_t row_pos(const int32_t *row, int32_t len, int32_t key)
+{
+    int32_t lo = 0, hi = len;
+    while (lo < hi) {
+        int32_t mid = lo + (hi - lo) / 2;
+        if (row[mid] < key) lo = mid + 1; else hi = mid;
+    }
+    return (lo < len && row[lo] == key) ? lo : -1;
+}
+
+static void recount_all_pairs(int64_t n, int64_t n_ids, const int64_t *row_ptr, const int32_t *cur_len,
+                              const int32_t *cur_idx, int32_t *const *cand, const int32_t *cand_len,
+                              int32_t *count, int32_t *touched, int64_t *best_out, int32_t *a_out, int32_t *b_out,
+                              int64_t *updates)
+{
+    int64_t best = 0;
+    int32_t ba = -1, bb = -1;
+    (void)n;
+    for (int64_t a = 0; a < n_ids; ++a) {
+        int32_t nt = 0;
+        for (int32_t q = 0; q < cand_len[a]; ++q) {
+            int32_t u = cand[a][q];
+            const int32_t *row = cur_idx + row_ptr[u];
+            int32_t p = row_pos(row, cur_len[u], (int32_t)a);
+            if (p < 0) continue;
+            for (int32_t i = p + 1; i < cur_len[u]; ++i) {      /* members b > a of a row that holds a */
+                int32_t b = row[i];
+                if (count[b]++ == 0) touched[nt++] = b;
+            }
+            *updates += cur_len[u] - p - 1;
+        }
+        int64_t loc = 0;
+        int32_t lb = -1;
+        for (int32_t t = 0; t < nt; ++t) {
+            int32_t b = touched[t], c = count[b];
+            count[b] = 0;
+            if (c > loc || (c == loc && b < lb)) { loc = c; lb = b; }
+        }
+        if (loc > best) { best = loc; ba = (int32_t)a; bb = lb; }   /* strictly larger only: the smallest a wins ties */
+    }
+    *best_out = best; *a_out = ba; *b_out = bb;
+}
+
+int64_t o_replay_trace(int64_t n, const int64_t *row_ptr, const int32_t *col, int64_t k,
+                       const int32_t *t1, const int32_t *t2, const int32_t *tr, int32_t min_redundancy,
+                       int64_t n_checks, const int64_t *check_steps,
+                       int32_t *cur_len, int32_t *cur_idx, int64_t *report)
+{
+    int64_t E = row_ptr[n], n_ids = n + k, rc = 0, next_check = 0;
+    int64_t extra = 0;
+    for (int64_t i = 0; i < k; ++i) extra += tr[i] > 0 ? tr[i] : 0;
+    int32_t **cand = (int32_t **)calloc((size_t)(n_ids > 0 ? n_ids : 1), sizeof(int32_t *));
+    int32_t *cand_len = (int32_t *)calloc((size_t)(n_ids > 0 ? n_ids : 1), sizeof(int32_t));
+    int32_t *store = (int32_t *)malloc(sizeof(int32_t) * (size_t)(E + extra + 1));
+    int32_t *count = (int32_t *)calloc((size_t)(n_ids > 0 ? n_ids : 1), sizeof(int32_t));
+    int32_t *touched = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n_ids > 0 ? n_ids : 1));
+    for (int j = 0; j < 8; ++j) report[j] = -1;
+    report[3] = 0; report[4] = 0;
+    if (!cand || !cand_len || !store || !count || !touched) { report[0] = 0; report[1] = 5; rc = -1; goto done; }
+    memcpy(cur_idx, col, sizeof(int32_t) * (size_t)E);
+    for (int64_t u = 0; u < n; ++u) cur_len[u] = (int32_t)(row_ptr[u + 1] - row_ptr[u]);
+    {
+        int64_t *fill = (int64_t *)calloc((size_t)n + 1, sizeof(int64_t));
+        if (!fill) { report[0] = 0; report[1] = 5; rc = -1; goto done; }
+        for (int64_t e = 0; e < E; ++e) fill[col[e] + 1]++;
+        for (int64_t s = 0; s < n; ++s) fill[s + 1] += fill[s];
+        for (int64_t s = 0; s < n; ++s) cand[s] = store + fill[s];
+        for (int64_t u = 0; u < n; ++u)
+            for (int64_t e = row_ptr[u]; e < row_ptr[u + 1]; ++e) { int32_t s = col[e]; cand[s][cand_len[s]++] = (int32_t)u; }
+        free(fill);
+    }
+    int32_t *free_store = store + E;
+    for (int64_t i = 0; i <= k; ++i) {
+        int check = 0;
+        while (next_check < n_checks && check_steps[next_check] < i) ++next_check;
+        if (next_check < n_checks && check_steps[next_check] == i) check = 1;
+        if (check) {
+            int64_t best; int32_t a, b;
+            recount_all_pairs(n, n + i, row_ptr, cur_len, cur_idx, cand, cand_len, count, touched, &best, &a, &b, &report[4]);
+            report[3]++;
+            if (i == k) { report[2] = best; break; }
+            if (best != tr[i] || a != t1[i] || b != t2[i]) {
+                report[0] = i; report[1] = 4; report[5] = a; report[6] = b; report[7] = best; rc = -1; goto done;
+            }
+        }
+        if (i == k) break;
+        int32_t v1 = t1[i], v2 = t2[i], r = tr[i], w = (int32_t)(n + i);
+        if (!(0 <= v1 && v1 < v2 && v2 < w)) { report[0] = i; report[1] = 1; rc = -1; goto done; }
+        if (r < min_redundancy) { report[0] = i; report[1] = 3; rc = -1; goto done; }
+        /* Redundancy(v1, v2): rows holding both; every row that holds v1 is in cand(v1) */
+        int32_t nu = 0;
+        int32_t *users = free_store;
+        for (int32_t q = 0; q < cand_len[v1]; ++q) {
+            int32_t u = cand[v1][q];
+            const int32_t *row = cur_idx + row_ptr[u];
+            if (row_pos(row, cur_len[u], v1) >= 0 && row_pos(row, cur_len[u], v2) >= 0) {
+                if (nu < r) users[nu] = u;
+                ++nu;
+            }
+        }
+        if (nu != r) { report[0] = i; report[1] = 2; report[5] = nu; rc = -1; goto done; }
+        for (int32_t q = 0; q < nu; ++q) {                       /* E-hat <- E-hat - (v1,u) - (v2,u) + (w,u) */
+            int32_t u = users[q];
+            int32_t *row = cur_idx + row_ptr[u];
+            int32_t len = cur_len[u], o = 0;
+            for (int32_t j = 0; j < len; ++j) if (row[j] != v1 && row[j] != v2) row[o++] = row[j];
+            row[o++] = w;                                        /* w is the largest id so far: the row stays sorted */
+            cur_len[u] = o;
+        }
+        cand[w] = users; cand_len[w] = nu;
+        free_store += nu;
+    }
+done:
+    free(cand); free(cand_len); free(store); free(count); free(touched);
+    return rc;
+}
+
+/* Theorem 2's condition on rows in creation-id space: expanding every aggregation
+ * node of row u into its two inputs (t1, t2) until only graph nodes remain must
+ * give N(u) of the input graph, every source exactly once.  Returns -1 when all
+ * rows pass, else the first row that does not.                                 */
+static int cmp_i32(const void *a, const void *b)
+{
+    int32_t x = *(const int32_t *)a, y = *(const int32_t *)b;
+    return (x > y) - (x < y);
+}
+
+int64_t o_cover_check(int64_t n, const int64_t *row_ptr, const int32_t *col, int64_t k,
+                      const int32_t *t1, const int32_t *t2, const int32_t *cur_len, const int32_t *cur_idx)
+{
+    int64_t max_deg = 0, bad = -1;
+    (void)k;
+    for (int64_t u = 0; u < n; ++u) if (row_ptr[u + 1] - row_ptr[u] > max_deg) max_deg = row_ptr[u + 1] - row_ptr[u];
+    int32_t *leaves = (int32_t *)malloc(sizeof(int32_t) * (size_t)(max_deg + 1));
+    int32_t *stack = (int32_t *)malloc(sizeof(int32_t) * (size_t)(max_deg + 2));
+    if (!leaves || !stack) { free(leaves); free(stack); return -2; }
+    for (int64_t u = 0; u < n && bad < 0; ++u) {
+        int64_t deg = row_ptr[u + 1] - row_ptr[u], nl = 0, ns = 0;
+        if (cur_len[u] > deg) { bad = u; break; }
+        for (int32_t i = 0; i < cur_len[u]; ++i) stack[ns++] = cur_idx[row_ptr[u] + i];
+        while (ns > 0 && bad < 0) {
+            int32_t s = stack[--ns];
+            if (s < n) { leaves[nl++] = s; }
+            else { stack[ns++] = t1[s - n]; stack[ns++] = t2[s - n]; }
+            if (nl + ns > deg) bad = u;              /* more sources than N(u) has: stop before the buffers overflow */
+        }
+        if (bad >= 0) break;
+        if (nl != deg) { bad = u; break; }
+        qsort(leaves, (size_t)nl, sizeof(int32_t), cmp_i32);
+        for (int64_t j = 0; j < nl; ++j) if (leaves[j] != col[row_ptr[u] + j]) { bad = u; break; }
+    }
+    free(leaves); free(stack);
+    return bad;
+}

@@ -22,7 +22,13 @@ What it computes, and where the paper (arxiv 1906.03707) defines it:
   layout, fp64.
 * ``cover_multiset_ok``, ``counters``, ``replay_trace`` -- Theorem 2's condition,
   the cost function of Section 4.1 in both forms, f = |E| - |E-hat| + |V_A| of
-  the Theorem 4 proof, and a from-the-definition replay of a merge trace.
+  the Theorem 4 proof, and a from-the-definition replay of a merge trace;
+  ``replay_trace_full`` / ``cover_check_rows`` -- the same two checks in plain C,
+  for the full-size workload shapes.
+* ``expanded_tails`` / ``expanded_forward`` -- for GIVEN cuts, the cover-restricted
+  input lists (Section 3.1, Eq. 1) and transitive users of the deep levels.  The
+  choice of a cut is a launch heuristic of whoever evaluates the HAG; the paper
+  fixes nothing about it, so nothing here chooses one.
 
 * ``graph_pool_forward`` / ``graph_pool_backward`` -- the mean-pooling layer that the
   experimental setup (Section 5.1) puts after the GNN layers for graph
@@ -100,6 +106,10 @@ def _c():
         lib.o3b_greedy.restype = i64
         lib.o3c_greedy.argtypes = [i64, p, p, i64, i32, p, p, p, p, p, p]
         lib.o3c_greedy.restype = i64
+        lib.o_replay_trace.argtypes = [i64, p, p, i64, p, p, p, i32, i64, p, p, p, p]
+        lib.o_replay_trace.restype = i64
+        lib.o_cover_check.argtypes = [i64, p, p, i64, p, p, p, p]
+        lib.o_cover_check.restype = i64
         _lib = lib
     return _lib
 
@@ -344,59 +354,43 @@ def canonical_hag(row_ptr, search: SearchResult) -> CanonicalHag:
     return CanonicalHag(n, k, num_levels, level_ptr, agg_in, res_ptr, res_idx, t_ptr, t_idx, in_degree, c2c)
 
 
-LAUNCH_ROWS = 32768       # what the layout rule charges for one forward kernel launch, in rows moved
-BWD_LAUNCH_ROWS = 131072  # the same for a backward launch
+def expanded_tails(h: CanonicalHag, fwd_cut: int, bwd_cut: int) -> dict:
+    """Deep levels evaluated without their intermediate nodes, for GIVEN cuts.
 
-
-def expanded_tails(h: CanonicalHag) -> dict:
-    """The layout's treatment of deep levels, restated from its rule.
-
-    Forward: with a cut c, an aggregation node deeper than level c is the sum over
-    its cover restricted to ids of level <= c (Section 3.1: aggr(v) aggregates
-    cover(v)); c minimises  LAUNCH_ROWS * (c + [some node is deeper than c])
-    + sum over deep nodes of (expanded inputs - 1), ties to the larger c.
-    Backward: a node deeper than the cut collects the gradient of every graph-node
-    output that uses it, directly or through deeper nodes; a launch is charged
-    BWD_LAUNCH_ROWS there and the cost term is
-    (transitive users - direct users)."""
+    Forward, cut c (0 <= c <= L): an aggregation node deeper than level c is the
+    Aggregate over its cover restricted to ids of level <= c, i.e. its inputs with
+    every input deeper than c replaced, recursively, by that input's own list
+    (Section 3.1, Eq. 1: aggr(v) aggregates cover(v); with c = 0 the list IS
+    cover(v)).  Backward, cut c: a node deeper than c collects the gradient of
+    every graph-node output that uses it, directly or through deeper nodes (the
+    transitive users over the transposed HAG).  Which cut a library picks is a
+    launch heuristic that the paper does not fix: every cut gives the same values,
+    so the cut is an input here and only the lists are derived.  Lists are sorted;
+    a source reached along several paths would appear several times (it never
+    does when the cover condition of Theorem 2 holds)."""
     n, k, L = h.n, h.num_agg, h.num_levels
+    if not (0 <= fwd_cut <= L and 0 <= bwd_cut <= L):
+        raise ValueError("cut outside 0..num_levels")
     level = np.zeros(n + k, dtype=np.int64)
     for l in range(1, L + 1):
         level[n + h.level_ptr[l - 1]: n + h.level_ptr[l]] = l
     pairs = h.agg_in.reshape(-1, 2)
 
-    def fwd_lists(c):
-        lists = {}
-        for j in range(int(h.level_ptr[c]), k):
-            out = []
-            for s in pairs[j]:
-                s = int(s)
-                out.extend([s] if level[s] <= c else lists[s])
-            lists[n + j] = sorted(out)
-        return lists
-
-    best = (LAUNCH_ROWS * L, L)
-    for c in range(L - 1, -1, -1):
-        cost = LAUNCH_ROWS * (c + 1) + sum(len(v) - 1 for v in fwd_lists(c).values())
-        if cost < best[0]:
-            best = (cost, c)
-    fwd_cut = best[1]
-    fl = fwd_lists(fwd_cut)
+    fl = {}
+    for j in range(int(h.level_ptr[fwd_cut]), k):
+        out = []
+        for s in pairs[j]:
+            s = int(s)
+            out.extend([s] if level[s] <= fwd_cut else fl[s])
+        fl[n + j] = sorted(out)
 
     users = {}
-    for j in range(k - 1, -1, -1):
+    for j in range(k - 1, int(h.level_ptr[bwd_cut]) - 1, -1):
         out = []
         for d in h.t_idx[h.t_ptr[n + j]: h.t_ptr[n + j + 1]]:
             d = int(d)
             out.extend([d] if d < n else users[d])
         users[n + j] = sorted(out)
-    best = (BWD_LAUNCH_ROWS * L, L)
-    for c in range(L - 1, -1, -1):
-        extra = sum(len(users[n + j]) - int(h.t_ptr[n + j + 1] - h.t_ptr[n + j]) for j in range(int(h.level_ptr[c]), k))
-        cost = BWD_LAUNCH_ROWS * (c + 1) + extra
-        if cost < best[0]:
-            best = (cost, c)
-    bwd_cut = best[1]
 
     def pack(ids, lists):
         ptr = np.zeros(len(ids) + 1, dtype=np.int64)
@@ -412,6 +406,26 @@ def expanded_tails(h: CanonicalHag) -> dict:
     btail_ptr, btail_idx = pack(b_ids, users)
     return dict(fwd_cut=fwd_cut, bwd_cut=bwd_cut, ftail_ptr=ftail_ptr, ftail_idx=ftail_idx,
                 btail_ptr=btail_ptr, btail_idx=btail_idx)
+
+
+def expanded_forward(h: CanonicalHag, x, fwd_cut: int, tails: dict):
+    """Algorithm 2 lines 3-6 with the deep levels taken from the given expansion lists:
+    levels 1..fwd_cut as pair sums, every deeper node as the sum over its list.  Returns
+    the (n + num_agg) x d buffer of a-hat values (fp64); it must equal what the plain level
+    order gives, which is how a set of lists from anywhere is checked for validity."""
+    x = np.asarray(x, dtype=np.float64)
+    n, k = h.n, h.num_agg
+    ahat = np.zeros((n + k, x.shape[1]), dtype=np.float64)
+    ahat[:n] = x
+    j0 = int(h.level_ptr[fwd_cut])
+    for j in range(j0):
+        ahat[n + j] = ahat[h.agg_in[2 * j]] + ahat[h.agg_in[2 * j + 1]]
+    ptr, idx = tails["ftail_ptr"], tails["ftail_idx"]
+    deep = np.zeros((k - j0, x.shape[1]), dtype=np.float64)
+    for i in range(k - j0):
+        deep[i] = ahat[idx[ptr[i]:ptr[i + 1]]].sum(axis=0)      # all ids in a list are of level <= fwd_cut
+    ahat[n + j0:] = deep
+    return ahat
 
 
 def transposed_csr(row_ptr, col_idx):
@@ -591,3 +605,46 @@ def replay_trace(row_ptr, col_idx, trace, check_argmax_at=()):
         final, _ = global_argmax(n + k)
     rows = [cur_idx[rp[u]:rp[u] + cur_len[u]].copy() for u in range(n)]
     return rows, final
+
+
+def replay_trace_full(row_ptr, col_idx, trace, check_argmax_at=(), min_redundancy=2):
+    """The same replay in plain C (oracle.c: o_replay_trace), for traces of any length.
+
+    Before every merge the recorded redundancy is recounted from the definition over the
+    current rows; at the steps in ``check_argmax_at`` every pair's redundancy is recounted
+    and the recorded pair must be the arg-max with the lowest-pair-id tie-break; a step equal
+    to the number of merges recounts once more after the last merge.  Returns a dict:
+    ok, failed_step, failure, rows (list of arrays, creation ids), final_max_redundancy
+    (None unless the terminal recount was asked for), full_recounts, pair_count_updates."""
+    rp, ci = _csr(row_ptr, col_idx)
+    n = rp.shape[0] - 1
+    tr = np.ascontiguousarray(np.asarray(trace, dtype=np.int32).reshape(-1, 3))
+    k = tr.shape[0]
+    t1, t2, r = (np.ascontiguousarray(tr[:, j]) for j in range(3))
+    steps = np.asarray(sorted(set(int(s) for s in check_argmax_at)), dtype=np.int64)
+    cur_len = np.zeros(max(n, 1), dtype=np.int32)
+    cur_idx = np.zeros(max(ci.shape[0], 1), dtype=np.int32)
+    report = np.zeros(8, dtype=np.int64)
+    _c().o_replay_trace(n, _ptr(rp), _ptr(ci), k, _ptr(t1), _ptr(t2), _ptr(r), int(min_redundancy),
+                        steps.shape[0], _ptr(steps), _ptr(cur_len), _ptr(cur_idx), _ptr(report))
+    what = {1: "bad pair ids", 2: "recorded redundancy differs from the recount", 3: "merge below the stop value",
+            4: "another pair has a larger redundancy or comes first", 5: "out of memory"}
+    ok = report[0] < 0
+    return dict(ok=bool(ok), failed_step=None if ok else int(report[0]), failure=None if ok else what[int(report[1])],
+                detail=[int(v) for v in report[5:8]],
+                rows=[cur_idx[rp[u]:rp[u] + cur_len[u]].copy() for u in range(n)] if ok else None,
+                row_len=cur_len[:n].copy(), row_store=cur_idx,
+                final_max_redundancy=None if report[2] < 0 else int(report[2]),
+                full_recounts=int(report[3]), pair_count_updates=int(report[4]))
+
+
+def cover_check_rows(row_ptr, col_idx, trace, row_len, row_store) -> int:
+    """Theorem 2 on rows in creation-id space (oracle.c: o_cover_check): every row, with its
+    aggregation nodes expanded down to graph nodes, must be N(u) of the input graph with every
+    source exactly once.  Returns -1 when all rows pass, else the first failing row."""
+    rp, ci = _csr(row_ptr, col_idx)
+    tr = np.asarray(trace, dtype=np.int32).reshape(-1, 3)
+    t1, t2 = np.ascontiguousarray(tr[:, 0]), np.ascontiguousarray(tr[:, 1])
+    rl = np.ascontiguousarray(row_len, dtype=np.int32)
+    rs = np.ascontiguousarray(row_store, dtype=np.int32)
+    return int(_c().o_cover_check(rp.shape[0] - 1, _ptr(rp), _ptr(ci), tr.shape[0], _ptr(t1), _ptr(t2), _ptr(rl), _ptr(rs)))

@@ -177,6 +177,27 @@ def test_pairmap_equals_bruteforce_on_tiny_graphs(seed):
         assert fin == b.final_max_redundancy
         if k < cap:
             assert fin <= 1
+        # the plain-C replay used at full size: same rows, same left-over, and it sees through a wrong trace
+        full = O.replay_trace_full(g.row_ptr, g.col_idx, b.trace, check_argmax_at=range(k + 1))
+        assert full["ok"] and full["final_max_redundancy"] == a.final_max_redundancy
+        assert full["full_recounts"] == k + 1
+        assert [r.tolist() for r in full["rows"]] == [r.tolist() for r in a.rows]
+        assert O.cover_check_rows(g.row_ptr, g.col_idx, b.trace, full["row_len"], full["row_store"]) == -1
+        if k >= 2:
+            wrong = b.trace.copy()
+            wrong[k - 1, 2] += 1                                        # a redundancy that the rows do not have
+            bad = O.replay_trace_full(g.row_ptr, g.col_idx, wrong)
+            assert not bad["ok"] and bad["failed_step"] == k - 1 and bad["detail"][0] == b.trace[k - 1, 2]
+            if tuple(b.trace[0, :2]) != tuple(b.trace[1, :2]) and b.trace[0, 2] > b.trace[1, 2]:
+                wrong = b.trace.copy()
+                wrong[[0, 1]] = wrong[[1, 0]]                           # a valid merge taken too early: not the arg-max
+                bad = O.replay_trace_full(g.row_ptr, g.col_idx, wrong, check_argmax_at=[0])
+                assert not bad["ok"] and bad["failed_step"] == 0
+            # a row that lost a source no longer covers its neighbourhood
+            rl = full["row_len"].copy()
+            u = int(np.argmax(rl))
+            rl[u] -= 1
+            assert O.cover_check_rows(g.row_ptr, g.col_idx, b.trace, rl, full["row_store"]) == u
 
 
 # --------------------------------------------------------------------------- #
@@ -356,35 +377,51 @@ def test_integer_features_are_exact():
 
 
 def test_expanded_deep_levels_are_covers_and_transitive_users():
-    """The expansion lists must reproduce the level-by-level values: the forward list of a deep
-    node sums to its a-hat, the backward list of a deep node to its gradient."""
+    """For EVERY cut the expansion lists must reproduce the level-by-level values: the forward
+    list of a deep node sums to its a-hat, the backward list of a deep node to its gradient;
+    cut 0 gives cover(v) itself (Section 3.1, Eq. 1), the deepest cut gives nothing to expand."""
     g = synth.clique_union_graph(seed=16, n=500, n_groups=140, g_lo=3, g_hi=30)
     res = O.greedy_pairmap(g.row_ptr, g.col_idx, g.n // 2)
     h = O.canonical_hag(g.row_ptr, res)
-    assert h.num_levels >= 4
-    t = O.expanded_tails(h)
+    L = h.num_levels
+    assert L >= 4
     rng = np.random.default_rng(0)
     x = rng.integers(-5, 6, size=(g.n, 3)).astype(np.float64)
     ahat = np.concatenate([x, np.zeros((h.num_agg, 3))])
     for j in range(h.num_agg):
         ahat[g.n + j] = ahat[h.agg_in[2 * j]] + ahat[h.agg_in[2 * j + 1]]
-    j0 = int(h.level_ptr[t["fwd_cut"]])
-    for i in range(h.num_agg - j0):
-        ids = t["ftail_idx"][t["ftail_ptr"][i]: t["ftail_ptr"][i + 1]]
-        assert len(set(ids.tolist())) == len(ids)
-        assert np.array_equal(ahat[ids].sum(0), ahat[g.n + j0 + i])
     gr = rng.integers(-5, 6, size=(g.n, 3)).astype(np.float64)
     ghat = np.zeros((h.num_agg, 3))
     for j in range(h.num_agg - 1, -1, -1):
         for d in h.t_idx[h.t_ptr[g.n + j]: h.t_ptr[g.n + j + 1]]:
             ghat[j] += gr[d] if d < g.n else ghat[d - g.n]
-    j0 = int(h.level_ptr[t["bwd_cut"]])
-    for i in range(h.num_agg - j0):
-        ids = t["btail_idx"][t["btail_ptr"][i]: t["btail_ptr"][i + 1]]
-        assert (ids < g.n).all() and len(set(ids.tolist())) == len(ids)
-        assert np.array_equal(gr[ids].sum(0), ghat[j0 + i])
-    # a small graph never pays for a launch per level: everything deeper than the cut is expanded
-    assert t["fwd_cut"] < h.num_levels and t["bwd_cut"] < h.num_levels
+    level = np.zeros(g.n + h.num_agg, dtype=np.int64)
+    for l in range(1, L + 1):
+        level[g.n + h.level_ptr[l - 1]: g.n + h.level_ptr[l]] = l
+    # cover(v) by its recursive definition, as a multiset of graph nodes
+    cover = {}
+    for j in range(h.num_agg):
+        c = []
+        for s_ in h.agg_in[2 * j: 2 * j + 2]:
+            c.extend([int(s_)] if s_ < g.n else cover[int(s_)])
+        cover[g.n + j] = sorted(c)
+    for cut in range(L + 1):
+        t = O.expanded_tails(h, cut, cut)
+        assert t["fwd_cut"] == cut and t["bwd_cut"] == cut
+        j0 = int(h.level_ptr[cut])
+        assert t["ftail_ptr"].shape[0] == h.num_agg - j0 + 1 == t["btail_ptr"].shape[0]
+        for i in range(h.num_agg - j0):
+            ids = t["ftail_idx"][t["ftail_ptr"][i]: t["ftail_ptr"][i + 1]]
+            assert len(set(ids.tolist())) == len(ids) and (level[ids] <= cut).all()
+            assert np.array_equal(ahat[ids].sum(0), ahat[g.n + j0 + i])
+            if cut == 0:
+                assert ids.tolist() == cover[g.n + j0 + i]
+            ids = t["btail_idx"][t["btail_ptr"][i]: t["btail_ptr"][i + 1]]
+            assert (ids < g.n).all() and len(set(ids.tolist())) == len(ids)
+            assert np.array_equal(gr[ids].sum(0), ghat[j0 + i])
+        assert np.array_equal(O.expanded_forward(h, x, cut, t), ahat)
+    with pytest.raises(ValueError):
+        O.expanded_tails(h, L + 1, 0)
 
 
 # --------------------------------------------------------------------------- #
