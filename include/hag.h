@@ -168,6 +168,15 @@ int32_t hag_build_threads(int32_t threads);
  * `src` stopped only because it hit its own capacity. */
 hag_status hag_truncate(const hag_t *src, int32_t capacity, hag_t **out);
 
+/* Replaces the cuts that hag_build chose (see there) and rebuilds the expansion lists of the
+ * deep levels.  Every cut 0 <= c <= num_levels evaluates the same HAG to the same values up to
+ * the order of additions (Section 3.1, Eq. 1: a node is the Aggregate over its cover); the
+ * choice only trades launches or dependent steps against longer input lists.  -1 for either
+ * argument keeps the library's own choice for that pass.  Host only, before hag_to_device.
+ * Errors: NULL; ARG (a cut outside -1..num_levels, or the handle is already on a device);
+ * OOM_HOST. */
+hag_status hag_set_cuts(hag_t *h, int32_t fwd_cut, int32_t bwd_cut);
+
 /* Frees host and device arrays.  NULL is allowed. */
 hag_status hag_destroy(hag_t *h);
 

@@ -26,7 +26,7 @@ HAG_F32, HAG_BF16 = 0, 1
  HAG_ERR_ALIGN, HAG_ERR_WORKSPACE, HAG_ERR_TIMEOUT, HAG_ERR_NOT_ON_DEVICE, HAG_ERR_TOO_LARGE) = range(13)
 
 EXPORTED_SYMBOLS = [
-    "hag_build", "hag_build_ex", "hag_build_threads", "hag_truncate", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes", "csr_workspace_bytes",
+    "hag_build", "hag_build_ex", "hag_build_threads", "hag_truncate", "hag_set_cuts", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes", "csr_workspace_bytes",
     "hag_aggregate_fwd", "hag_aggregate_bwd", "csr_aggregate_fwd", "csr_aggregate_bwd",
     "hag_aggregate_host", "hag_aggregate_fwd_static", "hag_graph_pool_fwd", "hag_graph_pool_bwd",
     "hag_max_workspace_bytes", "hag_max_fwd", "hag_max_bwd", "csr_max_fwd", "csr_max_bwd", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
@@ -84,6 +84,8 @@ def load_library():
     lib.hag_build_threads.restype = i32
     lib.hag_truncate.argtypes = [vp, i32, ctypes.POINTER(vp)]
     lib.hag_truncate.restype = ctypes.c_int
+    lib.hag_set_cuts.argtypes = [vp, i32, i32]
+    lib.hag_set_cuts.restype = ctypes.c_int
     lib.hag_destroy.argtypes = [vp]
     lib.hag_destroy.restype = ctypes.c_int
     lib.hag_get_info.argtypes = [vp, ctypes.POINTER(HagInfo)]
@@ -167,6 +169,8 @@ class Hag:
     def __init__(self, handle):
         self._h = handle
         self._ws = None
+        self._device = -1
+        self._n = int(self.info()["n"])
 
     # -- construction ------------------------------------------------------- #
     @classmethod
@@ -187,6 +191,11 @@ class Hag:
         handle = ctypes.c_void_p()
         _check(load_library().hag_truncate(self._h, int(capacity), ctypes.byref(handle)), "hag_truncate")
         return Hag(handle)
+
+    def set_cuts(self, fwd_cut: int = -1, bwd_cut: int = -1) -> "Hag":
+        """``hag_set_cuts``: force the levels evaluated level by level (-1 keeps the library's choice)."""
+        _check(load_library().hag_set_cuts(self._h, int(fwd_cut), int(bwd_cut)), "hag_set_cuts")
+        return self
 
     def close(self):
         if self._h:
@@ -284,19 +293,51 @@ class Hag:
             return HAG_BF16
         raise TypeError(f"features must be float32 or bfloat16, got {t.dtype}")
 
+    def _matrix(self, t, what, like=None, host=False):
+        """The C ABI takes raw pointers and trusts the caller on sizes: every tensor that reaches it is
+        checked here (device of the handle, 2-D, contiguous, N rows, dtype), so that a wrong argument is
+        a Python error and never an out-of-range device access."""
+        import torch
+        if not isinstance(t, torch.Tensor) or t.dim() != 2 or not t.is_contiguous():
+            raise ValueError(f"{what} must be a contiguous 2-D tensor")
+        if t.shape[0] != self._n:
+            raise ValueError(f"{what} has {t.shape[0]} rows, the graph has {self._n} nodes")
+        if t.shape[1] <= 0:
+            raise ValueError(f"{what} has no columns")
+        self._dtype_code(t)
+        if host:
+            if t.is_cuda:
+                raise ValueError(f"{what} must be a host tensor")
+        else:
+            if self._device < 0:
+                raise HagError(HAG_ERR_NOT_ON_DEVICE, what)
+            if not t.is_cuda or t.device.index != self._device:
+                raise ValueError(f"{what} must live on cuda:{self._device}, the handle's device")
+        if like is not None and (t.shape != like.shape or t.dtype != like.dtype or t.device != like.device):
+            raise ValueError(f"{what} must match the input's shape, dtype and device")
+        return t
+
+    def _scratch(self, ws, need_bytes, what="workspace"):
+        import torch
+        if need_bytes == 0:
+            return
+        if (not isinstance(ws, torch.Tensor) or not ws.is_cuda or ws.device.index != self._device
+                or not ws.is_contiguous() or ws.numel() * ws.element_size() < need_bytes):
+            raise ValueError(f"{what} must be a contiguous tensor of at least {need_bytes} bytes on cuda:{self._device}")
+
     def _run(self, name, use_hag, inp, reduce, out, workspace):
         import torch
-        if not inp.is_cuda or inp.dim() != 2 or not inp.is_contiguous():
-            raise ValueError("features must be a contiguous 2-D CUDA tensor")
+        self._matrix(inp, "features")
         if out is None:
             out = torch.empty_like(inp)
-        elif out.shape != inp.shape or out.dtype != inp.dtype or not out.is_contiguous() or out.device != inp.device:
-            raise ValueError("out must match the input's shape, dtype and device")
+        else:
+            self._matrix(out, "out", like=inp)
         d = inp.shape[1]
         stream = torch.cuda.current_stream(inp.device).cuda_stream
         lib = load_library()
         code = self._dtype_code(inp)
         ws = workspace if workspace is not None else self._workspace(d, inp.device)
+        self._scratch(ws, self.workspace_bytes(d) if use_hag else self.csr_workspace_bytes(d))
         st = getattr(lib, name)(self._h, _reduce_code(reduce), code, d, inp.data_ptr(), out.data_ptr(),
                                 ws.data_ptr() if ws is not None else None, stream)
         _check(st, name)
@@ -316,8 +357,8 @@ class Hag:
         scratch array built into the library (one per GPU, shared by all calls, so
         keep calls on one stream).  This wrapper allocates nothing either."""
         import torch
-        if out.shape != x.shape or out.dtype != x.dtype or not (x.is_contiguous() and out.is_contiguous()):
-            raise ValueError("out must match x")
+        self._matrix(x, "features")
+        self._matrix(out, "out", like=x)
         stream = torch.cuda.current_stream(x.device).cuda_stream
         st = load_library().hag_aggregate_fwd_static(self._h, _reduce_code(reduce), self._dtype_code(x), x.shape[1],
                                                      x.data_ptr(), out.data_ptr(), stream)
@@ -341,13 +382,17 @@ class Hag:
     def max_fwd(self, z, out=None, workspace=None, use_hag=True):
         """``hag_max_fwd`` (or ``csr_max_fwd``).  Returns (out, workspace); keep both for ``max_bwd``."""
         import torch
+        self._matrix(z, "z")
         if out is None:
             out = torch.empty_like(z)
-        s = torch.cuda.current_stream().cuda_stream
+        else:
+            self._matrix(out, "out", like=z)
+        s = torch.cuda.current_stream(z.device).cuda_stream
         lib = load_library()
         if use_hag:
             if workspace is None:
                 workspace = self.max_workspace(z.shape[1], z.device)
+            self._scratch(workspace, int(lib.hag_max_workspace_bytes(self._h, z.shape[1])))
             st = lib.hag_max_fwd(self._h, self._dtype_code(z), z.shape[1], z.data_ptr(), out.data_ptr(), workspace.data_ptr(), s)
         else:
             st = lib.csr_max_fwd(self._h, self._dtype_code(z), z.shape[1], z.data_ptr(), out.data_ptr(), s)
@@ -357,14 +402,22 @@ class Hag:
     def max_bwd(self, z, fwd_out, fwd_workspace, grad_out, out=None, workspace=None, use_hag=True):
         """``hag_max_bwd`` (or ``csr_max_bwd``): the gradient with respect to z."""
         import torch
+        self._matrix(z, "z")
+        self._matrix(fwd_out, "fwd_out", like=z)
+        self._matrix(grad_out, "grad_out", like=z)
         if out is None:
             out = torch.empty_like(z)
-        s = torch.cuda.current_stream().cuda_stream
+        else:
+            self._matrix(out, "out", like=z)
+        s = torch.cuda.current_stream(z.device).cuda_stream
         lib = load_library()
         code = self._dtype_code(z)
         if use_hag:
             if workspace is None:
                 workspace = self.max_workspace(z.shape[1], z.device)
+            need = int(lib.hag_max_workspace_bytes(self._h, z.shape[1]))
+            self._scratch(workspace, need)
+            self._scratch(fwd_workspace, need, "fwd_workspace")
             st = lib.hag_max_bwd(self._h, code, z.shape[1], z.data_ptr(), fwd_out.data_ptr(), fwd_workspace.data_ptr(),
                                  grad_out.data_ptr(), out.data_ptr(), workspace.data_ptr(), s)
         else:
@@ -376,9 +429,11 @@ class Hag:
         """``hag_aggregate_host``: host tensors in and out (pinned for async copies);
         enqueues copy-in, aggregation and copy-out on the stream; the caller synchronises."""
         import torch
-        if inp.is_cuda or out.is_cuda or inp.shape != out.shape or inp.dtype != out.dtype:
-            raise ValueError("aggregate_host takes matching host tensors")
-        s = torch.cuda.current_stream().cuda_stream if stream is None else stream
+        self._matrix(inp, "input", host=True)
+        self._matrix(out, "out", like=inp, host=True)
+        if self._device < 0:
+            raise HagError(HAG_ERR_NOT_ON_DEVICE, "aggregate_host")
+        s = torch.cuda.current_stream(self._device).cuda_stream if stream is None else stream
         st = load_library().hag_aggregate_host(self._h, int(backward), int(use_hag), _reduce_code(reduce),
                                                self._dtype_code(inp), inp.shape[1], inp.data_ptr(), out.data_ptr(), s)
         _check(st, "hag_aggregate_host")

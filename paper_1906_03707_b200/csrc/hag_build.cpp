@@ -330,6 +330,149 @@ hag_status hag_search(hag *h, std::vector<int32_t> &rows_store, std::vector<int3
     return HAG_OK;
 }
 
+namespace {
+
+// Deep levels without their intermediate nodes (Section 3.1, Eq. 1: aggr(v) aggregates cover(v)).
+// Forward, cut c: every node deeper than level c gets the list of its cover restricted to ids of
+// level <= c.  Backward, cut c: every node deeper than c gets the graph-node outputs that use it,
+// directly or through deeper nodes.  Any 0 <= c <= L gives the same values; which one is taken is
+// a question of launch cost only (choose_cuts).
+void expand_tails(hag *h, int32_t fwd_cut, int32_t bwd_cut) {
+    const int32_t n = h->n, k = h->num_agg, L = h->num_levels;
+    std::vector<int32_t> clevel(k);      // level per canonical aggregation node
+    for (int32_t l = 1; l <= L; ++l)
+        for (int64_t j = h->level_ptr[l - 1]; j < h->level_ptr[l]; ++j) clevel[j] = l;
+    auto level_of = [&](int32_t id) { return id < n ? 0 : clevel[id - n]; };
+    h->fwd_cut = fwd_cut;
+    {
+        const int64_t j0 = h->level_ptr[fwd_cut];
+        std::vector<std::vector<int32_t>> lists(size_t(k - j0));
+        h->ftail_ptr.assign(size_t(k - j0) + 1, 0);
+        for (int64_t j = j0; j < k; ++j) {
+            std::vector<int32_t> &dst = lists[j - j0];
+            for (int q = 0; q < 2; ++q) {
+                const int32_t in = h->agg_in[2 * j + q];
+                if (level_of(in) <= fwd_cut) dst.push_back(in);
+                else dst.insert(dst.end(), lists[in - n - j0].begin(), lists[in - n - j0].end());
+            }
+            std::sort(dst.begin(), dst.end());
+            h->ftail_ptr[j - j0 + 1] = h->ftail_ptr[j - j0] + int64_t(dst.size());
+        }
+        h->ftail_idx.clear();
+        h->ftail_idx.reserve(size_t(h->ftail_ptr.back()));
+        for (auto &l : lists) h->ftail_idx.insert(h->ftail_idx.end(), l.begin(), l.end());
+    }
+    h->bwd_cut = bwd_cut;
+    {
+        const int64_t j0 = h->level_ptr[bwd_cut];
+        std::vector<std::vector<int32_t>> lists(size_t(k - j0));
+        for (int64_t j = k - 1; j >= j0; --j) {
+            std::vector<int32_t> &dst = lists[j - j0];
+            for (int64_t i = h->t_ptr[n + j]; i < h->t_ptr[n + j + 1]; ++i) {
+                const int32_t d = h->t_idx[i];
+                if (d < n) dst.push_back(d);
+                else dst.insert(dst.end(), lists[d - n - j0].begin(), lists[d - n - j0].end());
+            }
+            std::sort(dst.begin(), dst.end());
+        }
+        h->btail_ptr.assign(size_t(k - j0) + 1, 0);
+        for (int64_t j = j0; j < k; ++j) h->btail_ptr[j - j0 + 1] = h->btail_ptr[j - j0] + int64_t(lists[j - j0].size());
+        h->btail_idx.clear();
+        h->btail_idx.reserve(size_t(h->btail_ptr.back()));
+        for (auto &l : lists) h->btail_idx.insert(h->btail_idx.end(), l.begin(), l.end());
+    }
+}
+
+// The cuts by launch cost.  What one extra launch costs, in rows moved; measured on B200: the
+// backward launches (rows of tens of users each) pay for a merge up to four times later than the
+// forward ones (rows of two to eight inputs).
+void choose_cuts(const hag *h, int32_t &fwd_cut, int32_t &bwd_cut) {
+    const int64_t kLaunchRows = 32768, kBwdLaunchRows = 131072;
+    const int32_t n = h->n, k = h->num_agg, L = h->num_levels;
+    std::vector<int32_t> clevel(k);
+    for (int32_t l = 1; l <= L; ++l)
+        for (int64_t j = h->level_ptr[l - 1]; j < h->level_ptr[l]; ++j) clevel[j] = l;
+    auto level_of = [&](int32_t id) { return id < n ? 0 : clevel[id - n]; };
+    // forward: size of the expansion of every node for a given cut
+    int32_t best_c = L;
+    int64_t best_cost = kLaunchRows * L;
+    std::vector<int64_t> sz(k);
+    for (int32_t c = L - 1; c >= 0; --c) {
+        int64_t extra = 0;
+        for (int64_t j = h->level_ptr[c]; j < k; ++j) {
+            int64_t t = 0;
+            for (int q = 0; q < 2; ++q) {
+                const int32_t in = h->agg_in[2 * j + q];
+                t += level_of(in) <= c ? 1 : sz[in - n];
+            }
+            sz[j] = t;
+            extra += t - 1;
+        }
+        const int64_t cost = kLaunchRows * (c + 1) + extra;
+        if (cost < best_cost) { best_cost = cost; best_c = c; }
+    }
+    fwd_cut = best_c;
+    // backward: every node's transitive graph-node users (independent of the cut)
+    std::vector<int64_t> usz(k);
+    for (int64_t j = k - 1; j >= 0; --j) {
+        int64_t t = 0;
+        for (int64_t i = h->t_ptr[n + j]; i < h->t_ptr[n + j + 1]; ++i) {
+            const int32_t d = h->t_idx[i];
+            t += d < n ? 1 : usz[d - n];
+        }
+        usz[j] = t;
+    }
+    int32_t best_b = L;
+    int64_t best_bcost = kBwdLaunchRows * L;
+    int64_t extra = 0;
+    for (int32_t c = L - 1; c >= 0; --c) {
+        for (int64_t j = h->level_ptr[c]; j < h->level_ptr[c + 1]; ++j)
+            extra += usz[j] - (h->t_ptr[n + j + 1] - h->t_ptr[n + j]);
+        const int64_t cost = kBwdLaunchRows * (c + 1) + extra;
+        if (cost < best_bcost) { best_bcost = cost; best_b = c; }
+    }
+    bwd_cut = best_b;
+}
+
+// Segments of the long rows of every table the gather walks.
+void build_segments(hag *h) {
+    const int32_t n = h->n, k = h->num_agg;
+    auto build = [](seg_set &set, const std::vector<int64_t> &ptr, int64_t rows, int32_t first_row_id) {
+        for (int gran = 0; gran < kSegGrans; ++gran) {
+            seg_table &t = set.g[gran];
+            const int64_t long_row = kSegLongRow[gran], seg_len = kSegLength[gran];
+            t.segs.clear();
+            t.slots.clear();
+            for (int64_t r = 0; r < rows; ++r) {
+                const int64_t b = ptr[r], e = ptr[r + 1];
+                if (e - b <= long_row) continue;
+                const int32_t slot = int32_t(t.slots.size() / 2);
+                const int32_t first = int32_t(t.segs.size() / 4);
+                int32_t n_seg = 0;
+                for (int64_t sb = b; sb < e; sb += seg_len, ++n_seg) {
+                    t.segs.push_back(int32_t(first_row_id + r));
+                    t.segs.push_back(int32_t(sb));
+                    t.segs.push_back(int32_t(std::min<int64_t>(sb + seg_len, e)));
+                    t.segs.push_back(slot);
+                }
+                t.slots.push_back(first);
+                t.slots.push_back(n_seg);
+            }
+        }
+    };
+    build(h->seg_res, h->res_ptr, n, 0);
+    build(h->seg_t, h->t_ptr, int64_t(n) + k, 0);
+    build(h->seg_csr, h->csr_ptr, n, 0);
+    build(h->seg_csr_t, h->csr_t_ptr, n, 0);
+    build(h->seg_ftail, h->ftail_ptr, int64_t(h->ftail_ptr.size()) - 1, int32_t(n + h->level_ptr[h->fwd_cut]));
+    build(h->seg_btail, h->btail_ptr, int64_t(h->btail_ptr.size()) - 1, int32_t(n + h->level_ptr[h->bwd_cut]));
+    h->max_segs_hag = std::max(std::max(h->seg_res.max_count(), h->seg_t.max_count()),
+                               std::max(h->seg_ftail.max_count(), h->seg_btail.max_count()));
+    h->max_segs_csr = std::max(h->seg_csr.max_count(), h->seg_csr_t.max_count());
+}
+
+}  // namespace
+
 hag_status hag_layout(hag *h, const std::vector<int32_t> &rows_store, const std::vector<int32_t> &rows_len) {
     try {
         const int32_t n = h->n, k = h->num_agg;
@@ -404,129 +547,10 @@ hag_status hag_layout(hag *h, const std::vector<int32_t> &rows_store, const std:
             for (int32_t v = 0; v < n; ++v)
                 for (int64_t i = h->csr_ptr[v]; i < h->csr_ptr[v + 1]; ++i) h->csr_t_idx[fill[h->csr_idx[i]]++] = v;
         }
-        // ---- deep levels in one launch: choose the cuts and expand ----
-        {
-            // what one extra launch costs, in rows moved; measured on B200: the backward launches (rows of tens of
-            // users each) pay for a merge up to four times later than the forward ones (rows of two to eight inputs)
-            const int64_t kLaunchRows = 32768, kBwdLaunchRows = 131072;
-            const int32_t L = max_level;
-            std::vector<int32_t> clevel(k);      // level per canonical aggregation node
-            for (int32_t l = 1; l <= L; ++l)
-                for (int64_t j = h->level_ptr[l - 1]; j < h->level_ptr[l]; ++j) clevel[j] = l;
-            auto level_of = [&](int32_t id) { return id < n ? 0 : clevel[id - n]; };
-            // forward: size of the expansion of every node for a given cut
-            int32_t best_c = L;
-            int64_t best_cost = kLaunchRows * L;
-            std::vector<int64_t> sz(k);
-            for (int32_t c = L - 1; c >= 0; --c) {
-                int64_t extra = 0;
-                for (int64_t j = h->level_ptr[c]; j < k; ++j) {
-                    int64_t t = 0;
-                    for (int q = 0; q < 2; ++q) {
-                        const int32_t in = h->agg_in[2 * j + q];
-                        t += level_of(in) <= c ? 1 : sz[in - n];
-                    }
-                    sz[j] = t;
-                    extra += t - 1;
-                }
-                const int64_t cost = kLaunchRows * (c + 1) + extra;
-                if (cost < best_cost) { best_cost = cost; best_c = c; }
-            }
-            h->fwd_cut = best_c;
-            {
-                const int64_t j0 = h->level_ptr[best_c];
-                std::vector<std::vector<int32_t>> lists(size_t(k - j0));
-                h->ftail_ptr.assign(size_t(k - j0) + 1, 0);
-                for (int64_t j = j0; j < k; ++j) {
-                    std::vector<int32_t> &dst = lists[j - j0];
-                    for (int q = 0; q < 2; ++q) {
-                        const int32_t in = h->agg_in[2 * j + q];
-                        if (level_of(in) <= best_c) dst.push_back(in);
-                        else dst.insert(dst.end(), lists[in - n - j0].begin(), lists[in - n - j0].end());
-                    }
-                    std::sort(dst.begin(), dst.end());
-                    h->ftail_ptr[j - j0 + 1] = h->ftail_ptr[j - j0] + int64_t(dst.size());
-                }
-                h->ftail_idx.clear();
-                h->ftail_idx.reserve(size_t(h->ftail_ptr.back()));
-                for (auto &l : lists) h->ftail_idx.insert(h->ftail_idx.end(), l.begin(), l.end());
-            }
-            // backward: every node's transitive graph-node users (independent of the cut)
-            std::vector<int64_t> usz(k);
-            for (int64_t j = k - 1; j >= 0; --j) {
-                int64_t t = 0;
-                for (int64_t i = h->t_ptr[n + j]; i < h->t_ptr[n + j + 1]; ++i) {
-                    const int32_t d = h->t_idx[i];
-                    t += d < n ? 1 : usz[d - n];
-                }
-                usz[j] = t;
-            }
-            int32_t best_b = L;
-            int64_t best_bcost = kBwdLaunchRows * L;
-            {
-                int64_t extra = 0;
-                for (int32_t c = L - 1; c >= 0; --c) {
-                    for (int64_t j = h->level_ptr[c]; j < h->level_ptr[c + 1]; ++j)
-                        extra += usz[j] - (h->t_ptr[n + j + 1] - h->t_ptr[n + j]);
-                    const int64_t cost = kBwdLaunchRows * (c + 1) + extra;
-                    if (cost < best_bcost) { best_bcost = cost; best_b = c; }
-                }
-            }
-            h->bwd_cut = best_b;
-            {
-                const int64_t j0 = h->level_ptr[best_b];
-                std::vector<std::vector<int32_t>> lists(size_t(k - j0));
-                for (int64_t j = k - 1; j >= j0; --j) {
-                    std::vector<int32_t> &dst = lists[j - j0];
-                    for (int64_t i = h->t_ptr[n + j]; i < h->t_ptr[n + j + 1]; ++i) {
-                        const int32_t d = h->t_idx[i];
-                        if (d < n) dst.push_back(d);
-                        else dst.insert(dst.end(), lists[d - n - j0].begin(), lists[d - n - j0].end());
-                    }
-                    std::sort(dst.begin(), dst.end());
-                }
-                h->btail_ptr.assign(size_t(k - j0) + 1, 0);
-                for (int64_t j = j0; j < k; ++j) h->btail_ptr[j - j0 + 1] = h->btail_ptr[j - j0] + int64_t(lists[j - j0].size());
-                h->btail_idx.clear();
-                h->btail_idx.reserve(size_t(h->btail_ptr.back()));
-                for (auto &l : lists) h->btail_idx.insert(h->btail_idx.end(), l.begin(), l.end());
-            }
-        }
-        // ---- segments of the long rows of every table the gather walks ----
-        {
-            auto build = [](seg_set &set, const std::vector<int64_t> &ptr, int64_t rows, int32_t first_row_id) {
-                for (int gran = 0; gran < kSegGrans; ++gran) {
-                    seg_table &t = set.g[gran];
-                    const int64_t long_row = kSegLongRow[gran], seg_len = kSegLength[gran];
-                    t.segs.clear();
-                    t.slots.clear();
-                    for (int64_t r = 0; r < rows; ++r) {
-                        const int64_t b = ptr[r], e = ptr[r + 1];
-                        if (e - b <= long_row) continue;
-                        const int32_t slot = int32_t(t.slots.size() / 2);
-                        const int32_t first = int32_t(t.segs.size() / 4);
-                        int32_t n_seg = 0;
-                        for (int64_t sb = b; sb < e; sb += seg_len, ++n_seg) {
-                            t.segs.push_back(int32_t(first_row_id + r));
-                            t.segs.push_back(int32_t(sb));
-                            t.segs.push_back(int32_t(std::min<int64_t>(sb + seg_len, e)));
-                            t.segs.push_back(slot);
-                        }
-                        t.slots.push_back(first);
-                        t.slots.push_back(n_seg);
-                    }
-                }
-            };
-            build(h->seg_res, h->res_ptr, n, 0);
-            build(h->seg_t, h->t_ptr, int64_t(n) + k, 0);
-            build(h->seg_csr, h->csr_ptr, n, 0);
-            build(h->seg_csr_t, h->csr_t_ptr, n, 0);
-            build(h->seg_ftail, h->ftail_ptr, int64_t(h->ftail_ptr.size()) - 1, int32_t(n + h->level_ptr[h->fwd_cut]));
-            build(h->seg_btail, h->btail_ptr, int64_t(h->btail_ptr.size()) - 1, int32_t(n + h->level_ptr[h->bwd_cut]));
-            h->max_segs_hag = std::max(std::max(h->seg_res.max_count(), h->seg_t.max_count()),
-                                       std::max(h->seg_ftail.max_count(), h->seg_btail.max_count()));
-            h->max_segs_csr = std::max(h->seg_csr.max_count(), h->seg_csr_t.max_count());
-        }
+        int32_t fwd_cut = 0, bwd_cut = 0;
+        choose_cuts(h, fwd_cut, bwd_cut);
+        expand_tails(h, fwd_cut, bwd_cut);
+        build_segments(h);
         // counters of the cost function
         hag_info &f = h->info;
         f = hag_info{};
@@ -616,6 +640,21 @@ extern "C" int32_t hag_build_threads(int32_t threads) {
     const int prev = g_build_threads.load();
     if (threads >= 0) g_build_threads.store(threads);
     return prev;
+}
+
+extern "C" hag_status hag_set_cuts(hag_t *h, int32_t fwd_cut, int32_t bwd_cut) {
+    if (!h) return HAG_ERR_NULL;
+    if (h->device >= 0) return HAG_ERR_ARG;                    // the device copy is made once
+    if (fwd_cut < -1 || fwd_cut > h->num_levels || bwd_cut < -1 || bwd_cut > h->num_levels) return HAG_ERR_ARG;
+    try {
+        int32_t f = 0, b = 0;
+        if (fwd_cut < 0 || bwd_cut < 0) choose_cuts(h, f, b);
+        expand_tails(h, fwd_cut < 0 ? f : fwd_cut, bwd_cut < 0 ? b : bwd_cut);
+        build_segments(h);
+    } catch (const std::bad_alloc &) {
+        return HAG_ERR_OOM_HOST;
+    }
+    return HAG_OK;
 }
 
 extern "C" hag_status hag_truncate(const hag_t *src, int32_t capacity, hag_t **out) {

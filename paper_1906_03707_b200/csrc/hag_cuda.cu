@@ -111,10 +111,6 @@ cudaError_t launch_pdl(void (*kernel)(Args), unsigned grid, const Args &args, cu
 constexpr int32_t kManyRows = 131072;
 constexpr int64_t kManyEdges = int64_t(4) << 20;
 
-#ifdef HAG_TUNING
-int g_tune = -1;   // tuning builds only: force a launch shape
-#endif
-
 // Persistent form: exactly as many CTAs as stay resident, rows handed out through a.sched.
 template <typename Kernel, typename Args>
 cudaError_t launch_persistent(Kernel kernel, const Args &a, int64_t items, int sm_count, cudaStream_t s) {
@@ -151,22 +147,6 @@ cudaError_t launch_gather_shape(const hagk::GatherArgs &ga, const hagk::SegArgs 
     const hagk::KernelArgs<SEGS> a = pack_args<SEGS>(ga, sg);
     const int64_t items = int64_t(ga.row_count) + (SEGS ? sg.seg_count : 0);
     const unsigned grid = unsigned((items + hagk::kWarps - 1) / hagk::kWarps);
-#ifdef HAG_TUNING
-    switch (g_tune) {
-        case 0: return launch_pdl(plain_kernel<T, LPR, 8, SS, 8, SEGS, SELF>(), grid, a, s);
-        case 2: return launch_pdl(plain_kernel<T, LPR, 4, SS, 12, SEGS, SELF>(), grid, a, s);
-        case 4: return launch_pdl(plain_kernel<T, LPR, 2, SS, 16, SEGS, SELF>(), grid, a, s);
-        case 5: return launch_pdl(plain_kernel<T, LPR, 4, SS, 10, SEGS, SELF>(), grid, a, s);
-        case 6: return launch_pdl(plain_kernel<T, LPR, 2, SS, 10, SEGS, SELF>(), grid, a, s);
-        case 7: return launch_pdl(plain_kernel<T, LPR, 4, SS, 8, SEGS, SELF>(), grid, a, s);
-        case 8: return launch_pdl(plain_kernel<T, LPR, 2, SS, 8, SEGS, SELF>(), grid, a, s);
-        case 3: return launch_pdl(plain_kernel<T, LPR, 2, SS, 12, SEGS, SELF>(), grid, a, s);
-        case 9: return launch_persistent(resident_kernel<T, LPR, 4, SS, 10, SEGS, SELF>(), a, items, sm_count, s);
-        case 10: return launch_persistent(resident_kernel<T, LPR, 4, SS, 8, SEGS, SELF>(), a, items, sm_count, s);
-        case 11: return launch_persistent(resident_kernel<T, LPR, 8, SS, 8, SEGS, SELF>(), a, items, sm_count, s);
-        default: break;
-    }
-#endif
     if constexpr (sizeof(T) == 4) {
         if (ga.resident) {
             if constexpr (LPR == 32) return launch_persistent(resident_kernel<T, LPR, 8, SS, 8, SEGS, SELF>(), a, items, sm_count, s);
@@ -714,7 +694,3 @@ extern "C" hag_status hag_aggregate_fwd_static(const hag_t *h, hag_reduce reduce
     if (dtype == HAG_F32) return fwd_static_impl<float>(h, reduce, D, x, out, static_cast<float *>(scratch), s);
     return fwd_static_impl<__nv_bfloat16>(h, reduce, D, x, out, static_cast<float *>(scratch), s);
 }
-
-#ifdef HAG_TUNING
-extern "C" void hag_debug_set_tune(int v) { g_tune = v; }
-#endif

@@ -59,13 +59,7 @@ struct PairMaxArgs {
 // Launch shapes from a sweep on B200 (loads or entries in flight per lane, resident CTAs per SM):
 // more resident warps beat more loads per warp, as for the sum kernels.
 //   fp32: forward 4 loads x 10 CTAs, backward 2 entries x 10 CTAs; bf16: forward 2 x 10, backward 1 x 8.
-#ifndef HAG_MAX_SHAPES
 #define HAG_MAX_SHAPES 4, 10, 2, 10, 2, 10, 1, 8
-#endif
-#ifdef HAG_MS0      // tuning builds: the eight numbers one by one
-#undef HAG_MAX_SHAPES
-#define HAG_MAX_SHAPES HAG_MS0, HAG_MS1, HAG_MS2, HAG_MS3, HAG_MS4, HAG_MS5, HAG_MS6, HAG_MS7
-#endif
 template <typename T> struct MaxShape;
 template <int FL, int FB, int BE, int BB, int HFL, int HFB, int HBE, int HBB> struct MaxShapeTable {
     static constexpr int f32[4] = {FL, FB, BE, BB};

@@ -46,8 +46,8 @@ __global__ void __launch_bounds__(hagk::kThreads) graph_pool_fwd_kernel(const Po
     const int lane = threadIdx.x & 31;
     const int seg = blockIdx.x * hagk::kWarps + (threadIdx.x >> 5);
     if (seg >= p.n_graphs) return;
-    const int32_t b = __ldg(p.seg_ptr + seg), e = __ldg(p.seg_ptr + seg + 1);
-    hagk::pdl_wait();
+    hagk::pdl_wait();      // seg_ptr is the caller's array: the kernel before this one may have written it
+    const int32_t b = p.seg_ptr[seg], e = p.seg_ptr[seg + 1];
     const int slice = lane / LPR, gl = lane % LPR;
     const int n_chunks = p.D / E;
     const size_t row_bytes = size_t(p.D) * sizeof(T);
@@ -115,16 +115,16 @@ __global__ void __launch_bounds__(hagk::kThreads) graph_pool_bwd_kernel(const Po
     const int slice = lane / LPR, gl = lane % LPR;
     const int n_chunks = p.D / E;
     int32_t b, e, zb = 0, ze = 0;                       // [b, e): rows that get the gradient; [zb, ze): rows cleared
+    hagk::pdl_wait();      // seg_ptr is the caller's array: the kernel before this one may have written it
     if (seg < p.n_graphs) {
-        b = __ldg(p.seg_ptr + seg);
-        e = __ldg(p.seg_ptr + seg + 1);
+        b = p.seg_ptr[seg];
+        e = p.seg_ptr[seg + 1];
         if (seg == 0) ze = b;
     } else {
         b = e = 0;
-        zb = (p.n_graphs > 0) ? __ldg(p.seg_ptr + p.n_graphs) : 0;
+        zb = (p.n_graphs > 0) ? p.seg_ptr[p.n_graphs] : 0;
         ze = p.n_rows;
     }
-    hagk::pdl_wait();
     const float scale = (p.mean && e > b) ? 1.0f / float(e - b) : 1.0f;
     for (int c0 = 0; c0 < n_chunks; c0 += LPR) {
         const int chunk = c0 + gl;

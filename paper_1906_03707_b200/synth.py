@@ -100,12 +100,6 @@ def csr_from_rows(rows) -> Graph:
     return Graph(n=n, row_ptr=row_ptr, col_idx=np.asarray(cols, dtype=np.int32))
 
 
-def transpose_csr(g: Graph) -> Graph:
-    """CSR of out-neighbours (row u lists the destinations v with u in N(v)), sorted."""
-    dst = np.repeat(np.arange(g.n, dtype=np.int64), np.diff(g.row_ptr))
-    return csr_from_directed_pairs(g.n, dst, g.col_idx.astype(np.int64), name=g.name + "^T")
-
-
 def permute_ids(g: Graph, seed: int) -> Graph:
     """Relabel nodes by a random permutation (locality stress test)."""
     rng = np.random.Generator(np.random.PCG64(seed))

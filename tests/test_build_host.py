@@ -34,7 +34,10 @@ def _same_structure(g, capacity, search=O.greedy_pairmap):
         assert got.dtype == want.dtype and np.array_equal(got, want), key
     t_ptr, t_idx = O.transposed_csr(g.row_ptr, g.col_idx)
     assert np.array_equal(arr["csr_t_ptr"], t_ptr) and np.array_equal(arr["csr_t_idx"], t_idx)
-    tails = O.expanded_tails(ref)
+    # the cuts are the library's own choice (a launch heuristic, nothing the paper fixes): any value in
+    # 0..L is valid; the lists must be the oracle's for THAT choice
+    assert 0 <= arr["fwd_cut"] <= ref.num_levels and 0 <= arr["bwd_cut"] <= ref.num_levels
+    tails = O.expanded_tails(ref, int(arr["fwd_cut"]), int(arr["bwd_cut"]))
     for key, want in tails.items():
         assert np.array_equal(arr[key], want), key
     info = h.info()
@@ -95,6 +98,57 @@ def test_structure_is_bit_exact_on_workload_shapes(maker, cap_frac):
     info = _same_structure(g, int(g.n * cap_frac))
     if cap_frac == 0.0:
         assert info["num_agg"] == 0 and info["e_hat"] == info["e"]
+
+
+@pytest.mark.parametrize("maker", [
+    lambda: synth.clique_union_graph(seed=15, n=1500, n_groups=400, g_lo=3, g_hi=40),
+    lambda: synth.config2_graph(seed=11, n=3000, n_comm=30),
+])
+def test_every_forced_cut_gives_the_oracles_lists_and_algorithm_2s_values(maker):
+    """hag_set_cuts: for every cut 0..L the library's expansion lists equal the oracle's for that
+    cut, and evaluating the deep levels from them gives Algorithm 2's level-by-level values."""
+    g = maker()
+    res = O.greedy_pairmap(g.row_ptr, g.col_idx, g.n // 4)
+    ref = O.canonical_hag(g.row_ptr, res)
+    L = ref.num_levels
+    assert L >= 3
+    x = synth.features(5, g.n, 4, "int").astype(np.float64)
+    ahat = np.zeros((g.n + ref.num_agg, 4))
+    ahat[:g.n] = x
+    for j in range(ref.num_agg):                                   # Algorithm 2 lines 5-6, node by node
+        ahat[g.n + j] = ahat[ref.agg_in[2 * j]] + ahat[ref.agg_in[2 * j + 1]]
+    h = hb.Hag.build(g.row_ptr, g.col_idx, g.n // 4)
+    own = (int(h.arrays()["fwd_cut"]), int(h.arrays()["bwd_cut"]))
+    for cut in range(L + 1):
+        h.set_cuts(cut, L - cut)
+        arr = h.arrays()
+        assert (arr["fwd_cut"], arr["bwd_cut"]) == (cut, L - cut)
+        want = O.expanded_tails(ref, cut, L - cut)
+        for key, v in want.items():
+            assert np.array_equal(arr[key], v), (cut, key)
+        lib_lists = dict(ftail_ptr=arr["ftail_ptr"], ftail_idx=arr["ftail_idx"])
+        assert np.array_equal(O.expanded_forward(ref, x, cut, lib_lists), ahat), cut
+    h.set_cuts(-1, -1)
+    assert (int(h.arrays()["fwd_cut"]), int(h.arrays()["bwd_cut"])) == own
+    lib = hb.load_library()
+    assert lib.hag_set_cuts(h._h, L + 1, 0) == 2 and lib.hag_set_cuts(h._h, 0, -2) == 2
+    assert lib.hag_set_cuts(None, 0, 0) == 1
+
+
+def test_full_size_search_replays_are_stored(golden_dir):
+    """The two largest shapes are reached only by the oracle's memory-light search.  Their stored digests are
+    backed by a from-the-definition replay of the whole trace (tests/golden/make_replay_pins.py): every
+    recorded redundancy recounted, the arg-max recounted over all pairs at about twenty seeded merges
+    and after the last one, the cover condition, both cost forms, the gain per merge, non-increasing
+    redundancies, and the layout of the replayed rows reproducing the digest."""
+    stored = json.load(open(os.path.join(golden_dir, "structure_hashes.json")))
+    for key in ("cfg3@1", "cfg5@1"):
+        rec = stored["cases"][key].get("replay_ok")
+        assert rec is not None, f"{key}: run tests/golden/make_replay_pins.py"
+        assert rec["ok"] is True and all(rec["checks"].values()), key
+        assert rec["merges_replayed"] == stored["cases"][key]["num_agg"]
+        assert len(rec["argmax_checked_at"]) >= 15 and rec["full_recounts"] == len(rec["argmax_checked_at"]) + 1
+        assert rec["redundancy_left_after_last_merge"] <= rec["last_redundancy"] <= rec["first_redundancy"]
 
 
 def test_stored_structure_hashes(golden_dir):
@@ -238,3 +292,29 @@ def test_min_redundancy_stops_the_search_earlier():
     lib = hb.load_library()
     out = ctypes.c_void_p()
     assert lib.hag_build_ex(g.n, g.row_ptr.ctypes.data, g.col_idx.ctypes.data, 10, 1, ctypes.byref(out)) == 2
+
+
+def test_binding_rejects_wrong_tensors_before_any_launch():
+    """The C ABI trusts pointers and sizes; the binding must turn every mismatch into a Python error."""
+    torch = pytest.importorskip("torch")
+    g = synth.workload(1).graph
+    h = hb.Hag.build(g.row_ptr, g.col_idx, 100)
+    good = torch.zeros((g.n, 16))
+    for call in (lambda t: h.aggregate_fwd(t), lambda t: h.aggregate_bwd(t), lambda t: h.csr_fwd(t), lambda t: h.csr_bwd(t),
+                 lambda t: h.max_fwd(t), lambda t: h.aggregate_fwd_static(t, torch.zeros_like(t)),
+                 lambda t: h.aggregate_host(t, torch.zeros_like(t))):
+        with pytest.raises(ValueError, match="rows"):
+            call(torch.zeros((g.n - 1, 16)))                      # too few rows: would be an out-of-range read
+        with pytest.raises(ValueError):
+            call(torch.zeros(g.n * 16))                           # not 2-D
+        with pytest.raises(ValueError):
+            call(torch.zeros((g.n, 32))[:, ::2])                  # not contiguous
+        with pytest.raises(TypeError):
+            call(torch.zeros((g.n, 16), dtype=torch.float64))
+        with pytest.raises(hb.HagError) as info:                  # right shape, but the handle is host-only
+            call(good)
+        assert info.value.status == hb.HAG_ERR_NOT_ON_DEVICE
+    with pytest.raises(ValueError):
+        h.aggregate_host(good, torch.zeros((g.n, 8)))             # out does not match
+    with pytest.raises(ValueError):
+        h.max_bwd(torch.zeros((g.n - 1, 16)), good, None, good)
