@@ -78,8 +78,12 @@ template <> struct Chunk<__nv_bfloat16> { static constexpr int kElems = 8; };
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-__device__ __forceinline__ float4 ld_f4(const void *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
-__device__ __forceinline__ uint4 ld_u4(const void *p) { return __ldg(reinterpret_cast<const uint4 *>(p)); }
+// Feature rows and aggregation-node rows are read with ld.global.cg (coherent, cached at L2 only): the rows
+// may have been written by the kernel before this one, which is still alive when this one starts under
+// programmatic dependent launch.  The non-coherent path (ld.global.nc, __ldg) is kept for the handle's
+// static structure arrays only.
+__device__ __forceinline__ float4 ld_f4(const void *p) { return __ldcg(reinterpret_cast<const float4 *>(p)); }
+__device__ __forceinline__ uint4 ld_u4(const void *p) { return __ldcg(reinterpret_cast<const uint4 *>(p)); }
 
 __device__ __forceinline__ void bf16x8_to_f32(const uint4 &v, float *f) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
