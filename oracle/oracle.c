@@ -19,7 +19,7 @@
  *                       per-node upper bounds confirmed by recounts from the definition
  *   o_count_pair / o_max_pair_recount   the Redundancy function of Algorithm 3
  *                       evaluated from its definition
- *   o6_max_forward / o6_max_backward    the element-wise max Aggregate of the GraphSAGE-P
+ *   o6_max_forward(_rows) / o6_max_backward    the element-wise max Aggregate of the GraphSAGE-P
  *                       row of Table 1, a_v = max over u in N(v) of z_u, straight
  *                       from the definition, and its gradient
  *   o7_hag_max_forward / o7_hag_max_backward   Algorithm 2 with max as the (associative,
@@ -171,6 +171,25 @@ void o6_max_forward(int64_t n, const int64_t *row_ptr, const int32_t *col, int64
 {
     for (int64_t v = 0; v < n; ++v) {
         double *o = out + v * d;
+        int64_t b = row_ptr[v], e = row_ptr[v + 1];
+        if (e == b) { for (int64_t k = 0; k < d; ++k) o[k] = 0.0; continue; }
+        const double *z0 = z + (int64_t)col[b] * d;
+        for (int64_t k = 0; k < d; ++k) o[k] = z0[k];
+        for (int64_t i = b + 1; i < e; ++i) {
+            const double *zu = z + (int64_t)col[i] * d;
+            for (int64_t k = 0; k < d; ++k) if (zu[k] > o[k]) o[k] = zu[k];
+        }
+    }
+}
+
+/* The same for a subset of the nodes: out is n_rows x d, row i holding a_v for v = rows[i]. */
+void o6_max_forward_rows(int64_t n, const int64_t *row_ptr, const int32_t *col, int64_t d,
+                         const double *z, const int64_t *rows, int64_t n_rows, double *out)
+{
+    (void)n;
+    for (int64_t r = 0; r < n_rows; ++r) {
+        int64_t v = rows[r];
+        double *o = out + r * d;
         int64_t b = row_ptr[v], e = row_ptr[v + 1];
         if (e == b) { for (int64_t k = 0; k < d; ++k) o[k] = 0.0; continue; }
         const double *z0 = z + (int64_t)col[b] * d;

@@ -92,6 +92,8 @@ def _c():
         lib.o4_hag_backward.restype = None
         lib.o6_max_forward.argtypes = [i64, p, p, i64, p, p]
         lib.o6_max_forward.restype = None
+        lib.o6_max_forward_rows.argtypes = [i64, p, p, i64, p, p, i64, p]
+        lib.o6_max_forward_rows.restype = None
         lib.o6_max_backward.argtypes = [i64, p, p, i64, p, p, p, p, p]
         lib.o6_max_backward.restype = None
         lib.o7_hag_max_forward.argtypes = [i64, i64, p, p, p, i64, p, p, p]
@@ -463,25 +465,45 @@ def hag_backward(h: CanonicalHag, g, reduce="sum"):
     return gx
 
 
-def direct_max_forward(row_ptr, col_idx, z):
-    """a_v = element-wise max over u in N(v) of z_u (zero row for an empty N(v)), fp64."""
+def direct_max_forward(row_ptr, col_idx, z, rows=None):
+    """a_v = element-wise max over u in N(v) of z_u (zero row for an empty N(v)), fp64.
+    ``rows``: optional subset of nodes; the result then has one row per entry."""
     rp, ci = _csr(row_ptr, col_idx)
     z = np.ascontiguousarray(z, dtype=np.float64)
-    out = np.empty_like(z)
-    _c().o6_max_forward(rp.shape[0] - 1, _ptr(rp), _ptr(ci), z.shape[1], _ptr(z), _ptr(out))
+    if rows is None:
+        out = np.empty_like(z)
+        _c().o6_max_forward(rp.shape[0] - 1, _ptr(rp), _ptr(ci), z.shape[1], _ptr(z), _ptr(out))
+        return out
+    sel = np.ascontiguousarray(rows, dtype=np.int64)
+    out = np.empty((sel.shape[0], z.shape[1]), dtype=np.float64)
+    _c().o6_max_forward_rows(rp.shape[0] - 1, _ptr(rp), _ptr(ci), z.shape[1], _ptr(z), _ptr(sel), sel.shape[0], _ptr(out))
     return out
 
 
-def direct_max_backward(row_ptr, col_idx, z, g):
+def direct_max_backward(row_ptr, col_idx, z, g, rows=None):
     """gz_u[k] = sum over v with u in N(v) and z_u[k] == a_v[k] of g_v[k].  Returns (gz, T),
-    T the same sum over |g| (the scale of the comparison tolerance)."""
+    T the same sum over |g| (the scale of the comparison tolerance).  ``rows``: optional subset of
+    source nodes u (one result row per entry): only the maxima of their out-neighbours are evaluated."""
     rp, ci = _csr(row_ptr, col_idx)
     z = np.ascontiguousarray(z, dtype=np.float64)
     g = np.ascontiguousarray(g, dtype=np.float64)
-    a = direct_max_forward(rp, ci, z)
-    gz = np.empty_like(z)
-    ab = np.empty_like(z)
-    _c().o6_max_backward(rp.shape[0] - 1, _ptr(rp), _ptr(ci), z.shape[1], _ptr(z), _ptr(a), _ptr(g), _ptr(gz), _ptr(ab))
+    if rows is None:
+        a = direct_max_forward(rp, ci, z)
+        gz = np.empty_like(z)
+        ab = np.empty_like(z)
+        _c().o6_max_backward(rp.shape[0] - 1, _ptr(rp), _ptr(ci), z.shape[1], _ptr(z), _ptr(a), _ptr(g), _ptr(gz), _ptr(ab))
+        return gz, ab
+    t_ptr, t_idx = transposed_csr(rp, ci)                      # out-neighbours v of every u, ascending
+    sel = np.asarray(rows, dtype=np.int64)
+    gz = np.zeros((sel.shape[0], z.shape[1]), dtype=np.float64)
+    ab = np.zeros_like(gz)
+    for i, u in enumerate(sel):
+        vs = t_idx[t_ptr[u]:t_ptr[u + 1]].astype(np.int64)
+        if vs.size == 0:
+            continue
+        hit = direct_max_forward(rp, ci, z, rows=vs) == z[u]   # v receives from u where u attains v's maximum
+        gz[i] = np.where(hit, g[vs], 0.0).sum(axis=0)
+        ab[i] = np.where(hit, np.abs(g[vs]), 0.0).sum(axis=0)
     return gz, ab
 
 

@@ -531,6 +531,11 @@ def test_max_matches_bruteforce_on_tiny_graphs(seed, ties):
     got, t = O.direct_max_backward(g.row_ptr, g.col_idx, z, gr)
     assert np.array_equal(got, gz)
     assert (t >= np.abs(got)).all()
+    # the row-subset forms used at full size: same loops over the definition, rows in any order
+    rows = rng.permutation(g.n)[: max(1, g.n // 2)]
+    assert np.array_equal(O.direct_max_forward(g.row_ptr, g.col_idx, z, rows=rows), a[rows])
+    sub, tsub = O.direct_max_backward(g.row_ptr, g.col_idx, z, gr, rows=rows)
+    assert np.array_equal(sub, gz[rows]) and np.array_equal(tsub, t[rows])
 
 
 def test_max_is_the_masked_dense_maximum_and_empty_rows_are_zero():
