@@ -64,7 +64,7 @@ typedef enum {
     HAG_ERR_DTYPE = 7,
     HAG_ERR_ALIGN = 8,       /* pointer or row size not 16-byte aligned                     */
     HAG_ERR_WORKSPACE = 9,   /* workspace missing although the HAG has aggregation nodes    */
-    HAG_ERR_TIMEOUT = 10,    /* reserved: a bounded device-side wait gave up                */
+    HAG_ERR_TIMEOUT = 10,    /* a bounded device-side wait gave up (see hag_device_status)  */
     HAG_ERR_NOT_ON_DEVICE = 11,/* hag_to_device has not been called                         */
     HAG_ERR_TOO_LARGE = 12     /* the problem needs more than the built-in scratch array holds */
 } hag_status;
@@ -192,9 +192,11 @@ hag_status hag_export(const hag_t *h, hag_arrays *out);
 hag_status hag_to_device(hag_t *h, int device);
 
 /* Bytes of workspace hag_aggregate_* need for feature width D: fp32 rows (whatever
- * the dtype) for the |V_A| aggregation nodes, plus one partial row per 128-entry
- * segment of the rows with more than 256 entries (such rows are summed by several
- * warps; the largest of the HAG's tables decides).  0 on bad arguments or when
+ * the dtype) for the |V_A| aggregation nodes, plus one partial row per segment of the
+ * rows that are summed by several warps.  Rows are split at one of three granularities,
+ * by the size of the launch or pass: more than 64 entries into segments of 32, more than
+ * 256 into 128, more than 1024 into 512; the table with the most segments decides.
+ * 0 on bad arguments or when
  * neither exists.  csr_workspace_bytes: the same for csr_aggregate_* (segments of
  * the input graph's long rows only; 0 for graphs without such rows). */
 size_t hag_workspace_bytes(const hag_t *h, int32_t D);
@@ -206,7 +208,7 @@ size_t csr_workspace_bytes(const hag_t *h, int32_t D);
  *   times 1/|N(v)| for HAG_MEAN (|N(v)| = in-degree in the input graph; an empty
  *   neighbourhood gives a zero row).
  * x and out are N x D of `dtype`, must not overlap; accumulation is fp32.
- * Enqueues 1 + (number of level launches) kernels on the stream.
+ * Enqueues 1 + (number of level launches) kernels on the stream (hag_set_schedule 1: one kernel).
  * Errors: NULL, ARG (D <= 0), DTYPE, ALIGN, WORKSPACE, NOT_ON_DEVICE, CUDA. */
 hag_status hag_aggregate_fwd(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D,
                              const void *x, void *out, void *workspace, void *cuda_stream);
@@ -251,7 +253,8 @@ hag_status hag_aggregate_host(hag_t *h, int backward, int use_hag, hag_reduce re
  * on the events of the LAST call and returns how many launches it made; for the
  * first `max` of them it fills ms[i] (device time), kind[i] (0 = level pair-sum,
  * 1 = gather over aggregation nodes: one level of the backward pass, or the
- * expanded deep levels of either pass, 2 = gather over the graph nodes), rows[i]
+ * expanded deep levels of either pass, 2 = gather over the graph nodes, 3 = a whole
+ * pass in one launch), rows[i]
  * (rows written) and edges[i] (source rows read).  A gather over a table with
  * split long rows is still one launch: segments and rows share it.
  * Arrays may be NULL.  Returns -1 on error. */
@@ -348,6 +351,62 @@ hag_status csr_max_bwd(const hag_t *h, hag_dtype dtype, int32_t D, const void *z
 #define HAG_STATIC_SCRATCH_BYTES (16u << 20)
 hag_status hag_aggregate_fwd_static(const hag_t *h, hag_reduce reduce, hag_dtype dtype, int32_t D,
                                     const void *x, void *out, void *cuda_stream);
+
+/* How a pass is scheduled on the device (no counterpart in the paper, which does not describe its kernels).
+ *   0 (default)  a launch per level: pair-sum kernels for the levels up to the cut, one gather for the expanded
+ *                deeper nodes, one gather for the graph nodes (hag_last_launch_count says how many).
+ *   1            ONE launch per pass.  Algorithm 2 only asks that every aggregation node comes after its
+ *                inputs and the graph nodes last.  The pass is a list of rows in that order -- one phase per
+ *                level evaluated pair by pair (rows of two entries), one for the expanded deeper nodes, the
+ *                graph-node rows last; a row too long for one warp is cut into chunk rows of a phase of their
+ *                own and becomes the short sum of their partial rows -- which resident warps take in list
+ *                order.  A row sums its entries from the layer input at once and waits, before it reads rows
+ *                of an earlier phase, until that phase's count of finished rows is complete.
+ *                The wait cannot deadlock (what it waits for was handed out earlier, to a running warp) and
+ *                is bounded anyway: after about a second of polling the warp records the failure and goes
+ *                on, the launch ends, and hag_device_status reports HAG_ERR_TIMEOUT (results of that call
+ *                are then undefined).  The plain-CSR calls use the same kernel (phases: chunk rows, rows).
+ *                Measured on B200 this form is level with the default on the two largest fp32 shapes and
+ *                slower on small graphs and deep hierarchies (resident warps hide less latency than the
+ *                hardware's block scheduling does on launches of 10^5 rows), which is why it is not the default.
+ * Passes whose hierarchy has more than 56 phases always run level by level.
+ * Errors: NULL; ARG (a value other than 0 or 1). */
+hag_status hag_set_schedule(hag_t *h, int32_t single_launch);
+
+/* HAG_OK, or HAG_ERR_TIMEOUT if a bounded device-side wait of an earlier call on this handle gave up
+ * (reading clears it).  Does not synchronise: call it after synchronising the stream of the calls
+ * in question.  Reads one word of pinned host memory that the kernels can write.
+ * Errors: NULL, NOT_ON_DEVICE. */
+hag_status hag_device_status(hag_t *h);
+
+/* Exercises the give-up path of that wait on purpose, safely: a launch of ONE thread block over a
+ * two-phase list of four rows whose first phase nobody ever finishes, with a poll limit of a few
+ * milliseconds.  The kernel must record the failure and end.  Synchronises the stream and returns what
+ * hag_device_status then says: HAG_ERR_TIMEOUT means the mechanism works, HAG_OK that it does not.
+ * Allocates a few hundred bytes with cudaMalloc for the call.  Errors: NULL, NOT_ON_DEVICE, OOM_DEVICE, CUDA. */
+hag_status hag_selftest_wait_limit(hag_t *h, void *cuda_stream);
+
+/* Borrowed HOST view of the row list of one pass (pass: 0 forward over the HAG, 1 backward over the HAG,
+ * 2 forward over the input graph, 3 backward over it), for inspection and checking.  rows: 4 int32 per row
+ * {b, e, row, phases}: the row sums the entries ids[b .. e) into output row `row` (row < 0: padding; row < n: a
+ * graph node; n <= row < n + |V_A|: an aggregation node; from n + |V_A| on: a chunk row, the fp32 partial sum of a
+ * piece of a long row, which a later short row adds up); phases = (phase that must be complete before the row
+ * reads, plus one; 0 = none) | (the row's own phase) << 8.  n_rows = 0: the pass has no list (it runs level by level). */
+typedef struct hag_pass_view {
+    int64_t n_rows, n_phases, n_chunk_rows, n_ids;
+    const int32_t *rows;        /* [4 * n_rows]  */
+    const int32_t *phase_size;  /* [n_phases] rows per phase, padding included */
+    const int32_t *ids;         /* [n_ids]       */
+} hag_pass_view;
+hag_status hag_export_pass(const hag_t *h, int32_t pass, hag_pass_view *out);
+
+/* Test hook (process-wide): makes one of the library's next allocation attempts fail as if memory had run out,
+ * so that callers can exercise their handling of HAG_ERR_OOM_HOST / HAG_ERR_OOM_DEVICE.  kind 0: host memory
+ * (the checked points are the start of the search, of the layout and of every array upload), 1: device memory
+ * (every array upload of hag_to_device).  countdown 0 fails the next attempt, 1 the one after it, ...; a
+ * negative value switches the hook off.  The failing call frees what it had built and returns the status;
+ * nothing is left half-made, and no GPU work is involved.  Errors: ARG (kind). */
+hag_status hag_test_fail_allocation(int32_t kind, int32_t countdown);
 
 /* Number of kernels the last aggregate call on this handle enqueued. */
 int32_t hag_last_launch_count(const hag_t *h);

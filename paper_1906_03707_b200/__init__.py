@@ -30,6 +30,7 @@ EXPORTED_SYMBOLS = [
     "hag_aggregate_fwd", "hag_aggregate_bwd", "csr_aggregate_fwd", "csr_aggregate_bwd",
     "hag_aggregate_host", "hag_aggregate_fwd_static", "hag_graph_pool_fwd", "hag_graph_pool_bwd",
     "hag_max_workspace_bytes", "hag_max_fwd", "hag_max_bwd", "csr_max_fwd", "csr_max_bwd", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
+    "hag_set_schedule", "hag_device_status", "hag_selftest_wait_limit", "hag_export_pass", "hag_test_fail_allocation",
 ]
 
 
@@ -53,6 +54,11 @@ class HagInfo(ctypes.Structure):
 
     def as_dict(self) -> dict:
         return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class HagPassView(ctypes.Structure):
+    _fields_ = [(k, ctypes.c_int64) for k in ("n_rows", "n_phases", "n_chunk_rows", "n_ids")] + [
+        (k, ctypes.c_void_p) for k in ("rows", "phase_size", "ids")]
 
 
 class HagArrays(ctypes.Structure):
@@ -126,6 +132,16 @@ def load_library():
     lib.hag_profile_read.restype = i32
     lib.hag_last_launch_count.argtypes = [vp]
     lib.hag_last_launch_count.restype = i32
+    lib.hag_set_schedule.argtypes = [vp, i32]
+    lib.hag_set_schedule.restype = ctypes.c_int
+    lib.hag_device_status.argtypes = [vp]
+    lib.hag_device_status.restype = ctypes.c_int
+    lib.hag_selftest_wait_limit.argtypes = [vp, vp]
+    lib.hag_selftest_wait_limit.restype = ctypes.c_int
+    lib.hag_export_pass.argtypes = [vp, i32, ctypes.POINTER(HagPassView)]
+    lib.hag_export_pass.restype = ctypes.c_int
+    lib.hag_test_fail_allocation.argtypes = [i32, i32]
+    lib.hag_test_fail_allocation.restype = ctypes.c_int
     lib.hag_status_str.argtypes = [ctypes.c_int]
     lib.hag_status_str.restype = ctypes.c_char_p
     _lib = lib
@@ -239,6 +255,22 @@ class Hag:
             trace=_view(a.trace, 3 * k, np.int32).reshape(-1, 3),
             csr_t_ptr=csr_t_ptr, csr_t_idx=_view(a.csr_t_idx, int(csr_t_ptr[-1]) if csr_t_ptr.size else 0, np.int32),
         )
+
+    def pass_rows(self, which: int) -> dict:
+        """``hag_export_pass``: copies of the row list of one pass (0 fwd, 1 bwd, 2 plain fwd, 3 plain bwd)."""
+        v = HagPassView()
+        _check(load_library().hag_export_pass(self._h, int(which), ctypes.byref(v)), "hag_export_pass")
+        return dict(rows=_view(v.rows, 4 * v.n_rows, np.int32).reshape(-1, 4), phase_size=_view(v.phase_size, v.n_phases, np.int32),
+                    ids=_view(v.ids, v.n_ids, np.int32), n_chunk_rows=int(v.n_chunk_rows))
+
+    def set_schedule(self, single_launch: bool) -> "Hag":
+        """``hag_set_schedule``: a launch per level (default) or one launch per pass."""
+        _check(load_library().hag_set_schedule(self._h, int(bool(single_launch))), "hag_set_schedule")
+        return self
+
+    def device_status(self) -> int:
+        """``hag_device_status``: 0, or HAG_ERR_TIMEOUT if a device-side wait gave up (call after synchronising)."""
+        return int(load_library().hag_device_status(self._h))
 
     def workspace_bytes(self, d: int) -> int:
         return int(load_library().hag_workspace_bytes(self._h, int(d)))

@@ -21,6 +21,7 @@
 // by a pool of threads at once.  Recounting a stale node early only tightens a
 // bound sooner: the merge sequence is the same for any number of threads.
 #include <algorithm>
+#include <limits>
 #include <atomic>
 #include <chrono>
 #include <cstring>
@@ -311,8 +312,26 @@ struct Searcher {
 
 }  // namespace
 
+namespace {
+std::atomic<int> g_fail_countdown[2] = {{-1}, {-1}};
+}
+
+bool hag_alloc_should_fail(int kind) {
+    int v = g_fail_countdown[kind].load();
+    while (v >= 0)
+        if (g_fail_countdown[kind].compare_exchange_weak(v, v - 1)) return v == 0;
+    return false;
+}
+
+extern "C" hag_status hag_test_fail_allocation(int32_t kind, int32_t countdown) {
+    if (kind != 0 && kind != 1) return HAG_ERR_ARG;
+    g_fail_countdown[kind].store(countdown < 0 ? -1 : countdown);
+    return HAG_OK;
+}
+
 hag_status hag_search(hag *h, std::vector<int32_t> &rows_store, std::vector<int32_t> &rows_len) {
     try {
+        if (hag_alloc_should_fail(0)) throw std::bad_alloc();
         rows_store = h->csr_idx;
         rows_len.resize(h->n);
         for (int32_t u = 0; u < h->n; ++u) rows_len[u] = int32_t(h->csr_ptr[u + 1] - h->csr_ptr[u]);
@@ -471,10 +490,192 @@ void build_segments(hag *h) {
     h->max_segs_csr = std::max(h->seg_csr.max_count(), h->seg_csr_t.max_count());
 }
 
+
+// The four passes as row lists for the single-launch kernel (see hag_internal.h).
+// How long a row may get before it is cut into chunk rows, by the size of the pass: a pass that cannot keep
+// the machine busy for long must not end on one warp walking a hub row.
+struct FusedSplit { int64_t long_row, chunk_len; };
+FusedSplit fused_split_for_entries(int64_t entries) {
+    if (entries < (int64_t(1) << 20)) return {64, 32};
+    if (entries < (int64_t(16) << 20)) return {128, 64};
+    return {1024, 512};
+}
+
+struct FusedBuilder {
+    fused_table &t;
+    const int32_t n, k;                 // graph nodes, aggregation nodes: chunk rows get the ids n + k, n + k + 1, ...
+    const FusedSplit split;
+    int32_t phase = -1;
+    int64_t phase_begin = 0;
+    FusedBuilder(fused_table &t_, int32_t n_, int32_t k_, FusedSplit sp) : t(t_), n(n_), k(k_), split(sp) { t = fused_table{}; }
+    // n_sec: how many of the row's entries (its last ones) are rows that this launch writes: read after the wait
+    void push(int64_t b, int64_t e, int32_t row, int req, int64_t n_sec = 0) {
+        t.items.push_back(int32_t(b));
+        t.items.push_back(int32_t(e));
+        t.items.push_back(row);
+        t.items.push_back(int32_t(uint32_t(req + 1) | (uint32_t(phase) << 8) | (uint32_t(req >= 0 ? n_sec : 0) << 16)));
+    }
+    // Rows per grab of four list slots, by the size of the phase: a phase that gives every resident warp only a
+    // few grabs is handed out one row at a time (the other three slots are padding), or it would end on warps that
+    // still have three rows to go while the rest wait for the phase to complete.
+    int real_per_grab = kFusedItemsPerGrab, in_grab = 0;
+    void begin_phase(int64_t rows = -1) {
+        ++phase;
+        phase_begin = t.n_items();
+        in_grab = 0;
+        real_per_grab = rows < 0 || rows >= kFusedRowsForFullGrabs ? 4 : (rows >= kFusedRowsForFullGrabs / 4 ? 2 : 1);
+    }
+    void push_row(int64_t b, int64_t e, int32_t row, int req, int64_t n_sec) {
+        push(b, e, row, req, n_sec);
+        if (++in_grab == real_per_grab) {
+            while (t.n_items() % kFusedItemsPerGrab) push(0, 0, -1, -1);
+            in_grab = 0;
+        }
+    }
+    void end_phase() {
+        while ((t.n_items() - phase_begin) % kFusedItemsPerGrab) push(0, 0, -1, -1);
+        t.phase_size.push_back(int32_t(t.n_items() - phase_begin));
+    }
+    // Appends `ids` to the pass's id list and returns where they start.
+    int64_t add_ids(const int32_t *ids, int64_t count) {
+        const int64_t at = int64_t(t.ids.size());
+        t.ids.insert(t.ids.end(), ids, ids + count);
+        return at;
+    }
+    // One logical phase of rows: row r (output id first_row + r) sums the entries [ptr[r0 + r], ptr[r0 + r + 1]) of the
+    // id list, which start at `at` in the pass's list and ascend within a row.  need(b, e) = the phase that must be
+    // complete before the entries [b, e) may be read, or -1.  Rows longer than split.long_row are cut: their chunk
+    // rows form a phase of their own, placed first, and the row itself becomes a short row over the chunks' partial rows.
+    // Returns the index of the phase that holds the rows themselves.
+    template <typename Need>
+    int32_t rows_phase(const std::vector<int64_t> &ptr, int64_t r0, int64_t count, int32_t first_row, int64_t at, Need need) {
+        const int64_t shift = at - ptr[r0];
+        // entries of the pass's list in [b, e) that are not rows of the layer input (ids ascend within a row)
+        auto n_sec_of = [&](int64_t b, int64_t e) {
+            return int64_t((t.ids.data() + e) - std::lower_bound(t.ids.data() + b, t.ids.data() + e, n));
+        };
+        std::vector<int64_t> chunk_first;        // per long row: id of its first chunk row
+        bool any_long = false;
+        for (int64_t r = 0; r < count && !any_long; ++r) any_long = ptr[r0 + r + 1] - ptr[r0 + r] > split.long_row;
+        int32_t chunk_phase = -1;
+        if (any_long) {
+            int64_t n_chunk_rows = 0;
+            for (int64_t r = 0; r < count; ++r) {
+                const int64_t len = ptr[r0 + r + 1] - ptr[r0 + r];
+                if (len > split.long_row) n_chunk_rows += (len + split.chunk_len - 1) / split.chunk_len;
+            }
+            begin_phase(n_chunk_rows);
+            chunk_phase = phase;
+            for (int64_t r = 0; r < count; ++r) {
+                const int64_t b = ptr[r0 + r], e = ptr[r0 + r + 1];
+                if (e - b <= split.long_row) continue;
+                chunk_first.push_back(int64_t(n) + k + t.n_chunks);
+                for (int64_t cb = b; cb < e; cb += split.chunk_len) {
+                    const int64_t ce = std::min<int64_t>(cb + split.chunk_len, e);
+                    push_row(cb + shift, ce + shift, int32_t(int64_t(n) + k + t.n_chunks++), need(cb, ce), n_sec_of(cb + shift, ce + shift));
+                }
+            }
+            end_phase();
+        }
+        begin_phase(count);
+        size_t li = 0;
+        for (int64_t r = 0; r < count; ++r) {
+            const int64_t b = ptr[r0 + r], e = ptr[r0 + r + 1];
+            if (e - b <= split.long_row) {
+                push_row(b + shift, e + shift, int32_t(first_row + r), need(b, e), n_sec_of(b + shift, e + shift));
+            } else {                             // the sum of its chunks' partial rows
+                const int64_t n_chunk = (e - b + split.chunk_len - 1) / split.chunk_len;
+                const int64_t eb = int64_t(t.ids.size());
+                for (int64_t c = 0; c < n_chunk; ++c) t.ids.push_back(int32_t(chunk_first[li] + c));
+                ++li;
+                push_row(eb, eb + n_chunk, int32_t(first_row + r), chunk_phase, n_chunk);
+            }
+        }
+        end_phase();
+        return phase;
+    }
+    void finish() {
+        t.last_phase = phase;
+        t.ok = phase >= 0 && phase < kFusedMaxPhases && t.n_items() > 0 && t.n_items() < (int64_t(1) << 30) &&
+               t.ids.size() < (size_t(1) << 31) && int64_t(n) + k + t.n_chunks < (int64_t(1) << 31);
+        if (!t.ok) {
+            t.items.clear();
+            t.phase_size.clear();
+            t.n_chunks = 0;
+        }
+    }
+};
+
+void build_fused(hag *h) {
+    const int32_t n = h->n, k = h->num_agg, L = h->num_levels;
+    std::vector<int32_t> clevel(k);
+    for (int32_t l = 1; l <= L; ++l)
+        for (int64_t j = h->level_ptr[l - 1]; j < h->level_ptr[l]; ++j) clevel[j] = l;
+    auto level_of = [&](int32_t id) { return id < n ? 0 : clevel[id - n]; };
+    std::vector<int32_t> phase_of_level(size_t(L) + 2, -1);      // phase that writes the rows of a level (forward: L + 1 = deeper than the cut)
+    {   // forward over the HAG: levels 1..fwd_cut as rows of two entries, the expanded deeper nodes, the graph nodes
+        const int32_t c = h->fwd_cut;
+        const int64_t j0 = h->level_ptr[c];
+        FusedBuilder fb(h->fz_fwd, n, k, fused_split_for_entries(h->e_res + int64_t(h->ftail_idx.size())));
+        auto phase_of = [&](int32_t id) { const int32_t l = level_of(id); return l == 0 ? -1 : phase_of_level[l <= c ? l : c + 1]; };
+        // ids ascend within a list and aggregation nodes are sorted by level: the last entry is written by the latest phase
+        const std::vector<int32_t> *src = &h->agg_in;
+        auto need = [&](int64_t b, int64_t e) { return e > b ? phase_of((*src)[e - 1]) : -1; };
+        std::vector<int64_t> pair_ptr(size_t(j0) + 1);
+        for (int64_t j = 0; j <= j0; ++j) pair_ptr[j] = 2 * j;
+        const int64_t at_pairs = fb.add_ids(h->agg_in.data(), 2 * j0);
+        for (int32_t l = 1; l <= c; ++l)
+            phase_of_level[l] = fb.rows_phase(pair_ptr, h->level_ptr[l - 1], h->level_ptr[l] - h->level_ptr[l - 1],
+                                              int32_t(n + h->level_ptr[l - 1]), at_pairs + 2 * h->level_ptr[l - 1], need);
+        h->fz_fwd.off_head = fb.add_ids(h->ftail_idx.data(), int64_t(h->ftail_idx.size()));
+        src = &h->ftail_idx;
+        if (j0 < k) phase_of_level[c + 1] = fb.rows_phase(h->ftail_ptr, 0, k - j0, int32_t(n + j0), h->fz_fwd.off_head, need);
+        h->fz_fwd.off_tail = fb.add_ids(h->res_idx.data(), h->e_res);
+        src = &h->res_idx;
+        if (n > 0) fb.rows_phase(h->res_ptr, 0, n, 0, h->fz_fwd.off_tail, need);
+        fb.finish();
+    }
+    {   // backward over the HAG: the expanded deep nodes, levels bwd_cut..1, the graph nodes as sources
+        const int32_t c = h->bwd_cut;
+        const int64_t j0 = h->level_ptr[c];
+        FusedBuilder fb(h->fz_bwd, n, k, fused_split_for_entries(h->e_hat + int64_t(h->btail_idx.size())));
+        std::fill(phase_of_level.begin(), phase_of_level.end(), -1);
+        auto phase_of = [&](int32_t id) { const int32_t l = level_of(id); return l == 0 ? -1 : phase_of_level[l <= c ? l : c + 1]; };
+        // destinations ascend: the first aggregation node among them is the shallowest, i.e. the one written by the latest phase
+        auto need = [&](int64_t b, int64_t e) {
+            const int32_t *lo = std::lower_bound(h->t_idx.data() + b, h->t_idx.data() + e, n);
+            return lo < h->t_idx.data() + e ? phase_of(*lo) : -1;
+        };
+        h->fz_bwd.off_head = fb.add_ids(h->btail_idx.data(), int64_t(h->btail_idx.size()));
+        if (j0 < k) phase_of_level[c + 1] = fb.rows_phase(h->btail_ptr, 0, k - j0, int32_t(n + j0), h->fz_bwd.off_head,
+                                                          [](int64_t, int64_t) { return -1; });     // all sources are graph-node outputs
+        h->fz_bwd.off_tail = fb.add_ids(h->t_idx.data(), h->e_hat);
+        for (int32_t l = c; l >= 1; --l)
+            phase_of_level[l] = fb.rows_phase(h->t_ptr, int64_t(n) + h->level_ptr[l - 1], h->level_ptr[l] - h->level_ptr[l - 1],
+                                              int32_t(n + h->level_ptr[l - 1]), h->fz_bwd.off_tail + h->t_ptr[size_t(n) + h->level_ptr[l - 1]], need);
+        if (n > 0) fb.rows_phase(h->t_ptr, 0, n, 0, h->fz_bwd.off_tail, need);
+        fb.finish();
+    }
+    {   // the input graph and its transpose: nothing to wait for but the chunks of long rows (k = 0: their ids start at n)
+        auto none = [](int64_t, int64_t) { return -1; };
+        FusedBuilder fb(h->fz_csr, n, 0, fused_split_for_entries(h->e));
+        h->fz_csr.off_tail = fb.add_ids(h->csr_idx.data(), h->e);
+        if (n > 0) fb.rows_phase(h->csr_ptr, 0, n, 0, 0, none);
+        fb.finish();
+        FusedBuilder ft(h->fz_csr_t, n, 0, fused_split_for_entries(h->e));
+        h->fz_csr_t.off_tail = ft.add_ids(h->csr_t_idx.data(), h->e);
+        if (n > 0) ft.rows_phase(h->csr_t_ptr, 0, n, 0, 0, none);
+        ft.finish();
+    }
+    h->max_segs_hag = std::max(h->max_segs_hag, std::max(h->fz_fwd.n_chunks, h->fz_bwd.n_chunks));
+    h->max_segs_csr = std::max(h->max_segs_csr, std::max(h->fz_csr.n_chunks, h->fz_csr_t.n_chunks));
+}
+
 }  // namespace
 
 hag_status hag_layout(hag *h, const std::vector<int32_t> &rows_store, const std::vector<int32_t> &rows_len) {
     try {
+        if (hag_alloc_should_fail(0)) throw std::bad_alloc();
         const int32_t n = h->n, k = h->num_agg;
         // level = 1 + the larger level of the two inputs (graph nodes are level 0)
         std::vector<int32_t> level(size_t(n) + k, 0);
@@ -551,6 +752,7 @@ hag_status hag_layout(hag *h, const std::vector<int32_t> &rows_store, const std:
         choose_cuts(h, fwd_cut, bwd_cut);
         expand_tails(h, fwd_cut, bwd_cut);
         build_segments(h);
+        build_fused(h);
         // counters of the cost function
         hag_info &f = h->info;
         f = hag_info{};
@@ -651,6 +853,7 @@ extern "C" hag_status hag_set_cuts(hag_t *h, int32_t fwd_cut, int32_t bwd_cut) {
         if (fwd_cut < 0 || bwd_cut < 0) choose_cuts(h, f, b);
         expand_tails(h, fwd_cut < 0 ? f : fwd_cut, bwd_cut < 0 ? b : bwd_cut);
         build_segments(h);
+        build_fused(h);
     } catch (const std::bad_alloc &) {
         return HAG_ERR_OOM_HOST;
     }
@@ -725,6 +928,22 @@ extern "C" hag_status hag_export(const hag_t *h, hag_arrays *out) {
     out->ftail_idx = h->ftail_idx.data();
     out->btail_ptr = h->btail_ptr.data();
     out->btail_idx = h->btail_idx.data();
+    return HAG_OK;
+}
+
+extern "C" hag_status hag_export_pass(const hag_t *h, int32_t pass, hag_pass_view *out) {
+    if (!h || !out) return HAG_ERR_NULL;
+    if (pass < 0 || pass > 3) return HAG_ERR_ARG;
+    const fused_table &t = pass == 0 ? h->fz_fwd : (pass == 1 ? h->fz_bwd : (pass == 2 ? h->fz_csr : h->fz_csr_t));
+    *out = hag_pass_view{};
+    if (!t.ok) return HAG_OK;
+    out->n_rows = t.n_items();
+    out->n_phases = int64_t(t.phase_size.size());
+    out->n_chunk_rows = t.n_chunks;
+    out->n_ids = int64_t(t.ids.size());
+    out->rows = t.items.data();
+    out->phase_size = t.phase_size.data();
+    out->ids = t.ids.data();
     return HAG_OK;
 }
 

@@ -32,11 +32,13 @@ template <typename V>
 hag_status upload_i32(int32_t **dst, const V *src, size_t count) {
     std::vector<int32_t> tmp;
     try {
+        if (hag_alloc_should_fail(0)) throw std::bad_alloc();
         tmp.resize(std::max<size_t>(count, 1));
     } catch (const std::bad_alloc &) {
         return HAG_ERR_OOM_HOST;
     }
     for (size_t i = 0; i < count; ++i) tmp[i] = int32_t(src[i]);
+    if (hag_alloc_should_fail(1)) return HAG_ERR_OOM_DEVICE;         // test hook: as if cudaMalloc had no memory left
     cudaError_t err = cudaMalloc(reinterpret_cast<void **>(dst), tmp.size() * sizeof(int32_t));
     if (err == cudaErrorMemoryAllocation) { cudaGetLastError(); return HAG_ERR_OOM_DEVICE; }
     if (err != cudaSuccess) { cudaGetLastError(); return HAG_ERR_CUDA; }
@@ -59,6 +61,12 @@ void free_device(hag *h) {
         t->d_segs = t->d_slots = nullptr;
         t->d_done = nullptr;
     }
+    for (fused_table *t : {&h->fz_fwd, &h->fz_bwd, &h->fz_csr, &h->fz_csr_t})
+        for (int32_t **p : {&t->d_items, &t->d_phase_size, &t->d_ids})
+            if (*p) { cudaFree(*p); *p = nullptr; }
+    if (d.err_host) cudaFreeHost(d.err_host);
+    // these point into the id lists freed above
+    d.res_idx = d.ftail_idx = d.t_idx = d.btail_idx = d.csr_idx = d.csr_t_idx = nullptr;
     if (d.copy_in_stream) {
         cudaStreamSynchronize(d.copy_in_stream);
         cudaStreamDestroy(d.copy_in_stream);
@@ -69,7 +77,7 @@ void free_device(hag *h) {
     }
     void *ptrs[] = {d.agg_in, d.res_ptr, d.res_idx, d.t_ptr, d.t_idx, d.csr_ptr, d.csr_idx, d.csr_t_ptr,
                     d.csr_t_idx, d.inv_degree, d.inv_degree1, d.stage_in, d.stage_in2, d.stage_out, d.stage_ws,
-                    d.ftail_ptr, d.ftail_idx, d.btail_ptr, d.btail_idx, d.sched};
+                    d.ftail_ptr, d.ftail_idx, d.btail_ptr, d.btail_idx, d.sched, d.fused_ctl};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     d = hag_device_arrays{};
@@ -156,7 +164,9 @@ cudaError_t launch_gather_shape(const hagk::GatherArgs &ga, const hagk::SegArgs 
         if constexpr (SS) return launch_pdl(plain_kernel<T, LPR, 4, SS, 8, SEGS, SELF>(), grid, a, s);
         return launch_pdl(plain_kernel<T, LPR, 4, SS, 10, SEGS, SELF>(), grid, a, s);
     } else {
-        return launch_pdl(plain_kernel<T, LPR, 2, SS, 12, SEGS, SELF>(), grid, a, s);
+        // bf16 rows are fetched as raw words and widened as they are added: four loads in flight fit the 40 registers of
+        // 12 CTAs per SM (sweep on B200: 4 x 12 beats 2 x 12, 4 x 10, 8 x 8, 4 x 8 and resident warps)
+        return launch_pdl(plain_kernel<T, LPR, 4, SS, 12, SEGS, SELF>(), grid, a, s);
     }
 }
 
@@ -221,6 +231,53 @@ cudaError_t launch_pairs(const hagk::PairArgs &p, int n_chunks, cudaStream_t s) 
         case 16: return launch_pdl(hagk::pair_sum_kernel<T, 16>, grid, p, s);
         default: return launch_pdl(hagk::pair_sum_kernel<T, 32>, grid, p, s);
     }
+}
+
+// One pass as one launch (fused_pass_kernel): exactly as many CTAs as stay resident.
+template <typename T, int LPR, bool SS, bool SELF>
+cudaError_t launch_fused_shape(const hagk::FusedArgs &k, int sm_count, cudaStream_t s) {
+    const int64_t warps = (int64_t(k.n_items) + kFusedItemsPerGrab - 1) / kFusedItemsPerGrab;
+    if constexpr (sizeof(T) == 4) {
+        if constexpr (LPR == 32 && !SS) return launch_persistent(hagk::fused_pass_kernel<T, LPR, 8, SS, 8, SELF>, k, warps, sm_count, s);
+        return launch_persistent(hagk::fused_pass_kernel<T, LPR, 4, SS, 8, SELF>, k, warps, sm_count, s);
+    } else {
+        return launch_persistent(hagk::fused_pass_kernel<T, LPR, 2, SS, 10, SELF>, k, warps, sm_count, s);
+    }
+}
+
+template <typename T>
+cudaError_t launch_fused(const hag *h, const fused_table &t, hagk::GatherArgs a, float *ahat, int n_chunks, cudaStream_t s) {
+    hagk::FusedArgs k{};
+    a.idx = t.d_ids;
+    a.row_ptr = nullptr;
+    a.row_begin = 0;
+    a.row_count = 0;
+    a.sec = ahat;
+    a.n_prim = h->n;           // ids from n on: aggregation nodes, then the chunk rows of this pass
+    k.a = a;
+    k.items = reinterpret_cast<const int4 *>(t.d_items);
+    k.n_items = int32_t(t.n_items());
+    k.last_phase = t.last_phase;
+    k.phase_size = t.d_phase_size;
+    hag *hm = const_cast<hag *>(h);
+    k.ctl = h->d.fused_ctl + size_t(kFusedCtlWords) * (hm->fused_seq++ % kFusedCtlSlots);
+    k.ahat = ahat;
+    k.err_host = h->d.err_dev;
+    k.spin_limit = h->spin_limit;
+    const int lpr = lanes_per_row(n_chunks);
+    const bool ss = a.src_scale != nullptr, self = (a.out_is_f32 & 2) != 0;
+#define HAG_FUSED_CASE(L)                                                                                          \
+    case L:                                                                                                        \
+        if (ss) return self ? launch_fused_shape<T, L, true, true>(k, h->sm_count, s) : launch_fused_shape<T, L, true, false>(k, h->sm_count, s); \
+        return self ? launch_fused_shape<T, L, false, true>(k, h->sm_count, s) : launch_fused_shape<T, L, false, false>(k, h->sm_count, s);
+    switch (lpr) {
+        HAG_FUSED_CASE(4)
+        HAG_FUSED_CASE(8)
+        HAG_FUSED_CASE(16)
+        default:
+        HAG_FUSED_CASE(32)
+    }
+#undef HAG_FUSED_CASE
 }
 
 // Brackets each launch with an event pair when profiling is on; always counts launches.
@@ -325,6 +382,13 @@ hag_status fwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
     a.n_prim = std::numeric_limits<int32_t>::max();
     // workspace layout: rows of the aggregation nodes (HAG calls only), then the partial rows of long-row segments
     float *partial = static_cast<float *>(ws) + (use_hag ? size_t(h->num_agg) * D : 0);
+    const fused_table &fz = use_hag ? h->fz_fwd : h->fz_csr;
+    if (h->schedule == 1 && fz.ok) {       // the whole pass in one launch; the plain graph's chunk rows start at ws row 0
+        if (rec) rec->begin(3, int64_t(h->n) + (use_hag ? h->num_agg : 0), use_hag ? h->e_hat : h->e);
+        if (launch_fused<T>(h, fz, a, static_cast<float *>(ws), n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+        if (rec) rec->end();
+        return HAG_OK;
+    }
     if (use_hag) {
         if (h->num_agg > 0) {
             hag_status st = enqueue_fwd_agg<T>(h, D, x, static_cast<float *>(ws), partial, s, rec);
@@ -363,6 +427,15 @@ hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
     a.D = D;
     a.n_prim = std::numeric_limits<int32_t>::max();
     float *partial = static_cast<float *>(ws) + (use_hag ? size_t(h->num_agg) * D : 0);
+    const fused_table &fz = use_hag ? h->fz_bwd : h->fz_csr_t;
+    if (h->schedule == 1 && fz.ok) {       // the whole pass in one launch
+        a.out = gx;
+        a.out_is_f32 = (reduce == HAG_GCN) ? 2 : 0;
+        if (rec) rec->begin(3, int64_t(h->n) + (use_hag ? h->num_agg : 0), use_hag ? h->e_hat : h->e);
+        if (launch_fused<T>(h, fz, a, static_cast<float *>(ws), n_chunks, s) != cudaSuccess) return HAG_ERR_CUDA;
+        if (rec) rec->end();
+        return HAG_OK;
+    }
     if (use_hag && h->num_agg > 0) {
         const int32_t j0 = int32_t(h->level_ptr[h->bwd_cut]);
         if (j0 < h->num_agg) {
@@ -477,17 +550,24 @@ extern "C" hag_status hag_to_device(hag_t *h, int device) {
     const size_t n = size_t(h->n), k = size_t(h->num_agg);
     if (st == HAG_OK) st = upload_i32(&d.agg_in, h->agg_in.data(), 2 * k);
     if (st == HAG_OK) st = upload_i32(&d.res_ptr, h->res_ptr.data(), n + 1);
-    if (st == HAG_OK) st = upload_i32(&d.res_idx, h->res_idx.data(), size_t(h->e_res));
+    // the id lists of the four passes: row lists and expansion lists are parts of them
+    if (st == HAG_OK) st = upload_i32(&h->fz_fwd.d_ids, h->fz_fwd.ids.data(), h->fz_fwd.ids.size());
+    if (st == HAG_OK) st = upload_i32(&h->fz_bwd.d_ids, h->fz_bwd.ids.data(), h->fz_bwd.ids.size());
+    if (st == HAG_OK) st = upload_i32(&h->fz_csr.d_ids, h->fz_csr.ids.data(), h->fz_csr.ids.size());
+    if (st == HAG_OK) st = upload_i32(&h->fz_csr_t.d_ids, h->fz_csr_t.ids.data(), h->fz_csr_t.ids.size());
+    if (st == HAG_OK) {
+        d.ftail_idx = h->fz_fwd.d_ids + h->fz_fwd.off_head;
+        d.res_idx = h->fz_fwd.d_ids + h->fz_fwd.off_tail;
+        d.btail_idx = h->fz_bwd.d_ids + h->fz_bwd.off_head;
+        d.t_idx = h->fz_bwd.d_ids + h->fz_bwd.off_tail;
+        d.csr_idx = h->fz_csr.d_ids + h->fz_csr.off_tail;
+        d.csr_t_idx = h->fz_csr_t.d_ids + h->fz_csr_t.off_tail;
+    }
     if (st == HAG_OK) st = upload_i32(&d.t_ptr, h->t_ptr.data(), n + k + 1);
-    if (st == HAG_OK) st = upload_i32(&d.t_idx, h->t_idx.data(), size_t(h->e_hat));
     if (st == HAG_OK) st = upload_i32(&d.csr_ptr, h->csr_ptr.data(), n + 1);
-    if (st == HAG_OK) st = upload_i32(&d.csr_idx, h->csr_idx.data(), size_t(h->e));
     if (st == HAG_OK) st = upload_i32(&d.csr_t_ptr, h->csr_t_ptr.data(), n + 1);
-    if (st == HAG_OK) st = upload_i32(&d.csr_t_idx, h->csr_t_idx.data(), size_t(h->e));
     if (st == HAG_OK) st = upload_i32(&d.ftail_ptr, h->ftail_ptr.data(), h->ftail_ptr.size());
-    if (st == HAG_OK) st = upload_i32(&d.ftail_idx, h->ftail_idx.data(), h->ftail_idx.size());
     if (st == HAG_OK) st = upload_i32(&d.btail_ptr, h->btail_ptr.data(), h->btail_ptr.size());
-    if (st == HAG_OK) st = upload_i32(&d.btail_idx, h->btail_idx.data(), h->btail_idx.size());
     if (st == HAG_OK) {
         std::vector<float> inv(std::max<size_t>(n, 1), 1.0f), inv1(std::max<size_t>(n, 1), 1.0f);
         for (size_t v = 0; v < n; ++v) {
@@ -525,6 +605,25 @@ extern "C" hag_status hag_to_device(hag_t *h, int device) {
             cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
             cudaGetLastError();
             st = HAG_ERR_CUDA;
+        }
+    }
+    for (fused_table *t : {&h->fz_fwd, &h->fz_bwd, &h->fz_csr, &h->fz_csr_t}) {
+        if (st != HAG_OK || !t->ok) continue;
+        st = upload_i32(&t->d_items, t->items.data(), t->items.size());
+        if (st == HAG_OK) st = upload_i32(&t->d_phase_size, t->phase_size.data(), t->phase_size.size());
+    }
+    if (st == HAG_OK) {
+        const size_t bytes = size_t(kFusedCtlSlots) * kFusedCtlWords * sizeof(unsigned int);
+        if (cudaMalloc(reinterpret_cast<void **>(&d.fused_ctl), bytes) != cudaSuccess || cudaMemset(d.fused_ctl, 0, bytes) != cudaSuccess ||
+            cudaHostAlloc(reinterpret_cast<void **>(&d.err_host), sizeof(unsigned int), cudaHostAllocMapped) != cudaSuccess) {
+            cudaGetLastError();
+            st = HAG_ERR_CUDA;
+        } else {
+            *d.err_host = 0;
+            if (cudaHostGetDevicePointer(reinterpret_cast<void **>(&d.err_dev), d.err_host, 0) != cudaSuccess) {
+                cudaGetLastError();
+                st = HAG_ERR_CUDA;
+            }
         }
     }
     if (st != HAG_OK) {
@@ -613,6 +712,75 @@ extern "C" hag_status hag_aggregate_host(hag_t *h, int backward, int use_hag, ha
 }
 
 extern "C" int32_t hag_last_launch_count(const hag_t *h) { return h ? h->last_launches : 0; }
+
+extern "C" hag_status hag_set_schedule(hag_t *h, int32_t single_launch) {
+    if (!h) return HAG_ERR_NULL;
+    if (single_launch != 0 && single_launch != 1) return HAG_ERR_ARG;
+    h->schedule = single_launch;
+    return HAG_OK;
+}
+
+extern "C" hag_status hag_device_status(hag_t *h) {
+    if (!h) return HAG_ERR_NULL;
+    if (h->device < 0 || !h->d.err_host) return HAG_ERR_NOT_ON_DEVICE;
+    volatile unsigned int *w = h->d.err_host;
+    if (*w == 0) return HAG_OK;
+    *w = 0;
+    return HAG_ERR_TIMEOUT;
+}
+
+// A one-CTA launch of the single-launch kernel over a two-phase list whose first phase is never
+// finished by anybody: the one row item must run out of polls, record it, and still end.
+extern "C" hag_status hag_selftest_wait_limit(hag_t *h, void *cuda_stream) {
+    if (!h) return HAG_ERR_NULL;
+    if (h->device < 0) return HAG_ERR_NOT_ON_DEVICE;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) { cudaGetLastError(); return HAG_ERR_CUDA; }
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    constexpr int D = 4;
+    struct Blob {
+        int32_t items[16];
+        int32_t phase_size[4];
+        int32_t idx[4];
+        unsigned int ctl[kFusedCtlWords];
+        float prim[D], sec[D], out[D];
+    } host{};
+    const int32_t row_item[4] = {0, 1, 0, (0 + 1) | (1 << 8) | (1 << 16)};     // a row of phase 1 whose one entry is read after a wait for phase 0
+    const int32_t pad_item[4] = {0, 0, -1, 0 | (1 << 8)};
+    for (int i = 0; i < 4; ++i) {
+        host.items[i] = row_item[i];
+        for (int q = 1; q < 4; ++q) host.items[4 * q + i] = pad_item[i];
+    }
+    host.phase_size[0] = 4;      // four rows that nobody holds
+    host.phase_size[1] = 4;
+    host.idx[0] = 1;             // an aggregation-node id (n_prim = 1): the row must wait before it loads it
+    Blob *dev = nullptr;
+    if (cudaMalloc(reinterpret_cast<void **>(&dev), sizeof(Blob)) != cudaSuccess) { cudaGetLastError(); return HAG_ERR_OOM_DEVICE; }
+    hag_status st = HAG_OK;
+    if (cudaMemcpyAsync(dev, &host, sizeof(Blob), cudaMemcpyHostToDevice, s) != cudaSuccess) st = HAG_ERR_CUDA;
+    if (st == HAG_OK) {
+        hagk::FusedArgs k{};
+        k.a.idx = dev->idx;
+        k.a.prim = dev->prim;
+        k.a.sec = dev->sec;
+        k.a.n_prim = 1;
+        k.a.out = dev->out;
+        k.a.D = D;
+        k.items = reinterpret_cast<const int4 *>(dev->items);
+        k.n_items = 4;
+        k.last_phase = 1;
+        k.phase_size = dev->phase_size;
+        k.ctl = dev->ctl;
+        k.ahat = dev->sec;
+        k.err_host = h->d.err_dev;
+        k.spin_limit = 2000;     // a few milliseconds
+        if (launch_pdl(hagk::fused_pass_kernel<float, 4, 4, false, 8, false>, 1u, k, s) != cudaSuccess) st = HAG_ERR_CUDA;
+    }
+    if (cudaStreamSynchronize(s) != cudaSuccess) st = HAG_ERR_CUDA;
+    cudaFree(dev);
+    if (st != HAG_OK) { cudaGetLastError(); return st; }
+    return hag_device_status(h);
+}
 
 extern "C" hag_status hag_profile_enable(hag_t *h, int enable) {
     if (!h) return HAG_ERR_NULL;

@@ -37,6 +37,35 @@ struct seg_set {
 
 constexpr int kSchedSlots = 64;      // far more than the kernels that can overlap on one stream
 
+// One whole pass (all aggregation-node levels, then the graph nodes) as ONE launch of resident warps.
+// The pass is a list of rows in dependency order: the rows of phase 0, then phase 1, ...; a phase is one
+// level of aggregation nodes (as rows of two entries where the level is evaluated pair by pair), or the
+// expanded deep nodes, or the chunk rows of the long rows of the phase after it, or (last) the graph-node
+// rows.  Warps take rows in list order from a counter; a row that reads rows written by an earlier phase
+// waits, with an iteration limit, until that phase's finished-row count is complete.  Because rows are
+// handed out in list order, whatever a row waits for is already in the hands of a running warp, so the
+// wait cannot deadlock.
+constexpr int kFusedItemsPerGrab = 4;     // a grab never straddles two phases (phases are padded to it)
+constexpr int kFusedMaxPhases = 56;       // deeper hierarchies run level by level
+constexpr int64_t kFusedRowsForFullGrabs = 320000;   // phases with fewer rows are handed out two rows, below a quarter of it one row, per grab
+constexpr int kFusedCtlWords = 64;        // per launch: [0] next row, [1] finished warps, [2] error, [4 + p] finished rows of phase p
+constexpr int kFusedCtlSlots = 16;        // ring: consecutive launches (overlapping under programmatic dependent launch) take turns
+constexpr int kFusedSpinLimit = 1 << 21;  // polls of a waiting warp before it gives up (about a second)
+
+struct fused_table {
+    bool ok = false;                 // false: no row list (too many phases, or no rows); the id list is built all the same
+    std::vector<int32_t> items;      // 4 per row: b, e, row, (required phase + 1) | phase << 8.  The row sums the entries [b, e) of
+                                     // `ids` into output row `row` (row < 0: padding; row >= n: an aggregation node or a chunk row)
+    std::vector<int32_t> phase_size; // rows per phase, padding included
+    std::vector<int32_t> ids;        // the pass's id list: pair inputs, expansion lists, row lists, chunk ids of the long rows
+    int64_t off_head = 0;            // where the expansion lists (ftail / btail) start in ids
+    int64_t off_tail = 0;            // where the row lists (residual rows / transposed HAG / input graph) start
+    int64_t n_chunks = 0;            // chunk rows: fp32 partial rows needed behind the aggregation nodes' rows
+    int32_t last_phase = 0;          // the graph-node rows: nothing waits for them
+    int64_t n_items() const { return int64_t(items.size() / 4); }
+    int32_t *d_items = nullptr, *d_phase_size = nullptr, *d_ids = nullptr;
+};
+
 struct hag_device_arrays {
     // HAG
     int32_t *agg_in = nullptr;     // [2*num_agg]
@@ -51,6 +80,11 @@ struct hag_device_arrays {
     int32_t *csr_t_idx = nullptr;  // [e]
     int32_t *ftail_ptr = nullptr, *ftail_idx = nullptr;   // forward expansion of the deep levels
     int32_t *btail_ptr = nullptr, *btail_idx = nullptr;   // backward expansion
+    // res_idx, t_idx, csr_idx, csr_t_idx and the expansion lists above point into the id lists of the four passes
+    // (fused_table::d_ids), which hold them next to what else a single-launch pass reads
+    unsigned int *fused_ctl = nullptr;     // kFusedCtlSlots x kFusedCtlWords, zero between launches
+    unsigned int *err_host = nullptr;      // one word of mapped pinned host memory: set by a kernel whose wait ran out
+    unsigned int *err_dev = nullptr;       // its device address
     float *inv_degree = nullptr;   // [n] 1/|N(v)| (1 for empty rows)
     float *inv_degree1 = nullptr;  // [n] 1/(|N(v)| + 1): the GCN normalisation
     unsigned int *sched = nullptr; // ring of kSchedSlots (next row, finished warps) pairs, zero between launches
@@ -88,6 +122,10 @@ struct hag {
     std::vector<int64_t> ftail_ptr, btail_ptr;
     std::vector<int32_t> ftail_idx, btail_idx;
     seg_set seg_res, seg_t, seg_csr, seg_csr_t, seg_ftail, seg_btail;
+    fused_table fz_fwd, fz_bwd, fz_csr, fz_csr_t;   // the four passes as single launches
+    int32_t schedule = 0;            // 0: a launch per level; 1: one launch per pass where a row list exists
+    uint32_t fused_seq = 0;          // next slot of the control ring
+    int32_t spin_limit = kFusedSpinLimit;
     int64_t max_segs_hag = 0, max_segs_csr = 0;   // partial rows the HAG / plain calls need in the workspace
     hag_info info{};
     int device = -1;
@@ -101,6 +139,10 @@ struct hag {
     struct launch_note { int32_t kind; int64_t rows, edges; };
     std::vector<launch_note> notes;           // launches of the last call
 };
+
+// Allocation-failure injection for tests (hag_test_fail_allocation): true when the allocation attempt that is
+// about to be made is the one chosen to fail.  kind 0: host memory, 1: device memory.
+bool hag_alloc_should_fail(int kind);
 
 // hag_build.cpp: the search (Algorithm 3) in creation-id space.  Fills
 // h->trace and returns the residual rows (creation ids, ascending) in

@@ -20,9 +20,17 @@
 //     or bf16); an id at or above it reads the fp32 rows of the aggregation
 //     nodes.  One kernel therefore serves Algorithm 2's final loop, the plain
 //     GNN-graph, and every step of the backward pass over the transposed HAG;
+//   * bf16 storage: the ids of a row ascend, so its bf16 rows (the layer input)
+//     come before its fp32 rows (aggregation nodes).  Each batch of 32 ids is
+//     split at that point; the bf16 rows are fetched as raw 16-byte words, kept
+//     raw while in flight (4 registers per load, not 8) and widened two at a
+//     time straight into packed fp32x2 adds;
 //   * every kernel is launched with programmatic stream serialisation: it lets
 //     its successor start launching at once and waits for its predecessor's
-//     memory only after it has fetched its own (static) row pointers and ids.
+//     memory only after it has fetched its own (static) row pointers and ids;
+//   * besides the launch-per-level kernels there is a single-launch form of a
+//     whole pass (fused_pass_kernel, further down), with bounded waits between
+//     the phases of the pass.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -77,11 +85,10 @@ template <> struct Chunk<__nv_bfloat16> { static constexpr int kElems = 8; };
 // Programmatic dependent launch (PTX griddepcontrol).
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
 // Feature rows and aggregation-node rows are read with ld.global.cg (coherent, cached at L2 only): the rows
 // may have been written by the kernel before this one, which is still alive when this one starts under
-// programmatic dependent launch.  The non-coherent path (ld.global.nc, __ldg) is kept for the handle's
-// static structure arrays only.
+// programmatic dependent launch, or by other warps of the same launch.  The non-coherent path
+// (ld.global.nc, __ldg) is kept for the handle's static structure arrays only.
 __device__ __forceinline__ float4 ld_f4(const void *p) { return __ldcg(reinterpret_cast<const float4 *>(p)); }
 __device__ __forceinline__ uint4 ld_u4(const void *p) { return __ldcg(reinterpret_cast<const uint4 *>(p)); }
 
@@ -121,6 +128,22 @@ __device__ __forceinline__ void add_rows(float *a, const float *b) {
     } else {
 #pragma unroll
         for (int j = 0; j < E; ++j) a[j] += b[j];
+    }
+}
+
+// acc[0..8) += (factor *) the eight bf16 values of one 16-byte word group, widened two at a time (a bf16 is the
+// upper half of an fp32: shift or mask) straight into packed fp32x2 adds: 8 widening and 4 arithmetic
+// instructions per 16 bytes, and the raw words stay raw (4 registers, not 8) until they are used.
+template <bool SCALED>
+__device__ __forceinline__ void add_bf16x8(float *acc, const uint4 &r, float factor) {
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 x = make_float2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xffff0000u));
+        const float2 a = make_float2(acc[2 * i], acc[2 * i + 1]);
+        const float2 s = SCALED ? __ffma2_rn(x, make_float2(factor, factor), a) : __fadd2_rn(a, x);
+        acc[2 * i] = s.x;
+        acc[2 * i + 1] = s.y;
     }
 }
 
@@ -178,6 +201,56 @@ __device__ __forceinline__ void store_chunk(void *out, int out_is_f32, int32_t D
     }
 }
 
+// Where a finished row goes.  The kernels that write one kind of row build it from GatherArgs; the
+// single-launch kernel chooses per row between the caller's output and the fp32 rows of the
+// aggregation nodes.
+struct RowOut {
+    void *out;
+    int32_t is_f32;
+    int32_t row_offset;
+};
+__device__ __forceinline__ RowOut row_out_of(const GatherArgs &a) { return RowOut{a.out, a.out_is_f32 & 1, a.out_row_offset}; }
+// How gather_row finds the output at the END of a row (nothing of it is kept in registers meanwhile).
+struct OutOfArgs {       // the launch writes one kind of row: taken from GatherArgs
+    static constexpr bool kMixed = false;
+    __device__ __forceinline__ RowOut get(const GatherArgs &a, int32_t) const { return row_out_of(a); }
+};
+struct OutPartial {      // a segment's partial row
+    static constexpr bool kMixed = false;
+    float *partial;
+    __device__ __forceinline__ RowOut get(const GatherArgs &, int32_t) const { return RowOut{partial, 1, 0}; }
+};
+struct OutByRow {        // single-launch kernel: aggregation-node rows (id >= n_prim) go to their fp32 rows
+    static constexpr bool kMixed = true;
+    float *ahat;
+    __device__ __forceinline__ RowOut get(const GatherArgs &a, int32_t row) const {
+        return row >= a.n_prim ? RowOut{ahat, 1, a.n_prim} : row_out_of(a);
+    }
+};
+
+// A row of the single-launch kernel may read rows that other warps of the same launch write.  Its entries
+// ascend, so the rows of the layer input come first and need nothing: the row is summed in two parts, the
+// entries before the first such row at once, the rest after the warp has waited for the phase that writes
+// the latest of them.  The wait sits between the two loops, never inside them.  NoGate: a single part.
+struct NoGate {
+    static constexpr bool kOn = false;
+    __device__ __forceinline__ int32_t split(int32_t e) const { return e; }
+    __device__ __forceinline__ void wait(int) const {}
+};
+struct FusedArgs;
+__device__ __forceinline__ void fused_wait(const FusedArgs &k, int phase, int lane);
+struct PhaseGate {
+    static constexpr bool kOn = true;
+    const FusedArgs *k;
+    int32_t req;          // phase to wait for before the second part, -1: none, or known to be complete
+    int32_t n_sec;        // entries of the second part (the last n_sec of the row)
+    // (always cut at the same place, waiting or not: the order of the additions must not depend on timing)
+    __device__ __forceinline__ int32_t split(int32_t e) const { return e - n_sec; }
+    __device__ __forceinline__ void wait(int lane) const {
+        if (req >= 0) fused_wait(*k, req, lane);
+    }
+};
+
 // What a warp needs before it can start on a row: the first 32 source ids (one per
 // lane, -1 past the end), their factors, and the row's own factor.  All of it is
 // static structure, so it can be fetched while the previous row is still summed.
@@ -194,13 +267,14 @@ __device__ __forceinline__ RowHead load_head(const GatherArgs &a, int32_t row, i
     // the factor of each source travels with its id: fetched a batch ahead, handed round by shuffle
     h.src_scale = 1.0f;
     if constexpr (SRC_SCALE) h.src_scale = (h.id >= 0 && h.id < a.n_prim) ? __ldg(a.src_scale + h.id) : 1.0f;
-    h.dst_scale = a.dst_scale ? __ldg(a.dst_scale + row) : 1.0f;
+    h.dst_scale = (a.dst_scale && row < a.n_prim) ? __ldg(a.dst_scale + row) : 1.0f;   // graph-node rows only
     return h;
 }
 
 // Gather-sum of one row [b, e) by one warp.  Returns with the result stored.
-template <typename T, int LPR, int UNROLL, bool SRC_SCALE, bool SELF>
-__device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int32_t b, int32_t e, const RowHead &head, int lane) {
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, bool SELF, typename Out = OutOfArgs, typename Gate = NoGate>
+__device__ __forceinline__ void gather_row(const GatherArgs &a, const Out &osel, int32_t row, int32_t b, int32_t e, const RowHead &head, int lane,
+                                           const Gate gate = Gate()) {
     constexpr int E = Chunk<T>::kElems;
     constexpr int G = 32 / LPR;                 // slices per warp
     constexpr int PER_BATCH = LPR;              // neighbours each slice takes from a batch of 32 ids
@@ -228,14 +302,84 @@ __device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int
             mine = (b + lane < e) ? __ldg(a.idx + b + lane) : -1;
             if constexpr (SRC_SCALE) mine_s = (mine >= 0 && mine < a.n_prim) ? __ldg(a.src_scale + mine) : 1.0f;
         }
-        for (int32_t base = b; base < e; base += 32) {
-            const int32_t cur = mine;
+        int32_t lo = b, hi = gate.split(e);
+#pragma unroll 1
+        for (int half = 0; half < (Gate::kOn ? 2 : 1); ++half) {
+        if (Gate::kOn && half == 1) {           // the rows written by earlier phases, at the end of the row
+            lo = hi;
+            hi = e;
+            if (lo >= hi) break;
+            mine = (lo + lane < hi) ? __ldg(a.idx + lo + lane) : -1;     // ids are static: in flight during the wait
+            mine_s = 1.0f;
+            gate.wait(lane);
+        }
+        for (int32_t base = lo; base < hi; base += 32) {
+            // first part: entries beyond it belong to the second part and must not be loaded yet
+            const int32_t cur = (Gate::kOn && base + lane >= hi) ? -1 : mine;
             const float cur_s = mine_s;
             const int32_t nb = base + 32;
-            mine = (nb + lane < e) ? __ldg(a.idx + nb + lane) : -1;      // next batch of ids, in flight early
+            mine = (nb + lane < hi) ? __ldg(a.idx + nb + lane) : -1;     // next batch of ids, in flight early
             if constexpr (SRC_SCALE) mine_s = (mine >= 0 && mine < a.n_prim) ? __ldg(a.src_scale + mine) : 1.0f;
-            const int cnt = min(32, e - base);
-            if constexpr (E == 4) {       // fp32 storage only: bf16 results are rounded to 8 bits anyway
+            const int cnt = min(32, hi - base);
+            if constexpr (E == 8) {
+                // bf16 storage.  The ids of a row ascend, so the rows of the layer input (bf16) are the first n_p
+                // entries of the batch and the fp32 rows of aggregation nodes the rest: two loops, neither of which
+                // has to choose a table per entry.  bf16 rows are fetched as raw words, U in flight, and widened
+                // only as they are added (add_bf16x8); sums go straight into the accumulator (the result is rounded
+                // to 8 bits anyway).
+                const int n_p = __popc(__ballot_sync(0xffffffffu, cur >= 0 && cur < a.n_prim));
+#pragma unroll
+                for (int k = 0; k < PER_BATCH; k += U) {
+                    if (k * G < n_p) {
+                        uint4 raw[U];
+                        if ((k + U) * G <= n_p) {       // every entry of this group exists: no checks, no zero fill
+#pragma unroll
+                            for (int u = 0; u < U; ++u)
+                                raw[u] = ld_u4(tab.prim + size_t(uint32_t(__shfl_sync(0xffffffffu, cur, (k + u) * G + slice))) * tab.prim_row_bytes);
+                        } else {
+#pragma unroll
+                            for (int u = 0; u < U; ++u) {
+                                const int32_t id = __shfl_sync(0xffffffffu, cur, (k + u) * G + slice);
+                                raw[u] = ((k + u) * G + slice < n_p && live) ? ld_u4(tab.prim + size_t(uint32_t(id)) * tab.prim_row_bytes)
+                                                                             : make_uint4(0u, 0u, 0u, 0u);
+                            }
+                        }
+#pragma unroll
+                        for (int u = 0; u < U; ++u) {
+                            float sc = 1.0f;
+                            if constexpr (SRC_SCALE) sc = __shfl_sync(0xffffffffu, cur_s, (k + u) * G + slice);
+                            add_bf16x8<SRC_SCALE>(acc, raw[u], sc);
+                        }
+                    }
+                }
+                // the fp32 rows (never scaled): 32 bytes per lane and row, so half as many rows in flight for the same registers
+                constexpr int US = (U >= 2) ? U / 2 : 1;
+                for (int j0 = n_p; j0 < cnt; j0 += US * G) {
+                    float4 q[US][2];
+#pragma unroll
+                    for (int u = 0; u < US; ++u) {
+                        const int j = j0 + u * G + slice;
+                        const int32_t id = __shfl_sync(0xffffffffu, cur, j < cnt ? j : 0);
+                        if (j < cnt && live) {
+                            const char *p = tab.sec + size_t(uint32_t(id)) * tab.sec_row_bytes;
+                            q[u][0] = ld_f4(p);
+                            q[u][1] = ld_f4(p + 16);
+                        } else {
+                            q[u][0] = q[u][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < US; ++u) {
+                        float2 s;
+                        s = __fadd2_rn(make_float2(acc[0], acc[1]), make_float2(q[u][0].x, q[u][0].y)); acc[0] = s.x; acc[1] = s.y;
+                        s = __fadd2_rn(make_float2(acc[2], acc[3]), make_float2(q[u][0].z, q[u][0].w)); acc[2] = s.x; acc[3] = s.y;
+                        s = __fadd2_rn(make_float2(acc[4], acc[5]), make_float2(q[u][1].x, q[u][1].y)); acc[4] = s.x; acc[5] = s.y;
+                        s = __fadd2_rn(make_float2(acc[6], acc[7]), make_float2(q[u][1].z, q[u][1].w)); acc[6] = s.x; acc[7] = s.y;
+                    }
+                }
+                continue;
+            }
+            if constexpr (E == 4) {       // fp32 storage: two-level sums
 #pragma unroll
                 for (int j = 0; j < E; ++j) part[j] = 0.0f;
             }
@@ -296,6 +440,7 @@ __device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int
             }
             if constexpr (E == 4) add_rows<E>(acc, part);
         }
+        }
         // combine the slices (fixed butterfly), then slice 0 stores
 #pragma unroll
         for (int off = LPR; off < 32; off <<= 1)
@@ -303,16 +448,19 @@ __device__ __forceinline__ void gather_row(const GatherArgs &a, int32_t row, int
             for (int j = 0; j < E; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], off);
         if (live && slice == 0) {
             if constexpr (SELF) {         // GCN: the row's own term, compiled only into the variants that need it
-                float self[E];
-                tab.load(row, self);
-                float sc = 1.0f;
-                if constexpr (SRC_SCALE) sc = __ldg(a.src_scale + row);
+                if (!Out::kMixed || row < a.n_prim) {    // (the single-launch kernel also writes aggregation-node rows)
+                    float self[E];
+                    tab.load(row, self);
+                    float sc = 1.0f;
+                    if constexpr (SRC_SCALE) sc = __ldg(a.src_scale + row);
 #pragma unroll
-                for (int j = 0; j < E; ++j) acc[j] = fmaf(self[j], sc, acc[j]);
+                    for (int j = 0; j < E; ++j) acc[j] = fmaf(self[j], sc, acc[j]);
+                }
             }
 #pragma unroll
             for (int j = 0; j < E; ++j) acc[j] *= dscale;
-            store_chunk<T>(a.out, a.out_is_f32 & 1, a.D, row - a.out_row_offset, chunk, acc);
+            const RowOut ro = osel.get(a, row);
+            store_chunk<T>(ro.out, ro.is_f32, a.D, row - ro.row_offset, chunk, acc);
         }
     }
 }
@@ -325,13 +473,9 @@ __device__ __forceinline__ void gather_segment(const GatherArgs &a, const SegArg
     constexpr int E = Chunk<T>::kElems;
     const int4 sg = __ldg(sa.segs + seg_local);
     const int32_t row = sg.x, b = sg.y, e = sg.z, slot = sg.w;
-    GatherArgs part = a;
-    part.out = sa.partial;
-    part.out_is_f32 = 1;
-    part.out_row_offset = 0;
     RowHead head = load_head<SRC_SCALE>(a, row, b, e, lane);
     head.dst_scale = 1.0f;
-    gather_row<T, LPR, UNROLL, SRC_SCALE, false>(part, sa.seg_first + seg_local, b, e, head, lane);
+    gather_row<T, LPR, UNROLL, SRC_SCALE, false, OutPartial>(a, OutPartial{sa.partial}, sa.seg_first + seg_local, b, e, head, lane);
     __threadfence();                                   // partial row visible before the count moves
     __syncwarp();
     const int2 sl = __ldg(sa.slots + slot);
@@ -341,7 +485,7 @@ __device__ __forceinline__ void gather_segment(const GatherArgs &a, const SegArg
     if (done != unsigned(sl.y) - 1u) return;
     __threadfence();
     if (lane == 0) sa.seg_done[slot] = 0;              // ready for the next launch
-    const float dscale = a.dst_scale ? __ldg(a.dst_scale + row) : 1.0f;
+    const float dscale = (a.dst_scale && row < a.n_prim) ? __ldg(a.dst_scale + row) : 1.0f;
     const int n_chunks = a.D / E;
     for (int chunk = lane; chunk < n_chunks; chunk += 32) {
         float acc[E];
@@ -356,13 +500,15 @@ __device__ __forceinline__ void gather_segment(const GatherArgs &a, const SegArg
             }
         }
         if constexpr (SELF) {
-            const Tables<T> tab(a.prim, a.sec, a.n_prim, a.D, chunk);
-            float self[E];
-            tab.load(row, self);
-            float sc = 1.0f;
-            if constexpr (SRC_SCALE) sc = __ldg(a.src_scale + row);
+            {
+                const Tables<T> tab(a.prim, a.sec, a.n_prim, a.D, chunk);
+                float self[E];
+                tab.load(row, self);
+                float sc = 1.0f;
+                if constexpr (SRC_SCALE) sc = __ldg(a.src_scale + row);
 #pragma unroll
-            for (int j = 0; j < E; ++j) acc[j] = fmaf(self[j], sc, acc[j]);
+                for (int j = 0; j < E; ++j) acc[j] = fmaf(self[j], sc, acc[j]);
+            }
         }
 #pragma unroll
         for (int j = 0; j < E; ++j) acc[j] *= dscale;
@@ -402,7 +548,7 @@ __device__ __forceinline__ void gather_sum_body(const KernelArgs<HAS_SEGS> &k) {
     }
     const RowHead head = load_head<SRC_SCALE>(a, row, b, e, lane);
     pdl_wait();        // structure arrays are static; features may come from the previous kernel
-    gather_row<T, LPR, UNROLL, SRC_SCALE, SELF>(a, row, b, e, head, lane);
+    gather_row<T, LPR, UNROLL, SRC_SCALE, SELF>(a, OutOfArgs{}, row, b, e, head, lane);
 }
 
 // Two entry points per form: the parameter block of the variant with long rows is declared
@@ -477,7 +623,7 @@ __device__ __forceinline__ void gather_sum_persistent_body(const KernelArgs<HAS_
             }
             bool whole = true;
             if constexpr (HAS_SEGS) whole = e - b <= k.sg.long_row;
-            if (whole) gather_row<T, LPR, UNROLL, SRC_SCALE, SELF>(a, a.row_begin + base + i, b, e, cur, lane);
+            if (whole) gather_row<T, LPR, UNROLL, SRC_SCALE, SELF>(a, OutOfArgs{}, a.row_begin + base + i, b, e, cur, lane);
             if (i == 0 && nrows > 1) {
                 nbase = __shfl_sync(FULL, grabbed, 0) - seg_items;
                 rp_next = load_rp(nbase);
@@ -502,6 +648,151 @@ __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_persistent_ke
 template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS, bool SELF>
 __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_persistent_long_kernel(const __grid_constant__ KernelArgs<true> k) {
     gather_sum_persistent_body<T, LPR, UNROLL, SRC_SCALE, true, SELF>(k);
+}
+
+// --------------------------------------------------------------------------- //
+// One whole pass as ONE launch.
+//
+// Algorithm 2 asks for the aggregation nodes in an order in which every node comes after its
+// inputs, then the graph nodes.  Launching a kernel per level keeps that order but pays a launch
+// and a pipeline drain per level, which costs more than the levels themselves once they are small
+// (hierarchies of 7 to 20 levels whose sizes fall off geometrically).  Here the pass is a list of
+// rows in that order -- phase 0, phase 1, ..., the graph-node rows last -- and resident warps take
+// rows from the list four at a time.  Everything is a row: an aggregation node of a level that is
+// evaluated pair by pair is a row of two entries; a row too long for one warp is cut into chunk rows
+// of a phase of their own, whose fp32 partial rows (kept behind the aggregation nodes' rows, ids from
+// n_prim + |V_A| on) a last short row adds up.  A row that reads rows of an earlier phase first
+// waits until that phase's count of finished rows is complete.  The wait cannot deadlock (whatever
+// is waited for was handed out earlier, to a warp that is running) and is bounded all the same: after
+// spin_limit polls the warp records the failure (device word for the other waiters, host-mapped
+// word for the caller), stops waiting and carries on, so the launch always ends.
+// --------------------------------------------------------------------------- //
+constexpr int kCtlNext = 0, kCtlFinished = 1, kCtlError = 2, kCtlDone = 4;
+constexpr int kFusedGrab = 4;      // rows per grab; a grab lies in one phase
+
+struct FusedArgs {
+    GatherArgs a;              // idx: the pass's id list; prim / sec / n_prim / scales / out as for the row kernels;
+                               // rows with id >= n_prim (aggregation nodes, chunk rows) go to ahat (fp32), row id - n_prim
+    const int4 *items;         // {b, e, row, (required phase + 1) | phase << 8 | (entries read after the wait) << 16}; row < 0: padding
+    int32_t n_items;           // a multiple of four; every group of four lies in one phase
+    int32_t last_phase;        // its rows are not counted: nothing waits for them
+    const int32_t *phase_size; // rows per phase, padding included
+    unsigned int *ctl;         // [kCtlNext] next row, [kCtlFinished] finished warps, [kCtlError], [kCtlDone + p] finished rows of phase p
+    float *ahat;               // = a.sec
+    unsigned int *err_host;    // mapped host word, set when a wait ran out
+    int32_t spin_limit;
+};
+
+// Every lane polls (one address: one request per poll) and the exits are taken on warp votes, so the
+// control flow is uniform by construction: the code after the wait keeps plain converged shuffles.
+__device__ __forceinline__ void fused_wait(const FusedArgs &k, int phase, int lane) {
+    constexpr unsigned FULL = 0xffffffffu;
+    const unsigned need = unsigned(__ldg(k.phase_size + phase));
+    const unsigned int *done = k.ctl + kCtlDone + phase;
+    const volatile unsigned int *failed = k.ctl + kCtlError;
+    bool ok = false;
+    for (int it = 0; it < k.spin_limit; ++it) {
+        unsigned v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(done) : "memory");
+        if (__all_sync(FULL, v >= need)) { ok = true; break; }
+        if (__any_sync(FULL, *failed != 0u)) break;     // somebody gave up already: do not add a second of waiting per row
+        __nanosleep(it < 32 ? 40 : 400);
+    }
+    if (!ok && lane == 0) {
+        k.ctl[kCtlError] = 1u;
+        *reinterpret_cast<volatile unsigned int *>(k.err_host) = 1u;
+        __threadfence_system();
+    }
+    __syncwarp();
+    __threadfence();
+}
+
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, bool SELF>
+__device__ __forceinline__ void fused_body(const FusedArgs &k) {
+    const GatherArgs &a = k.a;
+    pdl_launch_dependents();
+    constexpr int CH = kFusedGrab;
+    constexpr unsigned FULL = 0xffffffffu;
+    const int lane = threadIdx.x & 31;
+    const int32_t count = k.n_items;
+    auto grab = [&]() -> int32_t {          // meaningful in lane 0
+        int32_t v = 0;
+        if (lane == 0) v = int32_t(atomicAdd(k.ctl + kCtlNext, unsigned(CH)));
+        return v;
+    };
+    // the four rows of a grab in ONE register per lane: lane 4 w + i holds word w (b, e, row, phases) of row i
+    auto load_items = [&](int32_t at) -> int32_t {
+        return (lane < 4 * CH && at < count) ? __ldg(reinterpret_cast<const int32_t *>(k.items) + 4 * (at + (lane & 3)) + (lane >> 2)) : -1;
+    };
+    // first ids (and factors) of a row; nothing for padding
+    auto item_head = [&](int32_t words, int i) -> RowHead {
+        const int32_t b = __shfl_sync(FULL, words, i), e = __shfl_sync(FULL, words, 4 + i), row = __shfl_sync(FULL, words, 8 + i);
+        if (row >= 0) return load_head<SRC_SCALE>(a, row, b, e, lane);
+        return RowHead{-1, 1.0f, 1.0f};
+    };
+    int32_t base = __shfl_sync(FULL, grab(), 0);
+    int32_t it = load_items(base);
+    RowHead head = item_head(it, 0);
+    int known = -1;            // every phase <= known has been seen complete: no need to look again
+    unsigned pending = 0;      // rows of the current phase this warp has finished and not yet reported
+    pdl_wait();        // the row list is static; features may come from the kernel before
+    while (base < count) {
+        const int32_t grabbed = grab();     // the next four rows; consumed after the first row below
+        int32_t nbase = count, nit = -1;
+        const int phase = (__shfl_sync(FULL, it, 12) >> 8) & 255;
+#pragma unroll 1
+        for (int i = 0; i < CH; ++i) {
+            const int32_t b = __shfl_sync(FULL, it, i), e = __shfl_sync(FULL, it, 4 + i);
+            const int32_t row = __shfl_sync(FULL, it, 8 + i), word = __shfl_sync(FULL, it, 12 + i);
+            const RowHead cur = head;
+            head = (i + 1 < CH) ? item_head(it, i + 1) : item_head(nit, 0);
+            if (row >= 0) {
+                const int req = (word & 255) - 1;
+                gather_row<T, LPR, UNROLL, SRC_SCALE, SELF, OutByRow, PhaseGate>(a, OutByRow{k.ahat}, row, b, e, cur, lane,
+                                                                                 PhaseGate{&k, req > known ? req : -1, int32_t(uint32_t(word) >> 16)});
+                known = max(known, req);        // the row has waited for it (a row that waits for a phase reads from it)
+            }
+            if (i == 0) {
+                nbase = __shfl_sync(FULL, grabbed, 0);
+                nit = load_items(nbase);
+            }
+        }
+        pending += unsigned(CH);
+        // Finished rows are reported when the warp leaves their phase: its next grab lies in a later phase, or there is
+        // none (rows are handed out in list order, so that is the moment the phase runs out of rows to hand out).
+        // Always BEFORE the warp can wait for anything in the later phase, or it would wait for itself.
+        const int next_phase = nbase < count ? (__shfl_sync(FULL, nit, 12) >> 8) & 255 : -1;
+        if (next_phase != phase) {
+            if (phase != k.last_phase) {
+                // Reported only once the phase before is complete, so that "phase q is complete" implies that every
+                // earlier phase is (a row waits for the latest phase it reads from only).
+                if (phase - 1 > known) {
+                    fused_wait(k, phase - 1, lane);
+                    known = phase - 1;
+                }
+                __threadfence();                // this warp's rows visible before the count moves
+                __syncwarp();
+                if (lane == 0) atomicAdd(k.ctl + kCtlDone + phase, pending);
+            }
+            pending = 0;
+        }
+        base = nbase;
+        it = nit;
+    }
+    if (lane == 0) {
+        const unsigned finished = atomicAdd(k.ctl + kCtlFinished, 1u);
+        if (finished == gridDim.x * kWarps - 1) {   // every warp has made its last grab and finished its rows
+            for (int p = 0; p <= k.last_phase; ++p) k.ctl[kCtlDone + p] = 0;
+            k.ctl[kCtlNext] = 0;
+            k.ctl[kCtlError] = 0;
+            k.ctl[kCtlFinished] = 0;
+        }
+    }
+}
+
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS, bool SELF>
+__global__ void __launch_bounds__(kThreads, MIN_BLOCKS) fused_pass_kernel(const __grid_constant__ FusedArgs k) {
+    fused_body<T, LPR, UNROLL, SRC_SCALE, SELF>(k);
 }
 
 // Level kernel of Algorithm 2 (lines 5-6): every aggregation node of one level is

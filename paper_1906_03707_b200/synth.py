@@ -64,7 +64,13 @@ def csr_from_directed_pairs(n: int, src: np.ndarray, dst: np.ndarray, name: str 
     """Build the in-neighbour CSR from directed edges (src -> dst), dropping duplicates."""
     src = np.asarray(src, dtype=np.int64)
     dst = np.asarray(dst, dtype=np.int64)
-    key = np.unique(dst * np.int64(n) + src)          # sorted by (dst, src)
+    key = dst * np.int64(n) + src
+    key.sort()                                        # sorted by (dst, src)
+    if key.shape[0] > 1:                              # drop duplicates (what np.unique returns, without its hashing pass)
+        keep = np.empty(key.shape[0], dtype=bool)
+        keep[0] = True
+        np.not_equal(key[1:], key[:-1], out=keep[1:])
+        key = key[keep]
     d = key // n
     s = (key - d * n).astype(np.int32)
     counts = np.bincount(d, minlength=n).astype(np.int64)

@@ -318,3 +318,100 @@ def test_binding_rejects_wrong_tensors_before_any_launch():
         h.aggregate_host(good, torch.zeros((g.n, 8)))             # out does not match
     with pytest.raises(ValueError):
         h.max_bwd(torch.zeros((g.n - 1, 16)), good, None, good)
+
+
+def _emulate_pass(p, n, k, src, d):
+    """Walks the row list of one pass in list order on the CPU (fp64), the way the single-launch kernel's warps
+    are handed the rows, and checks what the kernel relies on: groups of four rows lie in one phase; the rows of
+    other phases that a row reads (aggregation nodes, chunk rows: ids >= n) were written by phases <= the phase it
+    waits for (the kernel itself reports a grab only after the phase before it is complete, so "phase q complete"
+    implies all earlier ones); only the last phase writes graph-node rows; every row is written exactly once.
+    Returns (graph-node rows, aggregation-node rows, writes per row)."""
+    rows, ids, c = p["rows"], p["ids"], p["n_chunk_rows"]
+    assert rows.shape[0] % 4 == 0 and int(p["phase_size"].sum()) == rows.shape[0]
+    word = rows[:, 3].astype(np.int64) & 0xffffffff
+    req, phase, n_sec = (word & 255) - 1, (word >> 8) & 255, word >> 16
+    assert (np.diff(phase) >= 0).all() and (phase.reshape(-1, 4) == phase[::4, None]).all()
+    assert np.array_equal(np.bincount(phase, minlength=p["phase_size"].shape[0]), p["phase_size"])
+    last = int(phase.max())
+    val = np.zeros((n + k + c, d))
+    val[:n] = src
+    out = np.zeros((n, d))
+    written_in = np.full(n + k + c, -1)             # phase that wrote an aggregation-node or chunk row
+    writes = np.zeros(n + k + c, dtype=np.int64)
+    for i in range(rows.shape[0]):
+        b, e, row = (int(v) for v in rows[i, :3])
+        if row < 0:
+            continue
+        acc = np.zeros(d)
+        # the entries read before the wait are rows of the layer input, the last n_sec are rows this pass writes
+        assert (ids[b:e - n_sec[i]] < n).all() and (ids[e - n_sec[i]:e] >= n).all() and (n_sec[i] > 0) == (req[i] >= 0), i
+        for s_ in ids[b:e]:
+            if s_ >= n:
+                assert 0 <= written_in[s_] <= req[i] < phase[i], (i, s_, written_in[s_], req[i])
+            acc += val[s_]
+        writes[row] += 1
+        if row >= n:
+            val[row] = acc
+            written_in[row] = phase[i]
+            assert phase[i] < last
+        else:
+            out[row] = acc
+            assert phase[i] == last
+    return out, val[n:n + k], writes
+
+
+@pytest.mark.parametrize("maker,cap_frac", [
+    (lambda: synth.clique_union_graph(seed=15, n=1500, n_groups=400, g_lo=3, g_hi=40), 0.25),
+    (lambda: synth.config2_graph(seed=11, n=3000, n_comm=30), 0.25),
+    (lambda: synth.config4_graph(seed=13, n_graphs=20, graph_size=60), 0.25),
+    (lambda: synth.workload(1).graph, 0.0),
+])
+def test_single_launch_item_lists_evaluate_algorithm_2_for_every_cut(maker, cap_frac):
+    g = maker()
+    cap = int(g.n * cap_frac)
+    h = hb.Hag.build(g.row_ptr, g.col_idx, cap)
+    arr = h.arrays()
+    n, k, L = g.n, arr["num_agg"], arr["num_levels"]
+    x = synth.features(5, n, 3, "int").astype(np.float64)
+    gr = synth.features(6, n, 3, "int").astype(np.float64)
+    want_f, _ = O.direct_forward(g.row_ptr, g.col_idx, x, "sum")
+    want_b, _ = O.direct_backward(g.row_ptr, g.col_idx, gr, "sum")
+    ref = O.canonical_hag(g.row_ptr, O.greedy_pairmap(g.row_ptr, g.col_idx, cap))
+    ahat = np.zeros((n + k, 3))
+    ahat[:n] = x
+    for j in range(k):
+        ahat[n + j] = ahat[ref.agg_in[2 * j]] + ahat[ref.agg_in[2 * j + 1]]
+    cuts = sorted({(-1, -1), (0, 0), (L, L), (L // 2, (L + 1) // 2), (1 if L else 0, L)})
+    for fc, bc in cuts:
+        h.set_cuts(fc, bc)
+        arr = h.arrays()
+        out, agg, writes = _emulate_pass(h.pass_rows(0), n, k, x, 3)
+        assert (writes == 1).all()
+        assert np.array_equal(out, want_f) and np.array_equal(agg, ahat[n:])
+        gx, _, writes = _emulate_pass(h.pass_rows(1), n, k, gr, 3)
+        assert (writes == 1).all() and np.array_equal(gx, want_b)
+        assert h.workspace_bytes(4) >= 16 * (k + max(h.pass_rows(0)["n_chunk_rows"], h.pass_rows(1)["n_chunk_rows"]))
+    out, _, writes = _emulate_pass(h.pass_rows(2), n, 0, x, 3)
+    assert np.array_equal(out, want_f) and (writes == 1).all()
+    gx, _, writes = _emulate_pass(h.pass_rows(3), n, 0, gr, 3)
+    assert np.array_equal(gx, want_b) and (writes == 1).all()
+    assert h.csr_workspace_bytes(4) >= 16 * max(h.pass_rows(2)["n_chunk_rows"], h.pass_rows(3)["n_chunk_rows"])
+
+
+def test_injected_host_allocation_failures_return_a_status_and_leave_nothing_behind():
+    lib = hb.load_library()
+    g = synth.config2_graph(seed=19, n=2500, n_comm=25)
+    out = ctypes.c_void_p()
+    try:
+        for countdown in (0, 1):          # the search, then the layout
+            assert lib.hag_test_fail_allocation(0, countdown) == 0
+            st = lib.hag_build(g.n, g.row_ptr.ctypes.data, g.col_idx.ctypes.data, g.n // 4, ctypes.byref(out))
+            assert st == hb.HAG_ERR_OOM_HOST and out.value is None
+            assert hb.status_str(st) == "out of host memory"
+        # the hook fires once: the next build succeeds
+        assert lib.hag_build(g.n, g.row_ptr.ctypes.data, g.col_idx.ctypes.data, g.n // 4, ctypes.byref(out)) == 0
+        lib.hag_destroy(out)
+        assert lib.hag_test_fail_allocation(2, 0) == 2
+    finally:
+        lib.hag_test_fail_allocation(0, -1)

@@ -145,3 +145,31 @@ def test_full_size_workloads(index):
     every element of the forward result and of the gradient against the oracle."""
     w = synth.workload(index)
     _check(w.graph, w.capacity, w.d, "f32", seed=w.seed)
+
+
+@pytest.mark.parametrize("index", [3, 5, 6])
+def test_full_size_workloads_sampled_rows(index):
+    """The two largest shapes (fp32 D = 128; bf16 D = 256) and the clique-union graph at full size, in the
+    storage type of the workload: the oracle evaluates sampled rows one by one (forward rows, and gradient
+    rows with the maxima of their out-neighbours), hub rows and empty-ish rows included."""
+    w = synth.workload(index)
+    g = w.graph
+    h = hb.Hag.build(g.row_ptr, g.col_idx, w.capacity).to_device(0)
+    z = synth.features(w.seed, g.n, w.d, "normal", w.dtype)
+    gr = synth.upstream_grad(w.seed, g.n, w.d, "normal", w.dtype)
+    rng = np.random.default_rng(index)
+    deg = np.diff(g.row_ptr)
+    out_deg = np.bincount(g.col_idx, minlength=g.n)
+    rows = np.unique(np.concatenate([rng.choice(g.n, 1200, replace=False), np.argsort(deg)[-20:], np.argsort(deg)[:20],
+                                     np.argsort(out_deg)[-20:], [0, g.n - 1]]))
+    z64, g64 = z.astype(np.float64), gr.astype(np.float64)
+    want = O.direct_max_forward(g.row_ptr, g.col_idx, z64, rows=rows)
+    wantg, tg = O.direct_max_backward(g.row_ptr, g.col_idx, z64, g64, rows=rows)
+    zd, gd = _dev(z, w.dtype), _dev(gr, w.dtype)
+    for use_hag in (True, False):
+        out, ws = h.max_fwd(zd, use_hag=use_hag)
+        assert np.array_equal(_host(out)[rows], want), f"max forward use_hag={use_hag}"
+        gz = _host(h.max_bwd(zd, out, ws, gd, use_hag=use_hag))[rows]
+        err = np.abs(gz - wantg)
+        assert (err <= _bound(tg, wantg, w.dtype)).all(), f"max backward use_hag={use_hag}: worst {err.max():.3e}"
+    h.close()

@@ -1,7 +1,8 @@
-"""The N > 1 path on CPU: two gloo ranks shard a block-diagonal batch, each builds
+"""The N > 1 path on CPU: two gloo ranks shard a block-diagonal batch by graph, each builds
 the HAG of its own graphs with the library (host code) and evaluates it with the
-oracle; the pieces must tile the unsharded result, and the timing reduction must
-be the max over ranks."""
+oracle; then they split the feature columns of one graph, each with the whole structure
+from the library; the pieces must tile the unsharded results, and the timing reduction
+must be the max over ranks."""
 import os
 import socket
 
@@ -61,6 +62,19 @@ def _worker(rank, world, port, tmpdir):
         gx = O.hag_backward(ref, x[first:first + mine.n], "sum")
         np.save(os.path.join(tmpdir, f"out{rank}.npy"), out)
         np.save(os.path.join(tmpdir, f"gx{rank}.npy"), gx)
+        # second split: the feature columns of ONE graph; every rank holds the whole structure (built by the library,
+        # evaluated over the library's own arrays) and a 16-byte-aligned slice of the columns: no exchange
+        g2 = synth.config2_graph(seed=23, n=1200, n_comm=12)
+        d2 = 24
+        c0, cn = sharding.shard_columns(d2, rank, world, 4)
+        h2 = hb.Hag.build(g2.row_ptr, g2.col_idx, g2.n // 4)
+        a2 = h2.arrays()
+        lay = O.CanonicalHag(g2.n, a2["num_agg"], a2["num_levels"], a2["level_ptr"], a2["agg_in"], a2["res_ptr"], a2["res_idx"],
+                             a2["t_ptr"], a2["t_idx"], a2["in_degree"], None)
+        x2 = synth.features(4, g2.n, d2, "normal").astype(np.float64)
+        mine2 = np.ascontiguousarray(x2[:, c0:c0 + cn])
+        np.save(os.path.join(tmpdir, f"cols_out{rank}.npy"), O.hag_forward(lay, mine2, "mean"))
+        np.save(os.path.join(tmpdir, f"cols_gx{rank}.npy"), O.hag_backward(lay, mine2, "mean"))
         # timing reduction: slowest rank decides, units add up
         ms = sharding.max_over_ranks(10.0 + 5.0 * rank)
         units = sharding.sum_over_ranks(float(mine.n))
@@ -86,6 +100,16 @@ def test_two_gloo_ranks_tile_the_batch(tmp_path):
     got_b = np.concatenate([np.load(tmp_path / f"gx{r}.npy") for r in range(world)])
     np.testing.assert_allclose(got, want, rtol=0, atol=1e-12)
     np.testing.assert_allclose(got_b, want_b, rtol=0, atol=1e-12)
+    # the column split: side by side the ranks' slices are the whole result
+    g2 = synth.config2_graph(seed=23, n=1200, n_comm=12)
+    x2 = synth.features(4, g2.n, 24, "normal").astype(np.float64)
+    want2, _ = O.direct_forward(g2.row_ptr, g2.col_idx, x2, "mean")
+    want2_b, _ = O.direct_backward(g2.row_ptr, g2.col_idx, x2, "mean")
+    got2 = np.concatenate([np.load(tmp_path / f"cols_out{r}.npy") for r in range(world)], axis=1)
+    got2_b = np.concatenate([np.load(tmp_path / f"cols_gx{r}.npy") for r in range(world)], axis=1)
+    assert got2.shape == want2.shape
+    np.testing.assert_allclose(got2, want2, rtol=0, atol=1e-11)
+    np.testing.assert_allclose(got2_b, want2_b, rtol=0, atol=1e-11)
 
 
 def test_column_slices_tile_the_features_and_need_no_exchange():
