@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhag_b200.so")
 SOURCES = ["hag_build.cpp", "hag_cuda.cu", "hag_pool.cu", "hag_max.cu"]
 HEADERS = [os.path.join(ROOT, "include", "hag.h"), os.path.join(CSRC, "hag_internal.h"),
-           os.path.join(CSRC, "hag_kernels.cuh")]
+           os.path.join(CSRC, "hag_kernels.cuh"), os.path.join(CSRC, "hag_launch.h")]
 
 
 def _stale() -> bool:
@@ -32,7 +32,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", LIB]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += [os.path.join(CSRC, s) for s in SOURCES]
+    cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-ldl"]     # -ldl: the header-only NVTX ranges load their tool lazily
     subprocess.check_call(cmd)
     return LIB
 

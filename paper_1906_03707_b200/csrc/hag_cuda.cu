@@ -1,6 +1,7 @@
 // Device side of the C ABI: upload of the structure arrays and the launch
 // sequences of the forward / backward aggregation (Algorithm 2 and its adjoint).
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>      // header-only; a no-op unless a profiler is attached
 
 #include <algorithm>
 #include <cstdint>
@@ -12,21 +13,13 @@
 
 #include "hag_internal.h"
 #include "hag_kernels.cuh"
+#include "hag_launch.h"
 
 namespace {
 
-struct DeviceGuard {
-    int prev = -1;
-    bool ok = true;
-    explicit DeviceGuard(int dev) {
-        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
-        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
-    }
-    ~DeviceGuard() {
-        int cur = -1;
-        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
-    }
-};
+using hagl::aligned16;
+using hagl::DeviceGuard;
+using hagl::lanes_per_row;
 
 template <typename V>
 hag_status upload_i32(int32_t **dst, const V *src, size_t count) {
@@ -83,26 +76,9 @@ void free_device(hag *h) {
     d = hag_device_arrays{};
 }
 
-int lanes_per_row(int n_chunks) {
-    int l = 4;
-    while (l < 32 && l < n_chunks) l *= 2;
-    return l;
-}
-
-// Every kernel is launched with programmatic stream serialisation (see hag_kernels.cuh).
 template <typename Args>
 cudaError_t launch_pdl(void (*kernel)(Args), unsigned grid, const Args &args, cudaStream_t s) {
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(hagk::kThreads);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, args);
+    return hagl::launch_pdl(kernel, grid, unsigned(hagk::kThreads), args, s);
 }
 
 // Launch shape of the gather (loads in flight per lane, resident warps per SM,
@@ -285,11 +261,19 @@ struct Recorder {
     hag *h;
     cudaStream_t s;
     bool failed = false;
+    int open_ranges = 0;
     Recorder(const hag *h_, cudaStream_t s_) : h(const_cast<hag *>(h_)), s(s_) {
         h->notes.clear();
         h->last_launches = 0;
     }
+    ~Recorder() {                      // a launch that failed left its range open
+        while (open_ranges-- > 0) nvtxRangePop();
+    }
     void begin(int32_t kind, int64_t rows, int64_t edges) {
+        static const char *const names[4] = {"hag: level pair sums", "hag: gather over aggregation nodes",
+                                             "hag: gather over graph nodes", "hag: whole pass in one launch"};
+        nvtxRangePushA(names[kind & 3]);       // one range per launch, nested in the call's range
+        ++open_ranges;
         if (h->profile) {
             const size_t i = h->notes.size();
             while (h->events.size() < 2 * (i + 1)) {
@@ -307,10 +291,10 @@ struct Recorder {
             if (cudaEventRecord(h->events[2 * i + 1], s) != cudaSuccess) { cudaGetLastError(); failed = true; }
         }
         ++h->last_launches;
+        nvtxRangePop();
+        --open_ranges;
     }
 };
-
-bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 hag_status check_call(const hag *h, hag_dtype dtype, int32_t D, const void *in, const void *out) {
     if (!h || !in || !out) return HAG_ERR_NULL;
@@ -501,12 +485,14 @@ hag_status run(const hag *h, bool backward, bool use_hag, hag_reduce reduce, hag
     if (!guard.ok) { cudaGetLastError(); return HAG_ERR_CUDA; }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     Recorder rec(h, s);
+    nvtxRangePushA(use_hag ? (backward ? "hag_aggregate_bwd" : "hag_aggregate_fwd") : (backward ? "csr_aggregate_bwd" : "csr_aggregate_fwd"));
     if (dtype == HAG_F32)
         st = backward ? bwd_impl<float>(h, use_hag, reduce, D, in, out, ws, s, &rec)
                       : fwd_impl<float>(h, use_hag, reduce, D, in, out, ws, s, &rec);
     else
         st = backward ? bwd_impl<__nv_bfloat16>(h, use_hag, reduce, D, in, out, ws, s, &rec)
                       : fwd_impl<__nv_bfloat16>(h, use_hag, reduce, D, in, out, ws, s, &rec);
+    nvtxRangePop();
     if (st == HAG_OK && rec.failed) st = HAG_ERR_CUDA;
     return st;
 }

@@ -21,6 +21,7 @@
 #include "hag.h"
 #include "hag_internal.h"
 #include "hag_kernels.cuh"
+#include "hag_launch.h"
 
 namespace {
 
@@ -232,38 +233,15 @@ __global__ void __launch_bounds__(kThreads, MaxShape<T>::kBwdBlocks) gather_maxg
     }
 }
 
-struct DeviceScope {
-    int prev = -1;
-    bool ok = true;
-    explicit DeviceScope(int device) {
-        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
-        if (prev != device && cudaSetDevice(device) != cudaSuccess) ok = false;
-    }
-    ~DeviceScope() {
-        int cur = -1;
-        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
-    }
-};
+using DeviceScope = hagl::DeviceGuard;
+using hagl::aligned16;
 
 template <typename Args>
 cudaError_t launch(void (*kernel)(Args), int64_t warps, const Args &args, cudaStream_t s) {
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(unsigned((warps + kWarps - 1) / kWarps));
-    cfg.blockDim = dim3(kThreads);
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, args);
+    return hagl::launch_pdl(kernel, unsigned((warps + kWarps - 1) / kWarps), unsigned(kThreads), args, s);
 }
 
-int lanes_for(int n_chunks) {
-    int l = 4;
-    while (l < 32 && l < n_chunks) l *= 2;
-    return l;
-}
+inline int lanes_for(int n_chunks) { return hagl::lanes_per_row(n_chunks); }
 
 template <typename T>
 cudaError_t launch_rows(bool grad, const MaxArgs &a, cudaStream_t s) {
@@ -288,8 +266,6 @@ cudaError_t launch_pair_level(const PairMaxArgs &p, cudaStream_t s) {
         default: return launch(pair_max_kernel<T, 32>, warps, p, s);
     }
 }
-
-bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 hag_status check(const hag *h, hag_dtype dtype, int32_t D) {
     if (!h) return HAG_ERR_NULL;

@@ -10,6 +10,7 @@
 
 #include "hag.h"
 #include "hag_kernels.cuh"
+#include "hag_launch.h"
 
 namespace {
 
@@ -142,24 +143,11 @@ __global__ void __launch_bounds__(hagk::kThreads) graph_pool_bwd_kernel(const Po
     }
 }
 
-int pool_lanes_per_row(int n_chunks) {
-    int l = 4;
-    while (l < 32 && l < n_chunks) l *= 2;
-    return l;
-}
+inline int pool_lanes_per_row(int n_chunks) { return hagl::lanes_per_row(n_chunks); }
 
-template <typename Kernel>
-cudaError_t launch_pool(Kernel kernel, int64_t items, const PoolArgs &p, cudaStream_t s) {
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(unsigned((items + hagk::kWarps - 1) / hagk::kWarps));
-    cfg.blockDim = dim3(hagk::kThreads);
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, p);
+template <typename Args>
+cudaError_t launch_pool(void (*kernel)(Args), int64_t items, const PoolArgs &p, cudaStream_t s) {
+    return hagl::launch_pdl(kernel, unsigned((items + hagk::kWarps - 1) / hagk::kWarps), unsigned(hagk::kThreads), p, s);
 }
 
 template <typename T, bool BWD>
