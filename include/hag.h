@@ -168,6 +168,17 @@ int32_t hag_build_threads(int32_t threads);
  * `src` stopped only because it hit its own capacity. */
 hag_status hag_truncate(const hag_t *src, int32_t capacity, hag_t **out);
 
+/* The HAG of a graph from a merge trace recorded earlier (hag_export's `trace`: 3 int32 per merge, v1 < v2 in
+ * creation ids, redundancy), without running the search again: a 30-second build becomes a replay of a second or
+ * two (the paper computes a HAG once per graph and reuses it: Section 5.1).  Every merge is checked as it is
+ * replayed: ids in range and ordered, recorded redundancy >= 2 and equal to the number of rows that hold both nodes
+ * at that point, so the result is always a correct HAG of THIS graph (Theorem 2's cover condition holds by
+ * construction); it equals hag_build's bit for bit when the trace came from hag_build on the same graph, which is
+ * not checked (whether each merge was the arg-max is the search's business).  The handle's capacity is num_merges.
+ * Errors: as hag_build for the graph; NULL (trace missing); ARG (num_merges < 0, or a merge that does not replay). */
+hag_status hag_import(int32_t n, const int64_t *row_ptr, const int32_t *col_idx, int32_t num_merges, const int32_t *trace,
+                      hag_t **out);
+
 /* Replaces the cuts that hag_build chose (see there) and rebuilds the expansion lists of the
  * deep levels.  Every cut 0 <= c <= num_levels evaluates the same HAG to the same values up to
  * the order of additions (Section 3.1, Eq. 1: a node is the Aggregate over its cover); the

@@ -26,7 +26,7 @@ HAG_F32, HAG_BF16 = 0, 1
  HAG_ERR_ALIGN, HAG_ERR_WORKSPACE, HAG_ERR_TIMEOUT, HAG_ERR_NOT_ON_DEVICE, HAG_ERR_TOO_LARGE) = range(13)
 
 EXPORTED_SYMBOLS = [
-    "hag_build", "hag_build_ex", "hag_build_threads", "hag_truncate", "hag_set_cuts", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes", "csr_workspace_bytes",
+    "hag_build", "hag_build_ex", "hag_build_threads", "hag_truncate", "hag_import", "hag_set_cuts", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes", "csr_workspace_bytes",
     "hag_aggregate_fwd", "hag_aggregate_bwd", "csr_aggregate_fwd", "csr_aggregate_bwd",
     "hag_aggregate_host", "hag_aggregate_fwd_static", "hag_graph_pool_fwd", "hag_graph_pool_bwd",
     "hag_max_workspace_bytes", "hag_max_fwd", "hag_max_bwd", "csr_max_fwd", "csr_max_bwd", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
@@ -90,6 +90,8 @@ def load_library():
     lib.hag_build_threads.restype = i32
     lib.hag_truncate.argtypes = [vp, i32, ctypes.POINTER(vp)]
     lib.hag_truncate.restype = ctypes.c_int
+    lib.hag_import.argtypes = [i32, vp, vp, i32, vp, ctypes.POINTER(vp)]
+    lib.hag_import.restype = ctypes.c_int
     lib.hag_set_cuts.argtypes = [vp, i32, i32]
     lib.hag_set_cuts.restype = ctypes.c_int
     lib.hag_destroy.argtypes = [vp]
@@ -200,6 +202,19 @@ class Hag:
         st = lib.hag_build_ex(n, rp.ctypes.data, ci.ctypes.data if ci.size else None, int(capacity),
                               int(min_redundancy), ctypes.byref(handle))
         _check(st, "hag_build")
+        return cls(handle)
+
+    @classmethod
+    def from_trace(cls, row_ptr, col_idx, trace) -> "Hag":
+        """``hag_import``: the HAG of the graph from a recorded merge trace (``arrays()["trace"]``), no search."""
+        lib = load_library()
+        rp = np.ascontiguousarray(row_ptr, dtype=np.int64)
+        ci = np.ascontiguousarray(col_idx, dtype=np.int32)
+        tr = np.ascontiguousarray(np.asarray(trace, dtype=np.int32).reshape(-1, 3))
+        handle = ctypes.c_void_p()
+        st = lib.hag_import(rp.shape[0] - 1, rp.ctypes.data, ci.ctypes.data if ci.size else None, tr.shape[0],
+                            tr.ctypes.data if tr.size else None, ctypes.byref(handle))
+        _check(st, "hag_import")
         return cls(handle)
 
     def truncate(self, capacity: int) -> "Hag":

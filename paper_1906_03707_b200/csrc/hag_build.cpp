@@ -788,20 +788,17 @@ extern "C" hag_status hag_build(int32_t n, const int64_t *row_ptr, const int32_t
     return hag_build_ex(n, row_ptr, col_idx, capacity, 2, out);
 }
 
-extern "C" hag_status hag_build_ex(int32_t n, const int64_t *row_ptr, const int32_t *col_idx, int32_t capacity,
-                                   int32_t min_redundancy, hag_t **out) {
-    if (!out) return HAG_ERR_NULL;
-    *out = nullptr;
-    if (min_redundancy < 2) return HAG_ERR_ARG;
+namespace {
+
+// Argument and graph checks shared by hag_build_ex and hag_import; nothing reads through the CSR before they pass.
+hag_status validate_graph(int32_t n, const int64_t *row_ptr, const int32_t *col_idx, int64_t capacity) {
     if (!row_ptr || (!col_idx && n > 0 && row_ptr[n] > 0)) return HAG_ERR_NULL;
     if (n < 0 || capacity < 0) return HAG_ERR_ARG;
-    if (int64_t(n) + int64_t(capacity) >= (int64_t(1) << 31)) return HAG_ERR_ARG;
-    // validate the CSR before anything reads through it
+    if (int64_t(n) + capacity >= (int64_t(1) << 31)) return HAG_ERR_ARG;
     if (row_ptr[0] != 0) return HAG_ERR_GRAPH;
     for (int32_t v = 0; v < n; ++v)
         if (row_ptr[v + 1] < row_ptr[v]) return HAG_ERR_GRAPH;
-    const int64_t e = row_ptr[n];
-    if (e >= (int64_t(1) << 31)) return HAG_ERR_ARG;
+    if (row_ptr[n] >= (int64_t(1) << 31)) return HAG_ERR_ARG;
     for (int32_t v = 0; v < n; ++v) {
         int64_t prev = -1;
         for (int64_t i = row_ptr[v]; i < row_ptr[v + 1]; ++i) {
@@ -810,6 +807,12 @@ extern "C" hag_status hag_build_ex(int32_t n, const int64_t *row_ptr, const int3
             prev = c;
         }
     }
+    return HAG_OK;
+}
+
+// Builds a handle from the graph and either the search (trace == nullptr) or a recorded trace of num_merges merges.
+hag_status build_handle(int32_t n, const int64_t *row_ptr, const int32_t *col_idx, int32_t capacity, int32_t min_redundancy,
+                        const int32_t *trace, int32_t num_merges, hag_t **out) {
     const auto t0 = std::chrono::steady_clock::now();
     hag *h = new (std::nothrow) hag();
     if (!h) return HAG_ERR_OOM_HOST;
@@ -818,13 +821,30 @@ extern "C" hag_status hag_build_ex(int32_t n, const int64_t *row_ptr, const int3
         h->n = n;
         h->capacity = capacity;
         h->min_redundancy = min_redundancy;
-        h->e = e;
+        h->e = row_ptr[n];
         h->csr_ptr.assign(row_ptr, row_ptr + n + 1);
-        h->csr_idx.assign(col_idx, col_idx + e);
+        h->csr_idx.assign(col_idx, col_idx + h->e);
         h->in_degree.resize(n);
         for (int32_t v = 0; v < n; ++v) h->in_degree[v] = int32_t(row_ptr[v + 1] - row_ptr[v]);
         std::vector<int32_t> rows_store, rows_len;
-        st = hag_search(h, rows_store, rows_len);
+        if (!trace) {
+            st = hag_search(h, rows_store, rows_len);
+        } else {
+            if (hag_alloc_should_fail(0)) throw std::bad_alloc();
+            rows_store = h->csr_idx;
+            rows_len.resize(n);
+            for (int32_t u = 0; u < n; ++u) rows_len[u] = int32_t(h->csr_ptr[u + 1] - h->csr_ptr[u]);
+            if (num_merges > 0) {
+                const std::vector<int32_t> recorded(trace, trace + size_t(3) * num_merges);
+                for (int32_t i = 0; i < num_merges; ++i)
+                    if (recorded[3 * i + 2] < 2) st = HAG_ERR_ARG;           // not a merge Algorithm 3 would make
+                if (st == HAG_OK) {
+                    Searcher s(n, num_merges, h->csr_ptr.data(), rows_store, rows_len);
+                    st = s.replay(recorded, num_merges, h->trace);
+                }
+            }
+            h->num_agg = int32_t(h->trace.size() / 3);
+        }
         if (st == HAG_OK) st = hag_layout(h, rows_store, rows_len);
     } catch (const std::bad_alloc &) {
         st = HAG_ERR_OOM_HOST;
@@ -836,6 +856,30 @@ extern "C" hag_status hag_build_ex(int32_t n, const int64_t *row_ptr, const int3
     h->info.build_seconds = std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count();
     *out = h;
     return HAG_OK;
+}
+
+}  // namespace
+
+extern "C" hag_status hag_build_ex(int32_t n, const int64_t *row_ptr, const int32_t *col_idx, int32_t capacity,
+                                   int32_t min_redundancy, hag_t **out) {
+    if (!out) return HAG_ERR_NULL;
+    *out = nullptr;
+    if (min_redundancy < 2) return HAG_ERR_ARG;
+    const hag_status st = validate_graph(n, row_ptr, col_idx, capacity);
+    if (st != HAG_OK) return st;
+    return build_handle(n, row_ptr, col_idx, capacity, min_redundancy, nullptr, 0, out);
+}
+
+extern "C" hag_status hag_import(int32_t n, const int64_t *row_ptr, const int32_t *col_idx, int32_t num_merges,
+                                 const int32_t *trace, hag_t **out) {
+    if (!out) return HAG_ERR_NULL;
+    *out = nullptr;
+    if (num_merges < 0) return HAG_ERR_ARG;
+    if (num_merges > 0 && !trace) return HAG_ERR_NULL;
+    const hag_status st = validate_graph(n, row_ptr, col_idx, num_merges);
+    if (st != HAG_OK) return st;
+    static const int32_t no_merges[3] = {0, 0, 0};          // (a non-null trace is what selects the replay)
+    return build_handle(n, row_ptr, col_idx, num_merges, 2, trace ? trace : no_merges, num_merges, out);
 }
 
 extern "C" int32_t hag_build_threads(int32_t threads) {

@@ -59,8 +59,9 @@ struct PairMaxArgs {
 
 // Launch shapes from a sweep on B200 (loads or entries in flight per lane, resident CTAs per SM):
 // more resident warps beat more loads per warp, as for the sum kernels.
-//   fp32: forward 4 loads x 10 CTAs, backward 2 entries x 10 CTAs; bf16: forward 2 x 10, backward 1 x 8.
-#define HAG_MAX_SHAPES 4, 10, 2, 10, 2, 10, 1, 8
+//   fp32: forward 4 loads x 10 CTAs, backward 2 entries x 10 CTAs; bf16: forward 4 x 12 (raw word groups: 4 registers
+//   per load in flight), backward 1 x 8.
+#define HAG_MAX_SHAPES 4, 10, 2, 10, 4, 12, 1, 8
 template <typename T> struct MaxShape;
 template <int FL, int FB, int BE, int BB, int HFL, int HFB, int HBE, int HBB> struct MaxShapeTable {
     static constexpr int f32[4] = {FL, FB, BE, BB};
@@ -76,12 +77,23 @@ template <> struct MaxShape<__nv_bfloat16> {
     static constexpr int kBwdEntries = MaxShapes::bf16[2], kBwdBlocks = MaxShapes::bf16[3];
 };
 
+// Packed maximum of two bf16 pairs (one instruction for two values; exact, as every maximum is).
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t x, uint32_t y) {
+    const __nv_bfloat162 r = __hmax2(*reinterpret_cast<const __nv_bfloat162 *>(&x), *reinterpret_cast<const __nv_bfloat162 *>(&y));
+    return *reinterpret_cast<const uint32_t *>(&r);
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {      // exact for values that are bf16 already
+    const __nv_bfloat162 r = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&r);
+}
+
 template <typename T, int LPR>
 __global__ void __launch_bounds__(kThreads, MaxShape<T>::kFwdBlocks) gather_max_kernel(const MaxArgs a) {
     hagk::pdl_launch_dependents();
     constexpr int E = Chunk<T>::kElems;
     constexpr int G = 32 / LPR;
     constexpr int U = MaxShape<T>::kFwdLoads < LPR ? MaxShape<T>::kFwdLoads : LPR;
+    constexpr unsigned FULL = 0xffffffffu;
     const int lane = threadIdx.x & 31;
     const int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
     if (r_local >= a.row_count) return;
@@ -96,46 +108,116 @@ __global__ void __launch_bounds__(kThreads, MaxShape<T>::kFwdBlocks) gather_max_
         const int chunk = c0 + gl;
         const bool live = chunk < n_chunks;
         const Tables<T> tab(a.val_prim, a.val_sec, a.n_prim, a.D, live ? chunk : 0);
-        float acc[E];
-#pragma unroll
-        for (int j = 0; j < E; ++j) acc[j] = ninf;
         int32_t mine = (c0 == 0) ? first : ((b + lane < e) ? __ldg(a.idx + b + lane) : -1);
-        for (int32_t base = b; base < e; base += 32) {
-            const int32_t cur = mine;
-            const int32_t nb = base + 32;
-            mine = (nb + lane < e) ? __ldg(a.idx + nb + lane) : -1;
-            const int cnt = min(32, e - base);
+        if constexpr (E == 8) {
+            // bf16 storage: the maximum is taken on the raw bf16 pairs (max.bf16x2: 4 instructions per 16 bytes, no
+            // widening), U raw word groups in flight.  The ids of a row ascend, so the bf16 rows (the first n_p entries
+            // of a batch) and the fp32 rows of aggregation nodes (whose values are bf16 values) have a loop each.
+            constexpr uint32_t kNinf2 = 0xff80ff80u;
+            uint32_t m[4] = {kNinf2, kNinf2, kNinf2, kNinf2};
+            for (int32_t base = b; base < e; base += 32) {
+                const int32_t cur = mine;
+                const int32_t nb = base + 32;
+                mine = (nb + lane < e) ? __ldg(a.idx + nb + lane) : -1;
+                const int cnt = min(32, e - base);
+                const int n_p = __popc(__ballot_sync(FULL, cur >= 0 && cur < a.n_prim));
 #pragma unroll
-            for (int k = 0; k < LPR; k += U) {
-                if (k * G < cnt) {
-                    float v[U][E];
+                for (int k = 0; k < LPR; k += U) {
+                    if (k * G < n_p) {
+                        uint4 raw[U];
+                        if ((k + U) * G <= n_p) {       // a full group: no checks (lanes beyond the row width read chunk 0, never stored)
 #pragma unroll
-                    for (int u = 0; u < U; ++u) {
-                        const int32_t id = __shfl_sync(0xffffffffu, cur, (k + u) * G + slice);
-                        if (id >= 0 && live) {
-                            tab.load(id, v[u]);
+                            for (int u = 0; u < U; ++u)
+                                raw[u] = hagk::ld_u4(tab.prim + size_t(uint32_t(__shfl_sync(FULL, cur, (k + u) * G + slice))) * tab.prim_row_bytes);
                         } else {
 #pragma unroll
-                            for (int j = 0; j < E; ++j) v[u][j] = ninf;
+                            for (int u = 0; u < U; ++u) {
+                                const int32_t id = __shfl_sync(FULL, cur, (k + u) * G + slice);
+                                raw[u] = ((k + u) * G + slice < n_p && live) ? hagk::ld_u4(tab.prim + size_t(uint32_t(id)) * tab.prim_row_bytes)
+                                                                             : make_uint4(kNinf2, kNinf2, kNinf2, kNinf2);
+                            }
+                        }
+#pragma unroll
+                        for (int u = 0; u < U; ++u) {
+                            m[0] = max_bf16x2(m[0], raw[u].x);
+                            m[1] = max_bf16x2(m[1], raw[u].y);
+                            m[2] = max_bf16x2(m[2], raw[u].z);
+                            m[3] = max_bf16x2(m[3], raw[u].w);
                         }
                     }
-#pragma unroll
-                    for (int u = 0; u < U; ++u)
-#pragma unroll
-                        for (int j = 0; j < E; ++j) acc[j] = fmaxf(acc[j], v[u][j]);
+                }
+                for (int j0 = n_p; j0 < cnt; j0 += G) {
+                    const int j = j0 + slice;
+                    const int32_t id = __shfl_sync(FULL, cur, j < cnt ? j : 0);
+                    if (j < cnt && live) {
+                        const char *p = tab.sec + size_t(uint32_t(id)) * tab.sec_row_bytes;
+                        const float4 q0 = hagk::ld_f4(p), q1 = hagk::ld_f4(p + 16);
+                        m[0] = max_bf16x2(m[0], pack_bf16x2(q0.x, q0.y));
+                        m[1] = max_bf16x2(m[1], pack_bf16x2(q0.z, q0.w));
+                        m[2] = max_bf16x2(m[2], pack_bf16x2(q1.x, q1.y));
+                        m[3] = max_bf16x2(m[3], pack_bf16x2(q1.z, q1.w));
+                    }
                 }
             }
-        }
 #pragma unroll
-        for (int off = LPR; off < 32; off <<= 1)
+            for (int off = LPR; off < 32; off <<= 1)
 #pragma unroll
-            for (int j = 0; j < E; ++j) acc[j] = fmaxf(acc[j], __shfl_xor_sync(0xffffffffu, acc[j], off));
-        if (live && slice == 0) {
-            if (e == b) {                 // empty neighbourhood: zero row
+                for (int i = 0; i < 4; ++i) m[i] = max_bf16x2(m[i], __shfl_xor_sync(FULL, m[i], off));
+            if (live && slice == 0) {
+                float acc[E];
+                hagk::bf16x8_to_f32(make_uint4(m[0], m[1], m[2], m[3]), acc);
+                if (e == b) {                 // empty neighbourhood: zero row
 #pragma unroll
-                for (int j = 0; j < E; ++j) acc[j] = 0.0f;
+                    for (int j = 0; j < E; ++j) acc[j] = 0.0f;
+                }
+                hagk::store_chunk<T>(a.out, a.out_is_f32, a.D, row - a.out_row_offset, chunk, acc);
             }
-            hagk::store_chunk<T>(a.out, a.out_is_f32, a.D, row - a.out_row_offset, chunk, acc);
+        } else {
+            float acc[E];
+#pragma unroll
+            for (int j = 0; j < E; ++j) acc[j] = ninf;
+            for (int32_t base = b; base < e; base += 32) {
+                const int32_t cur = mine;
+                const int32_t nb = base + 32;
+                mine = (nb + lane < e) ? __ldg(a.idx + nb + lane) : -1;
+                const int cnt = min(32, e - base);
+#pragma unroll
+                for (int k = 0; k < LPR; k += U) {
+                    if (k * G < cnt) {
+                        float v[U][E];
+                        if ((k + U) * G <= cnt) {       // a full group: no checks, no fill (lanes beyond the row width read chunk 0, never stored)
+#pragma unroll
+                            for (int u = 0; u < U; ++u) tab.load(__shfl_sync(FULL, cur, (k + u) * G + slice), v[u]);
+                        } else {
+#pragma unroll
+                            for (int u = 0; u < U; ++u) {
+                                const int32_t id = __shfl_sync(FULL, cur, (k + u) * G + slice);
+                                if (id >= 0 && live) {
+                                    tab.load(id, v[u]);
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < E; ++j) v[u][j] = ninf;
+                                }
+                            }
+                        }
+#pragma unroll
+                        for (int u = 0; u < U; ++u)
+#pragma unroll
+                            for (int j = 0; j < E; ++j) acc[j] = fmaxf(acc[j], v[u][j]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int off = LPR; off < 32; off <<= 1)
+#pragma unroll
+                for (int j = 0; j < E; ++j) acc[j] = fmaxf(acc[j], __shfl_xor_sync(FULL, acc[j], off));
+            if (live && slice == 0) {
+                if (e == b) {                 // empty neighbourhood: zero row
+#pragma unroll
+                    for (int j = 0; j < E; ++j) acc[j] = 0.0f;
+                }
+                hagk::store_chunk<T>(a.out, a.out_is_f32, a.D, row - a.out_row_offset, chunk, acc);
+            }
         }
     }
 }

@@ -415,3 +415,43 @@ def test_injected_host_allocation_failures_return_a_status_and_leave_nothing_beh
         assert lib.hag_test_fail_allocation(2, 0) == 2
     finally:
         lib.hag_test_fail_allocation(0, -1)
+
+
+def test_import_of_a_recorded_trace_reproduces_the_build_and_rejects_what_does_not_replay():
+    import hashlib
+
+    def digest(h):
+        arr = h.arrays()
+        dig = hashlib.sha256()
+        for k in sorted(arr):
+            dig.update(np.ascontiguousarray(arr[k]).tobytes() if hasattr(arr[k], "tobytes") else str(arr[k]).encode())
+        info = {k: v for k, v in h.info().items() if k not in ("build_seconds", "capacity")}
+        return dig.hexdigest(), info
+
+    g = synth.config2_graph(seed=17, n=6000, n_comm=40)
+    built = hb.Hag.build(g.row_ptr, g.col_idx, g.n // 4)
+    trace = built.arrays()["trace"]
+    assert digest(hb.Hag.from_trace(g.row_ptr, g.col_idx, trace)) == digest(built)
+    # a prefix of the trace is the HAG of the smaller capacity; no trace is the GNN-graph itself
+    assert digest(hb.Hag.from_trace(g.row_ptr, g.col_idx, trace[:100])) == digest(hb.Hag.build(g.row_ptr, g.col_idx, 100))
+    assert hb.Hag.from_trace(g.row_ptr, g.col_idx, trace[:0]).info()["num_agg"] == 0
+    lib = hb.load_library()
+    out = ctypes.c_void_p()
+
+    def imp(tr, rp=g.row_ptr, ci=g.col_idx):
+        tr = np.ascontiguousarray(tr, dtype=np.int32)
+        return lib.hag_import(g.n, rp.ctypes.data, ci.ctypes.data, tr.shape[0], tr.ctypes.data, ctypes.byref(out))
+
+    wrong = trace.copy()
+    wrong[5, 2] += 1                                   # a redundancy the rows do not have
+    assert imp(wrong) == 2 and out.value is None
+    wrong = trace.copy()
+    wrong[7, :2] = wrong[7, 1], wrong[7, 0]            # pair out of order
+    assert imp(wrong) == 2
+    wrong = trace.copy()
+    wrong[3, 1] = g.n + 50                             # a node that does not exist yet
+    assert imp(wrong) == 2
+    other = synth.config2_graph(seed=18, n=6000, n_comm=40)
+    assert imp(trace, other.row_ptr, other.col_idx) == 2      # the trace of another graph does not replay
+    assert lib.hag_import(g.n, g.row_ptr.ctypes.data, g.col_idx.ctypes.data, 3, None, ctypes.byref(out)) == 1
+    assert lib.hag_import(g.n, g.row_ptr.ctypes.data, g.col_idx.ctypes.data, -1, None, ctypes.byref(out)) == 2
