@@ -256,7 +256,7 @@ class Runner:
         if args.cuts:
             h.set_cuts(*(int(v) for v in args.cuts.split(",")))
         h.to_device(local_rank)
-        h.set_schedule(args.single_launch)
+        h.set_schedule(args.schedule)
         self.build_s = time.perf_counter() - t0
         self.h = h
         self.info = h.info()
@@ -333,7 +333,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-per-config", action="store_true", help="measure the headline workload only")
-    ap.add_argument("--single-launch", action="store_true", help="one launch per pass instead of a launch per level (hag_set_schedule 1)")
+    ap.add_argument("--schedule", type=int, default=0, choices=[0, 1, 2],
+                    help="hag_set_schedule: 0 a launch per level, 1 one launch per pass, 2 the aggregation nodes in one launch "
+                         "and the graph nodes in a second")
+    ap.add_argument("--single-launch", action="store_const", const=1, dest="schedule", help="same as --schedule 1")
     ap.add_argument("--cuts", type=str, default="", help="forced cuts 'fwd,bwd' (hag_set_cuts); default: the library's choice")
     ap.add_argument("--shard", default="replicas", choices=["replicas", "graphs", "columns"],
                     help="N > 1: one whole workload per rank (weak), the graphs of workload 4 split over ranks, or the "
@@ -540,7 +543,7 @@ def main():
         keep_h, keep_ws, keep_nb = r.h, r.ws, r.nbytes
         for frac_name, cap in (("0", 0), ("N/8", g.n // 8), ("N/4", g.n // 4), ("N/2", g.n // 2)):
             hc = big.truncate(cap).to_device(local_rank)
-            hc.set_schedule(args.single_launch)
+            hc.set_schedule(args.schedule)
             ic, ac = hc.info(), hc.arrays()
             r.h, r.nbytes = hc, algorithmic_bytes(g.n, r.d, w.dtype, ac, ic)
             r.ws = torch.empty(max(hc.workspace_bytes(r.d), hc.csr_workspace_bytes(r.d), 16) // 4, dtype=torch.float32, device=dev)
@@ -601,13 +604,13 @@ def main():
     if rank == 0:
         value = total_bytes / (hag_ms * 1e-3) / 1e9
         ncu = NCU_FWD_GATHER.get(w.name) if (args.scale == 1.0 and not args.permute_ids and column_slice is None
-                                            and not args.single_launch and not args.cuts and world == 1) else None
+                                            and not args.schedule and not args.cuts and world == 1) else None
         traffic = ncu["dram_bytes"] if ncu else None
         dram_frac = (traffic / (dom_ms * 1e-3) / 1e9 / peak) if traffic else None
         l2_frac = (ncu["lts_throughput_pct"] / 100.0) if ncu else None
         # the rows come from HBM only when the matrices do not fit in L2; otherwise the L2 / load path binds
         if dram_frac is not None:
-            bound = "hbm" if dram_frac >= 0.2 else "l2"
+            bound = "hbm" if dram_frac >= l2_frac else "l2"      # whichever of the two measured fractions is nearer its peak
         else:
             bound = "hbm" if x_bytes > (126 << 20) else "l2"
         line = {
@@ -619,7 +622,7 @@ def main():
                 "l2": "flushed between timed steps (256 MiB write outside the per-step events)",
                 "timing": "sum of per-step CUDA-event intervals on the launching stream, max over ranks",
                 "clocks": "nvidia-smi sampled every 100 ms across all GPU arms",
-                "schedule": "one launch per pass" if args.single_launch else "a launch per level",
+                "schedule": ("a launch per level", "one launch per pass", "aggregation nodes in one launch, graph nodes in a second")[args.schedule],
                 "ranks": shard_note,
             },
             "clocks": clocks,

@@ -380,9 +380,14 @@ hag_status hag_aggregate_fwd_static(const hag_t *h, hag_reduce reduce, hag_dtype
  *                Measured on B200 this form is level with the default on the two largest fp32 shapes and
  *                slower on small graphs and deep hierarchies (resident warps hide less latency than the
  *                hardware's block scheduling does on launches of 10^5 rows), which is why it is not the default.
+ *   2            TWO launches per pass: the rows of the aggregation nodes (every phase of the list of form 1 before
+ *                the graph nodes) in one launch of that kernel, then the graph nodes by the row kernels of form
+ *                0.  For hierarchies of many small levels, where form 0 spends most of a pass launching and
+ *                draining kernels of a few thousand rows; the same bounded waits and the same report apply.
+ *                The plain-CSR calls are not affected (they have no aggregation nodes).
  * Passes whose hierarchy has more than 56 phases always run level by level.
- * Errors: NULL; ARG (a value other than 0 or 1). */
-hag_status hag_set_schedule(hag_t *h, int32_t single_launch);
+ * Errors: NULL; ARG (a value other than 0, 1 or 2). */
+hag_status hag_set_schedule(hag_t *h, int32_t schedule);
 
 /* HAG_OK, or HAG_ERR_TIMEOUT if a bounded device-side wait of an earlier call on this handle gave up
  * (reading clears it).  Does not synchronise: call it after synchronising the stream of the calls
@@ -410,6 +415,18 @@ typedef struct hag_pass_view {
     const int32_t *ids;         /* [n_ids]       */
 } hag_pass_view;
 hag_status hag_export_pass(const hag_t *h, int32_t pass, hag_pass_view *out);
+
+/* The order in which the kernels that walk several rows per warp take the rows of one list (feature rows of 256 bytes
+ * or less: every group of lanes walks a row of its own, in lock step with the warp's other groups, so rows of like
+ * length belong side by side).  list: 0 residual rows (Algorithm 2 lines 7-8), 1 transposed HAG, 2 input graph
+ * (Algorithm 1 line 4), 3 its transpose, 4 / 5 the expansion lists of the forward / backward cut.  order[i] is the
+ * row taking the place of row first_row + i: a permutation that sorts the rows by length (longest first) within
+ * windows of 2048 rows, the windows never crossing from the graph nodes into a level or from one level into the next,
+ * so every launch's rows map onto themselves.  count = 0 (order NULL): the rows are taken as they are (pairs of
+ * neighbouring rows already lose less than 8 % of the lock-step rounds).  No value depends on the order: each row is
+ * summed by one group in the row's own order of entries.  The array lives as long as the handle; hag_set_cuts
+ * rebuilds lists 4 and 5.  Errors: NULL, ARG (list outside 0..5). */
+hag_status hag_export_row_order(const hag_t *h, int32_t list, int32_t *first_row, int64_t *count, const int32_t **order);
 
 /* Test hook (process-wide): makes one of the library's next allocation attempts fail as if memory had run out,
  * so that callers can exercise their handling of HAG_ERR_OOM_HOST / HAG_ERR_OOM_DEVICE.  kind 0: host memory

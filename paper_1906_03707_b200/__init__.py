@@ -26,7 +26,7 @@ HAG_F32, HAG_BF16 = 0, 1
  HAG_ERR_ALIGN, HAG_ERR_WORKSPACE, HAG_ERR_TIMEOUT, HAG_ERR_NOT_ON_DEVICE, HAG_ERR_TOO_LARGE) = range(13)
 
 EXPORTED_SYMBOLS = [
-    "hag_build", "hag_build_ex", "hag_build_threads", "hag_truncate", "hag_import", "hag_set_cuts", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes", "csr_workspace_bytes",
+    "hag_build", "hag_build_ex", "hag_build_threads", "hag_truncate", "hag_import", "hag_export_row_order", "hag_set_cuts", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes", "csr_workspace_bytes",
     "hag_aggregate_fwd", "hag_aggregate_bwd", "csr_aggregate_fwd", "csr_aggregate_bwd",
     "hag_aggregate_host", "hag_aggregate_fwd_static", "hag_graph_pool_fwd", "hag_graph_pool_bwd",
     "hag_max_workspace_bytes", "hag_max_fwd", "hag_max_bwd", "csr_max_fwd", "csr_max_bwd", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
@@ -90,6 +90,8 @@ def load_library():
     lib.hag_build_threads.restype = i32
     lib.hag_truncate.argtypes = [vp, i32, ctypes.POINTER(vp)]
     lib.hag_truncate.restype = ctypes.c_int
+    lib.hag_export_row_order.argtypes = [vp, i32, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(vp)]
+    lib.hag_export_row_order.restype = ctypes.c_int
     lib.hag_import.argtypes = [i32, vp, vp, i32, vp, ctypes.POINTER(vp)]
     lib.hag_import.restype = ctypes.c_int
     lib.hag_set_cuts.argtypes = [vp, i32, i32]
@@ -278,9 +280,18 @@ class Hag:
         return dict(rows=_view(v.rows, 4 * v.n_rows, np.int32).reshape(-1, 4), phase_size=_view(v.phase_size, v.n_phases, np.int32),
                     ids=_view(v.ids, v.n_ids, np.int32), n_chunk_rows=int(v.n_chunk_rows))
 
-    def set_schedule(self, single_launch: bool) -> "Hag":
-        """``hag_set_schedule``: a launch per level (default) or one launch per pass."""
-        _check(load_library().hag_set_schedule(self._h, int(bool(single_launch))), "hag_set_schedule")
+    def row_order(self, which: int):
+        """``hag_export_row_order``: (first_row, order) of one list; order is empty where rows are taken as they are."""
+        first, count, ptr = ctypes.c_int32(), ctypes.c_int64(), ctypes.c_void_p()
+        _check(load_library().hag_export_row_order(self._h, int(which), ctypes.byref(first), ctypes.byref(count), ctypes.byref(ptr)),
+               "hag_export_row_order")
+        order = _view(ptr.value, count.value, np.int32).copy() if count.value else np.zeros(0, np.int32)
+        return int(first.value), order
+
+    def set_schedule(self, schedule) -> "Hag":
+        """``hag_set_schedule``: 0 / False a launch per level, 1 / True one launch per pass, 2 the aggregation nodes in one
+        launch and the graph nodes in a second."""
+        _check(load_library().hag_set_schedule(self._h, int(schedule)), "hag_set_schedule")
         return self
 
     def device_status(self) -> int:

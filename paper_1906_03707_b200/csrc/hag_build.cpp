@@ -479,12 +479,46 @@ void build_segments(hag *h) {
             }
         }
     };
+    // the row order of the several-rows-per-warp kernels (see seg_set); `bounds`: ascending local row indices where
+    // launches begin (0 and rows included)
+    auto order = [](seg_set &set, const std::vector<int64_t> &ptr, int64_t rows, int32_t first_row_id, const std::vector<int64_t> &bounds) {
+        set.order.clear();
+        set.order_first_row = first_row_id;
+        if (rows < 2) return;
+        auto rounds = [&](int64_t r) { return (ptr[r + 1] - ptr[r] + 3) / 4; };
+        int64_t own = 0, paired = 0;
+        for (int64_t r = 0; r < rows; r += 2) {
+            const int64_t a = rounds(r), b = r + 1 < rows ? rounds(r + 1) : 0;
+            own += a + b;
+            paired += 2 * std::max(a, b);
+        }
+        if (double(paired) < kOrderMinWaste * double(std::max<int64_t>(own, 1))) return;
+        set.order.resize(size_t(rows));
+        for (int64_t r = 0; r < rows; ++r) set.order[size_t(r)] = int32_t(first_row_id + r);
+        for (size_t i = 0; i + 1 < bounds.size(); ++i)
+            for (int64_t w0 = bounds[i]; w0 < bounds[i + 1]; w0 += kOrderWindow) {
+                const int64_t w1 = std::min<int64_t>(w0 + kOrderWindow, bounds[i + 1]);
+                std::stable_sort(set.order.begin() + w0, set.order.begin() + w1, [&](int32_t x, int32_t y) {
+                    const int64_t lx = ptr[x - first_row_id + 1] - ptr[x - first_row_id], ly = ptr[y - first_row_id + 1] - ptr[y - first_row_id];
+                    return lx > ly;
+                });
+            }
+    };
+    std::vector<int64_t> t_bounds{0, n};
+    for (size_t l = 1; l < h->level_ptr.size(); ++l) t_bounds.push_back(n + h->level_ptr[l]);
+    const int64_t f_rows = int64_t(h->ftail_ptr.size()) - 1, b_rows = int64_t(h->btail_ptr.size()) - 1;
     build(h->seg_res, h->res_ptr, n, 0);
     build(h->seg_t, h->t_ptr, int64_t(n) + k, 0);
     build(h->seg_csr, h->csr_ptr, n, 0);
     build(h->seg_csr_t, h->csr_t_ptr, n, 0);
-    build(h->seg_ftail, h->ftail_ptr, int64_t(h->ftail_ptr.size()) - 1, int32_t(n + h->level_ptr[h->fwd_cut]));
-    build(h->seg_btail, h->btail_ptr, int64_t(h->btail_ptr.size()) - 1, int32_t(n + h->level_ptr[h->bwd_cut]));
+    build(h->seg_ftail, h->ftail_ptr, f_rows, int32_t(n + h->level_ptr[h->fwd_cut]));
+    build(h->seg_btail, h->btail_ptr, b_rows, int32_t(n + h->level_ptr[h->bwd_cut]));
+    order(h->seg_res, h->res_ptr, n, 0, {0, n});
+    order(h->seg_t, h->t_ptr, int64_t(n) + k, 0, t_bounds);
+    order(h->seg_csr, h->csr_ptr, n, 0, {0, n});
+    order(h->seg_csr_t, h->csr_t_ptr, n, 0, {0, n});
+    order(h->seg_ftail, h->ftail_ptr, f_rows, int32_t(n + h->level_ptr[h->fwd_cut]), {0, std::max<int64_t>(f_rows, 0)});
+    order(h->seg_btail, h->btail_ptr, b_rows, int32_t(n + h->level_ptr[h->bwd_cut]), {0, std::max<int64_t>(b_rows, 0)});
     h->max_segs_hag = std::max(std::max(h->seg_res.max_count(), h->seg_t.max_count()),
                                std::max(h->seg_ftail.max_count(), h->seg_btail.max_count()));
     h->max_segs_csr = std::max(h->seg_csr.max_count(), h->seg_csr_t.max_count());
@@ -632,8 +666,10 @@ void build_fused(hag *h) {
         if (j0 < k) phase_of_level[c + 1] = fb.rows_phase(h->ftail_ptr, 0, k - j0, int32_t(n + j0), h->fz_fwd.off_head, need);
         h->fz_fwd.off_tail = fb.add_ids(h->res_idx.data(), h->e_res);
         src = &h->res_idx;
+        const int64_t head = h->fz_fwd.n_items();
         if (n > 0) fb.rows_phase(h->res_ptr, 0, n, 0, h->fz_fwd.off_tail, need);
         fb.finish();
+        h->fz_fwd.head_items = h->fz_fwd.ok ? head : 0;
     }
     {   // backward over the HAG: the expanded deep nodes, levels bwd_cut..1, the graph nodes as sources
         const int32_t c = h->bwd_cut;
@@ -653,8 +689,10 @@ void build_fused(hag *h) {
         for (int32_t l = c; l >= 1; --l)
             phase_of_level[l] = fb.rows_phase(h->t_ptr, int64_t(n) + h->level_ptr[l - 1], h->level_ptr[l] - h->level_ptr[l - 1],
                                               int32_t(n + h->level_ptr[l - 1]), h->fz_bwd.off_tail + h->t_ptr[size_t(n) + h->level_ptr[l - 1]], need);
+        const int64_t head = h->fz_bwd.n_items();
         if (n > 0) fb.rows_phase(h->t_ptr, 0, n, 0, h->fz_bwd.off_tail, need);
         fb.finish();
+        h->fz_bwd.head_items = h->fz_bwd.ok ? head : 0;
     }
     {   // the input graph and its transpose: nothing to wait for but the chunks of long rows (k = 0: their ids start at n)
         auto none = [](int64_t, int64_t) { return -1; };
@@ -988,6 +1026,16 @@ extern "C" hag_status hag_export_pass(const hag_t *h, int32_t pass, hag_pass_vie
     out->rows = t.items.data();
     out->phase_size = t.phase_size.data();
     out->ids = t.ids.data();
+    return HAG_OK;
+}
+
+extern "C" hag_status hag_export_row_order(const hag_t *h, int32_t list, int32_t *first_row, int64_t *count, const int32_t **order) {
+    if (!h || !first_row || !count || !order) return HAG_ERR_NULL;
+    if (list < 0 || list > 5) return HAG_ERR_ARG;
+    const seg_set *sets[6] = {&h->seg_res, &h->seg_t, &h->seg_csr, &h->seg_csr_t, &h->seg_ftail, &h->seg_btail};
+    *first_row = sets[list]->order_first_row;
+    *count = int64_t(sets[list]->order.size());
+    *order = sets[list]->order.empty() ? nullptr : sets[list]->order.data();
     return HAG_OK;
 }
 

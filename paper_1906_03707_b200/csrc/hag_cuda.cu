@@ -46,6 +46,10 @@ void free_device(hag *h) {
     hag_device_arrays &d = h->d;
     for (cudaEvent_t ev : h->events) cudaEventDestroy(ev);
     h->events.clear();
+    for (seg_set *set : {&h->seg_res, &h->seg_t, &h->seg_csr, &h->seg_csr_t, &h->seg_ftail, &h->seg_btail}) {
+        if (set->d_order) cudaFree(set->d_order);
+        set->d_order = nullptr;
+    }
     for (seg_set *set : {&h->seg_res, &h->seg_t, &h->seg_csr, &h->seg_csr_t, &h->seg_ftail, &h->seg_btail})
     for (seg_table *t = set->g; t != set->g + kSegGrans; ++t) {
         if (t->d_segs) cudaFree(t->d_segs);
@@ -126,11 +130,31 @@ auto resident_kernel() {
     else return hagk::gather_sum_persistent_kernel<T, LPR, U, SS, MINB, SELF>;
 }
 
+template <typename T, int LPR, int U, bool SS, int MINB, bool SEGS, bool SELF>
+auto sub_kernel() {
+    if constexpr (SEGS) return hagk::gather_sum_sub_long_kernel<T, LPR, U, SS, MINB, SELF>;
+    else return hagk::gather_sum_sub_kernel<T, LPR, U, SS, MINB, SELF>;
+}
+
+// A launch that cannot give every resident warp a group of rows is bound by the latency of one row, which is shorter
+// with the whole warp on it.
+constexpr int64_t kSubMinWarps = 4096;
+inline bool use_sub_rows(int lpr, int64_t rows) { return lpr < 32 && rows >= kSubMinWarps * (32 / lpr); }
+
 template <typename T, int LPR, bool SS, bool SEGS, bool SELF>
 cudaError_t launch_gather_shape(const hagk::GatherArgs &ga, const hagk::SegArgs &sg, int sm_count, cudaStream_t s) {
     const hagk::KernelArgs<SEGS> a = pack_args<SEGS>(ga, sg);
     const int64_t items = int64_t(ga.row_count) + (SEGS ? sg.seg_count : 0);
     const unsigned grid = unsigned((items + hagk::kWarps - 1) / hagk::kWarps);
+    if constexpr (LPR < 32) {
+        if (use_sub_rows(LPR, ga.row_count)) {
+            constexpr int G = 32 / LPR;
+            const int64_t sub_items = (int64_t(ga.row_count) + G - 1) / G + (SEGS ? sg.seg_count : 0);
+            const unsigned sub_grid = unsigned((sub_items + hagk::kWarps - 1) / hagk::kWarps);
+            if constexpr (sizeof(T) == 4) return launch_pdl(sub_kernel<T, LPR, 4, SS, SS ? 8 : 10, SEGS, SELF>(), sub_grid, a, s);
+            else return launch_pdl(sub_kernel<T, LPR, 2, SS, 8, SEGS, SELF>(), sub_grid, a, s);
+        }
+    }
     if constexpr (sizeof(T) == 4) {
         if (ga.resident) {
             if constexpr (LPR == 32) return launch_persistent(resident_kernel<T, LPR, 8, SS, 8, SEGS, SELF>(), a, items, sm_count, s);
@@ -159,7 +183,12 @@ template <typename T>
 cudaError_t launch_gather(const hag *h, hagk::GatherArgs a, const seg_set &set, float *partial, int64_t edges,
                           int n_chunks, cudaStream_t s) {
     if (a.row_count <= 0) return cudaSuccess;
-    const int gran = seg_gran_for_rows(a.row_count);
+    a.resident = (a.row_count >= kManyRows || edges >= kManyEdges) ? 1 : 0;
+    const int lpr = lanes_per_row(n_chunks);
+    const bool sub = use_sub_rows(lpr, a.row_count);
+    // a lane group walks its row alone: nothing longer than 256 entries stays whole there
+    const int gran = sub ? std::min(seg_gran_for_rows(a.row_count), 1) : seg_gran_for_rows(a.row_count);
+    a.order = (sub && set.d_order) ? set.d_order - set.order_first_row : nullptr;
     const seg_table &table = set.g[gran];
     hagk::SegArgs sg{};
     sg.long_row = kSegLongRow[gran];
@@ -182,10 +211,8 @@ cudaError_t launch_gather(const hag *h, hagk::GatherArgs a, const seg_set &set, 
         sg.seg_first = int32_t(lo);
         sg.seg_count = int32_t(hi - lo);
     }
-    a.resident = (a.row_count >= kManyRows || edges >= kManyEdges) ? 1 : 0;
     hag *hm = const_cast<hag *>(h);
     a.sched = h->d.sched + 2 * (hm->sched_seq++ % kSchedSlots);
-    const int lpr = lanes_per_row(n_chunks);
     const bool ss = a.src_scale != nullptr;
     switch (lpr) {
         case 4: return ss ? launch_gather_lpr<T, 4, true>(a, sg, h->sm_count, s) : launch_gather_lpr<T, 4, false>(a, sg, h->sm_count, s);
@@ -222,7 +249,8 @@ cudaError_t launch_fused_shape(const hagk::FusedArgs &k, int sm_count, cudaStrea
 }
 
 template <typename T>
-cudaError_t launch_fused(const hag *h, const fused_table &t, hagk::GatherArgs a, float *ahat, int n_chunks, cudaStream_t s) {
+cudaError_t launch_fused(const hag *h, const fused_table &t, hagk::GatherArgs a, float *ahat, int n_chunks, cudaStream_t s,
+                         bool head_only = false) {
     hagk::FusedArgs k{};
     a.idx = t.d_ids;
     a.row_ptr = nullptr;
@@ -232,7 +260,9 @@ cudaError_t launch_fused(const hag *h, const fused_table &t, hagk::GatherArgs a,
     a.n_prim = h->n;           // ids from n on: aggregation nodes, then the chunk rows of this pass
     k.a = a;
     k.items = reinterpret_cast<const int4 *>(t.d_items);
-    k.n_items = int32_t(t.n_items());
+    // head_only: the list ends where the graph-node rows begin; last_phase still names their phase, which is then never
+    // reached, so every phase that runs is counted and can be waited for
+    k.n_items = int32_t(head_only ? t.head_items : t.n_items());
     k.last_phase = t.last_phase;
     k.phase_size = t.d_phase_size;
     hag *hm = const_cast<hag *>(h);
@@ -241,7 +271,7 @@ cudaError_t launch_fused(const hag *h, const fused_table &t, hagk::GatherArgs a,
     k.err_host = h->d.err_dev;
     k.spin_limit = h->spin_limit;
     const int lpr = lanes_per_row(n_chunks);
-    const bool ss = a.src_scale != nullptr, self = (a.out_is_f32 & 2) != 0;
+    const bool ss = a.src_scale != nullptr, self = !head_only && (a.out_is_f32 & 2) != 0;
 #define HAG_FUSED_CASE(L)                                                                                          \
     case L:                                                                                                        \
         if (ss) return self ? launch_fused_shape<T, L, true, true>(k, h->sm_count, s) : launch_fused_shape<T, L, true, false>(k, h->sm_count, s); \
@@ -375,8 +405,14 @@ hag_status fwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
     }
     if (use_hag) {
         if (h->num_agg > 0) {
-            hag_status st = enqueue_fwd_agg<T>(h, D, x, static_cast<float *>(ws), partial, s, rec);
-            if (st != HAG_OK) return st;
+            if (h->schedule == 2 && fz.ok && fz.head_items > 0) {     // the aggregation nodes, all levels, in one launch
+                if (rec) rec->begin(3, h->num_agg, h->e_hat - h->e_res);
+                if (launch_fused<T>(h, fz, a, static_cast<float *>(ws), n_chunks, s, true) != cudaSuccess) return HAG_ERR_CUDA;
+                if (rec) rec->end();
+            } else {
+                hag_status st = enqueue_fwd_agg<T>(h, D, x, static_cast<float *>(ws), partial, s, rec);
+                if (st != HAG_OK) return st;
+            }
             a.sec = static_cast<const float *>(ws);
             a.n_prim = h->n;
         }
@@ -420,7 +456,16 @@ hag_status bwd_impl(const hag *h, bool use_hag, hag_reduce reduce, int32_t D, co
         if (rec) rec->end();
         return HAG_OK;
     }
-    if (use_hag && h->num_agg > 0) {
+    if (use_hag && h->num_agg > 0 && h->schedule == 2 && fz.ok && fz.head_items > 0) {
+        // the aggregation nodes' gradients, the expanded ones and every level, in one launch
+        if (rec) rec->begin(3, h->num_agg, h->e_hat - h->t_ptr[h->n]);
+        if (launch_fused<T>(h, fz, a, static_cast<float *>(ws), n_chunks, s, true) != cudaSuccess) return HAG_ERR_CUDA;
+        if (rec) rec->end();
+        a.row_ptr = d.t_ptr;
+        a.idx = d.t_idx;
+        a.sec = static_cast<const float *>(ws);
+        a.n_prim = h->n;
+    } else if (use_hag && h->num_agg > 0) {
         const int32_t j0 = int32_t(h->level_ptr[h->bwd_cut]);
         if (j0 < h->num_agg) {
             hagk::GatherArgs t = a;              // all sources are graph-node outputs
@@ -573,6 +618,8 @@ extern "C" hag_status hag_to_device(hag_t *h, int device) {
         }
     }
     for (seg_set *set : {&h->seg_res, &h->seg_t, &h->seg_csr, &h->seg_csr_t, &h->seg_ftail, &h->seg_btail})
+        if (st == HAG_OK && !set->order.empty()) st = upload_i32(&set->d_order, set->order.data(), set->order.size());
+    for (seg_set *set : {&h->seg_res, &h->seg_t, &h->seg_csr, &h->seg_csr_t, &h->seg_ftail, &h->seg_btail})
     for (seg_table *t = set->g; t != set->g + kSegGrans; ++t) {
         if (st != HAG_OK || t->segs.empty()) continue;
         st = upload_i32(&t->d_segs, t->segs.data(), t->segs.size());
@@ -699,10 +746,10 @@ extern "C" hag_status hag_aggregate_host(hag_t *h, int backward, int use_hag, ha
 
 extern "C" int32_t hag_last_launch_count(const hag_t *h) { return h ? h->last_launches : 0; }
 
-extern "C" hag_status hag_set_schedule(hag_t *h, int32_t single_launch) {
+extern "C" hag_status hag_set_schedule(hag_t *h, int32_t schedule) {
     if (!h) return HAG_ERR_NULL;
-    if (single_launch != 0 && single_launch != 1) return HAG_ERR_ARG;
-    h->schedule = single_launch;
+    if (schedule < 0 || schedule > 2) return HAG_ERR_ARG;
+    h->schedule = schedule;
     return HAG_OK;
 }
 

@@ -26,8 +26,19 @@ constexpr int32_t kSegLongRow[kSegGrans] = {64, 256, 1024};   // rows with more 
 constexpr int32_t kSegLength[kSegGrans] = {32, 128, 512};     // ... into segments of this many entries
 inline int seg_gran_for_rows(int64_t rows) { return rows < 8192 ? 0 : (rows < 65536 ? 1 : 2); }
 
+// Rows of like length side by side, for the kernels that walk several rows per warp in lock step: within windows of
+// kOrderWindow rows (so that rows that share neighbours stay close in time) the rows are sorted by length, longest
+// first.  order[r - first_row] is the row that takes the place of row r; windows never cross a boundary between
+// launches (graph nodes | level 1 | level 2 ...), so every launch's range of rows maps onto itself.  Empty where the
+// rows as they are lose less than kOrderMinWaste of the lock-step rounds.
+constexpr int32_t kOrderWindow = 2048;
+constexpr double kOrderMinWaste = 1.08;
+
 struct seg_set {
     seg_table g[kSegGrans];
+    std::vector<int32_t> order;
+    int32_t order_first_row = 0;
+    int32_t *d_order = nullptr;
     int64_t max_count() const {
         int64_t m = 0;
         for (const seg_table &t : g) m = m > t.count() ? m : t.count();
@@ -58,6 +69,8 @@ struct fused_table {
                                      // `ids` into output row `row` (row < 0: padding; row >= n: an aggregation node or a chunk row)
     std::vector<int32_t> phase_size; // rows per phase, padding included
     std::vector<int32_t> ids;        // the pass's id list: pair inputs, expansion lists, row lists, chunk ids of the long rows
+    int64_t head_items = 0;          // rows of the list before the graph-node rows (and the chunk rows of their long rows): the
+                                     // aggregation nodes' part of the pass, which can be launched by itself
     int64_t off_head = 0;            // where the expansion lists (ftail / btail) start in ids
     int64_t off_tail = 0;            // where the row lists (residual rows / transposed HAG / input graph) start
     int64_t n_chunks = 0;            // chunk rows: fp32 partial rows needed behind the aggregation nodes' rows

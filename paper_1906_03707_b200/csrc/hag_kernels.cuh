@@ -59,6 +59,8 @@ struct GatherArgs {
     int32_t out_is_f32;
     int32_t D;
     int32_t resident;         // host-side choice of the launch form; the kernels ignore it
+    const int32_t *order;     // several-rows-per-warp kernels only: the row that takes the place of absolute row r
+                              // (rows of like length side by side), or null for the rows as they are
 };
 
 // Long rows (more than long_row entries) are not walked by one warp: they are cut into segments that
@@ -560,6 +562,143 @@ __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_kernel(const 
 template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS, bool SELF>
 __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_long_kernel(const __grid_constant__ KernelArgs<true> k) {
     gather_sum_body<T, LPR, UNROLL, SRC_SCALE, true, SELF>(k);
+}
+
+// Several rows per warp, for rows of 256 bytes or less (LPR < 32).  gather_row spreads ONE row over the warp's
+// 32 / LPR lane groups and adds the groups' sums up at the end; with the short rows of clustered graphs (half of them
+// 8 entries or fewer once a HAG has taken their common pairs away) most of the ~150 instructions around the loads
+// are spent per row, not per entry, and the kernel is bound by instruction issue.  Here every lane group takes a row
+// of its own: G = 32 / LPR rows share each instruction, no sums cross lanes, and a group keeps U loads of its row in
+// flight.  The groups of a warp run in lock step for as long as the longest of their rows lasts.
+// Order of additions of a row: per batch of LPR ids the tree sums of U rows at a time into `part`, batches into the
+// accumulator (two-level, as in gather_row).
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, bool HAS_SEGS, bool SELF>
+__device__ __forceinline__ void gather_sum_sub_body(const KernelArgs<HAS_SEGS> &k) {
+    static_assert(LPR < 32, "one row per warp is gather_row's job");
+    const GatherArgs &a = k.a;
+    pdl_launch_dependents();
+    constexpr int E = Chunk<T>::kElems;
+    constexpr int G = 32 / LPR;
+    constexpr int U = (UNROLL < LPR) ? UNROLL : LPR;
+    constexpr unsigned FULL = 0xffffffffu;
+    const int lane = threadIdx.x & 31;
+    int item = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if constexpr (HAS_SEGS) {
+        if (item < k.sg.seg_count) {
+            pdl_wait();
+            gather_segment_call<T, LPR, UNROLL, SRC_SCALE, SELF>(a, k.sg, item, lane);
+            return;
+        }
+        item -= k.sg.seg_count;
+    }
+    const int slice = lane / LPR, gl = lane % LPR;
+    const int32_t r_local = item * G + slice;
+    if (item * G >= a.row_count) return;
+    bool have = r_local < a.row_count;
+    int32_t row = a.row_begin + (have ? r_local : 0);
+    if (a.order) row = __ldg(a.order + row);
+    int32_t b = 0, e = 0;
+    if (have) {
+        b = __ldg(a.row_ptr + row);
+        e = __ldg(a.row_ptr + row + 1);
+    }
+    if constexpr (HAS_SEGS) {
+        if (e - b > k.sg.long_row) { have = false; e = b; }      // a long row: its segments are items of their own
+    }
+    int32_t mine = (b + gl < e) ? __ldg(a.idx + b + gl) : -1;
+    float mine_s = 1.0f;
+    if constexpr (SRC_SCALE) mine_s = (mine >= 0 && mine < a.n_prim) ? __ldg(a.src_scale + mine) : 1.0f;
+    const float dscale = (have && a.dst_scale && row < a.n_prim) ? __ldg(a.dst_scale + row) : 1.0f;
+    const int32_t len = e - b;
+    const int32_t max_len = __reduce_max_sync(FULL, len);
+    pdl_wait();        // structure arrays are static; features may come from the previous kernel
+    const int n_chunks = a.D / E;
+    const bool live = gl < n_chunks;
+    const Tables<T> tab(a.prim, a.sec, a.n_prim, a.D, live ? gl : 0);
+    float acc[E];
+#pragma unroll
+    for (int j = 0; j < E; ++j) acc[j] = 0.0f;
+    for (int32_t off = 0; off < max_len; off += LPR) {
+        const int32_t cur = mine;
+        const float cur_s = mine_s;
+        const int32_t nb = b + off + LPR + gl;
+        mine = (nb < e) ? __ldg(a.idx + nb) : -1;                 // next batch of ids, in flight early
+        if constexpr (SRC_SCALE) mine_s = (mine >= 0 && mine < a.n_prim) ? __ldg(a.src_scale + mine) : 1.0f;
+        const int32_t cnt = len - off;                            // entries left in this group's row (<= 0: none)
+        const int32_t max_cnt = max_len - off;
+        float part[E];
+#pragma unroll
+        for (int j = 0; j < E; ++j) part[j] = 0.0f;
+#pragma unroll
+        for (int kk = 0; kk < LPR; kk += U) {
+            if (kk < max_cnt) {
+                float v[U][E];
+                if (__all_sync(FULL, kk + U <= cnt)) {            // every group has U entries left: no checks, no fill
+#pragma unroll
+                    for (int u = 0; u < U; ++u) tab.load(__shfl_sync(FULL, cur, kk + u, LPR), v[u]);
+                } else {
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        const int32_t id = __shfl_sync(FULL, cur, kk + u, LPR);
+                        if (id >= 0 && live) {
+                            tab.load(id, v[u]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < E; ++j) v[u][j] = 0.0f;
+                        }
+                    }
+                }
+                if constexpr (SRC_SCALE && E == 4) {
+                    // part += factor * row as packed fused multiply-adds, as in gather_row
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        const float sc = __shfl_sync(FULL, cur_s, kk + u, LPR);
+                        const float2 s2 = make_float2(sc, sc);
+                        const float2 lo = __ffma2_rn(make_float2(v[u][0], v[u][1]), s2, make_float2(part[0], part[1]));
+                        const float2 hi = __ffma2_rn(make_float2(v[u][2], v[u][3]), s2, make_float2(part[2], part[3]));
+                        part[0] = lo.x; part[1] = lo.y; part[2] = hi.x; part[3] = hi.y;
+                    }
+                } else {
+                    if constexpr (SRC_SCALE) {
+#pragma unroll
+                        for (int u = 0; u < U; ++u) {
+                            const float sc = __shfl_sync(FULL, cur_s, kk + u, LPR);
+#pragma unroll
+                            for (int j = 0; j < E; ++j) v[u][j] *= sc;
+                        }
+                    }
+#pragma unroll
+                    for (int w = U / 2; w >= 1; w /= 2)
+#pragma unroll
+                        for (int u = 0; u < w; ++u) add_rows<E>(v[u], v[u + w]);
+                    add_rows<E>(part, v[0]);
+                }
+            }
+        }
+        add_rows<E>(acc, part);
+    }
+    if (have && live) {
+        if constexpr (SELF) {         // GCN: the row's own term
+            float self[E];
+            tab.load(row, self);
+            float sc = 1.0f;
+            if constexpr (SRC_SCALE) sc = __ldg(a.src_scale + row);
+#pragma unroll
+            for (int j = 0; j < E; ++j) acc[j] = fmaf(self[j], sc, acc[j]);
+        }
+#pragma unroll
+        for (int j = 0; j < E; ++j) acc[j] *= dscale;
+        store_chunk<T>(a.out, a.out_is_f32 & 1, a.D, row - a.out_row_offset, gl, acc);
+    }
+}
+
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS, bool SELF>
+__global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_sub_kernel(const KernelArgs<false> k) {
+    gather_sum_sub_body<T, LPR, UNROLL, SRC_SCALE, false, SELF>(k);
+}
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS, bool SELF>
+__global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_sub_long_kernel(const __grid_constant__ KernelArgs<true> k) {
+    gather_sum_sub_body<T, LPR, UNROLL, SRC_SCALE, true, SELF>(k);
 }
 
 // The same, with resident warps that take items four at a time from a shared

@@ -60,8 +60,8 @@ struct PairMaxArgs {
 // Launch shapes from a sweep on B200 (loads or entries in flight per lane, resident CTAs per SM):
 // more resident warps beat more loads per warp, as for the sum kernels.
 //   fp32: forward 4 loads x 10 CTAs, backward 2 entries x 10 CTAs; bf16: forward 4 x 12 (raw word groups: 4 registers
-//   per load in flight), backward 1 x 8.
-#define HAG_MAX_SHAPES 4, 10, 2, 10, 4, 12, 1, 8
+//   per load in flight), backward 4 x 8 (a maximum and a gradient word group per entry).
+#define HAG_MAX_SHAPES 4, 10, 2, 10, 4, 12, 4, 8
 template <typename T> struct MaxShape;
 template <int FL, int FB, int BE, int BB, int HFL, int HFB, int HBE, int HBB> struct MaxShapeTable {
     static constexpr int f32[4] = {FL, FB, BE, BB};
@@ -70,11 +70,14 @@ template <int FL, int FB, int BE, int BB, int HFL, int HFB, int HBE, int HBB> st
 using MaxShapes = MaxShapeTable<HAG_MAX_SHAPES>;
 template <> struct MaxShape<float> {
     static constexpr int kFwdLoads = MaxShapes::f32[0], kFwdBlocks = MaxShapes::f32[1];
-    static constexpr int kBwdEntries = MaxShapes::f32[2], kBwdBlocks = MaxShapes::f32[3];
+    static constexpr int kBwdEntries = MaxShapes::f32[2];
+    // 512-byte rows and wider: the unchecked loop body needs the registers of one CTA fewer, or it spills
+    static constexpr int bwd_blocks(int lpr) { return lpr == 32 ? MaxShapes::f32[3] - 1 : MaxShapes::f32[3]; }
 };
 template <> struct MaxShape<__nv_bfloat16> {
     static constexpr int kFwdLoads = MaxShapes::bf16[0], kFwdBlocks = MaxShapes::bf16[1];
-    static constexpr int kBwdEntries = MaxShapes::bf16[2], kBwdBlocks = MaxShapes::bf16[3];
+    static constexpr int kBwdEntries = MaxShapes::bf16[2];
+    static constexpr int bwd_blocks(int) { return MaxShapes::bf16[3]; }
 };
 
 // Packed maximum of two bf16 pairs (one instruction for two values; exact, as every maximum is).
@@ -246,13 +249,27 @@ __global__ void __launch_bounds__(kThreads) pair_max_kernel(const PairMaxArgs p)
     }
 }
 
+// acc[0..8) += the gradient words g where the destination's maximum words v equal this row's value words (bf16 pairs
+// compared two at a time: ordered equality, +0 == -0, NaN equal to nothing, as for floats; the kept gradient pairs are
+// widened by a shift or a mask and added as packed fp32 pairs).
+__device__ __forceinline__ void add_where_equal_bf16x8(float *acc, const uint4 &v, const uint4 &g, const uint4 &own) {
+    const uint32_t vw[4] = {v.x, v.y, v.z, v.w}, gw[4] = {g.x, g.y, g.z, g.w}, ow[4] = {own.x, own.y, own.z, own.w};
+    uint4 kept;
+    uint32_t *kw = &kept.x;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        kw[i] = gw[i] & __heq2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&vw[i]), *reinterpret_cast<const __nv_bfloat162 *>(&ow[i]));
+    hagk::add_bf16x8<false>(acc, kept, 1.0f);
+}
+
 // grad_s[k] = sum over the destinations t of row s with max_t[k] == value_s[k] of grad_t[k].
 template <typename T, int LPR>
-__global__ void __launch_bounds__(kThreads, MaxShape<T>::kBwdBlocks) gather_maxgrad_kernel(const MaxArgs a) {
+__global__ void __launch_bounds__(kThreads, MaxShape<T>::bwd_blocks(LPR)) gather_maxgrad_kernel(const MaxArgs a) {
     hagk::pdl_launch_dependents();
     constexpr int E = Chunk<T>::kElems;
     constexpr int G = 32 / LPR;
     constexpr int U = MaxShape<T>::kBwdEntries < LPR ? MaxShape<T>::kBwdEntries : LPR;
+    constexpr unsigned FULL = 0xffffffffu;
     const int lane = threadIdx.x & 31;
     const int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
     if (r_local >= a.row_count) return;
@@ -267,50 +284,127 @@ __global__ void __launch_bounds__(kThreads, MaxShape<T>::kBwdBlocks) gather_maxg
         const bool live = chunk < n_chunks;
         const Tables<T> vals(a.val_prim, a.val_sec, a.n_prim, a.D, live ? chunk : 0);
         const Tables<T> grads(a.grad_prim, a.grad_sec, a.n_prim, a.D, live ? chunk : 0);
-        float own[E], acc[E];
-        {
-            const Tables<T> self(a.own_prim, a.own_sec, a.n_prim, a.D, live ? chunk : 0);
-            self.load(row, own);
-        }
+        const Tables<T> self(a.own_prim, a.own_sec, a.n_prim, a.D, live ? chunk : 0);
+        float acc[E];
 #pragma unroll
         for (int j = 0; j < E; ++j) acc[j] = 0.0f;
         int32_t mine = (c0 == 0) ? first : ((b + lane < e) ? __ldg(a.idx + b + lane) : -1);
-        for (int32_t base = b; base < e; base += 32) {
-            const int32_t cur = mine;
-            const int32_t nb = base + 32;
-            mine = (nb + lane < e) ? __ldg(a.idx + nb + lane) : -1;
-            const int cnt = min(32, e - base);
-            float part[E];            // two-level sum: one partial per batch of 32 ids
+        if constexpr (E == 8) {
+            // bf16 storage.  Maxima are bf16 values wherever they are kept, so the comparison runs on bf16 pairs (this
+            // row's value packed once); the rows of graph-node destinations stay raw words from the load to the masked
+            // add, U entries (a maximum and a gradient word group each) in flight.  The ids of a row ascend: the
+            // graph-node destinations are the first n_p entries of a batch, the aggregation nodes (fp32 maxima and fp32
+            // gradients) the rest, a loop each.
+            uint4 own;
+            if (row < a.n_prim) {
+                own = hagk::ld_u4(self.prim + size_t(uint32_t(row)) * self.prim_row_bytes);
+            } else {
+                const char *p = self.sec + size_t(uint32_t(row)) * self.sec_row_bytes;
+                const float4 q0 = hagk::ld_f4(p), q1 = hagk::ld_f4(p + 16);
+                own = make_uint4(pack_bf16x2(q0.x, q0.y), pack_bf16x2(q0.z, q0.w), pack_bf16x2(q1.x, q1.y), pack_bf16x2(q1.z, q1.w));
+            }
+            for (int32_t base = b; base < e; base += 32) {
+                const int32_t cur = mine;
+                const int32_t nb = base + 32;
+                mine = (nb + lane < e) ? __ldg(a.idx + nb + lane) : -1;
+                const int cnt = min(32, e - base);
+                const int n_p = __popc(__ballot_sync(FULL, cur >= 0 && cur < a.n_prim));
 #pragma unroll
-            for (int j = 0; j < E; ++j) part[j] = 0.0f;
+                for (int k = 0; k < LPR; k += U) {
+                    if (k * G < n_p) {
+                        uint4 rv[U], rg[U];
+                        if ((k + U) * G <= n_p) {       // a full group: no checks (lanes beyond the row width read chunk 0, never stored)
 #pragma unroll
-            for (int k = 0; k < LPR; k += U) {
-                if (k * G < cnt) {
-                    float tv[U][E], tg[U][E];
-#pragma unroll
-                    for (int u = 0; u < U; ++u) {
-                        const int32_t id = __shfl_sync(0xffffffffu, cur, (k + u) * G + slice);
-                        if (id >= 0 && live) {
-                            vals.load(id, tv[u]);
-                            grads.load(id, tg[u]);
+                            for (int u = 0; u < U; ++u) {
+                                const size_t off = size_t(uint32_t(__shfl_sync(FULL, cur, (k + u) * G + slice))) * vals.prim_row_bytes;
+                                rv[u] = hagk::ld_u4(vals.prim + off);
+                                rg[u] = hagk::ld_u4(grads.prim + off);
+                            }
                         } else {
 #pragma unroll
-                            for (int j = 0; j < E; ++j) { tv[u][j] = own[j]; tg[u][j] = 0.0f; }
+                            for (int u = 0; u < U; ++u) {
+                                const int32_t id = __shfl_sync(FULL, cur, (k + u) * G + slice);
+                                if ((k + u) * G + slice < n_p && live) {
+                                    const size_t off = size_t(uint32_t(id)) * vals.prim_row_bytes;
+                                    rv[u] = hagk::ld_u4(vals.prim + off);
+                                    rg[u] = hagk::ld_u4(grads.prim + off);
+                                } else {
+                                    rv[u] = rg[u] = make_uint4(0u, 0u, 0u, 0u);      // a zero gradient adds nothing
+                                }
+                            }
+                        }
+#pragma unroll
+                        for (int u = 0; u < U; ++u) add_where_equal_bf16x8(acc, rv[u], rg[u], own);
+                    }
+                }
+                for (int j0 = n_p; j0 < cnt; j0 += G) {
+                    const int j = j0 + slice;
+                    const int32_t id = __shfl_sync(FULL, cur, j < cnt ? j : 0);
+                    if (j < cnt && live) {
+                        const size_t off = size_t(uint32_t(id)) * vals.sec_row_bytes;
+                        const float4 v0 = hagk::ld_f4(vals.sec + off), v1 = hagk::ld_f4(vals.sec + off + 16);
+                        const float4 g0 = hagk::ld_f4(grads.sec + off), g1 = hagk::ld_f4(grads.sec + off + 16);
+                        const uint32_t ow[4] = {own.x, own.y, own.z, own.w};
+                        const uint32_t vw[4] = {pack_bf16x2(v0.x, v0.y), pack_bf16x2(v0.z, v0.w), pack_bf16x2(v1.x, v1.y), pack_bf16x2(v1.z, v1.w)};
+                        const float gf[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint32_t m = __heq2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&vw[i]), *reinterpret_cast<const __nv_bfloat162 *>(&ow[i]));
+                            acc[2 * i] += (m & 0xffffu) ? gf[2 * i] : 0.0f;
+                            acc[2 * i + 1] += (m >> 16) ? gf[2 * i + 1] : 0.0f;
                         }
                     }
-#pragma unroll
-                    for (int u = 0; u < U; ++u)
-#pragma unroll
-                        for (int j = 0; j < E; ++j) part[j] += (tv[u][j] == own[j]) ? tg[u][j] : 0.0f;
                 }
             }
+        } else {
+            float own[E];
+            self.load(row, own);
+            for (int32_t base = b; base < e; base += 32) {
+                const int32_t cur = mine;
+                const int32_t nb = base + 32;
+                mine = (nb + lane < e) ? __ldg(a.idx + nb + lane) : -1;
+                const int cnt = min(32, e - base);
+                float part[E];            // two-level sum: one partial per batch of 32 ids
 #pragma unroll
-            for (int j = 0; j < E; ++j) acc[j] += part[j];
+                for (int j = 0; j < E; ++j) part[j] = 0.0f;
+#pragma unroll
+                for (int k = 0; k < LPR; k += U) {
+                    if (k * G < cnt) {
+                        float tv[U][E], tg[U][E];
+                        if ((k + U) * G <= cnt) {       // a full group: no checks, no fill
+#pragma unroll
+                            for (int u = 0; u < U; ++u) {
+                                const int32_t id = __shfl_sync(FULL, cur, (k + u) * G + slice);
+                                vals.load(id, tv[u]);
+                                grads.load(id, tg[u]);
+                            }
+                        } else {
+#pragma unroll
+                            for (int u = 0; u < U; ++u) {
+                                const int32_t id = __shfl_sync(FULL, cur, (k + u) * G + slice);
+                                if (id >= 0 && live) {
+                                    vals.load(id, tv[u]);
+                                    grads.load(id, tg[u]);
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < E; ++j) { tv[u][j] = own[j]; tg[u][j] = 0.0f; }
+                                }
+                            }
+                        }
+#pragma unroll
+                        for (int u = 0; u < U; ++u)
+#pragma unroll
+                            for (int j = 0; j < E; ++j) part[j] += (tv[u][j] == own[j]) ? tg[u][j] : 0.0f;
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < E; ++j) acc[j] += part[j];
+            }
         }
 #pragma unroll
         for (int off = LPR; off < 32; off <<= 1)
 #pragma unroll
-            for (int j = 0; j < E; ++j) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], off);
+            for (int j = 0; j < E; ++j) acc[j] += __shfl_xor_sync(FULL, acc[j], off);
         if (live && slice == 0) hagk::store_chunk<T>(a.out, a.out_is_f32, a.D, row - a.out_row_offset, chunk, acc);
     }
 }

@@ -455,3 +455,54 @@ def test_import_of_a_recorded_trace_reproduces_the_build_and_rejects_what_does_n
     assert imp(trace, other.row_ptr, other.col_idx) == 2      # the trace of another graph does not replay
     assert lib.hag_import(g.n, g.row_ptr.ctypes.data, g.col_idx.ctypes.data, 3, None, ctypes.byref(out)) == 1
     assert lib.hag_import(g.n, g.row_ptr.ctypes.data, g.col_idx.ctypes.data, -1, None, ctypes.byref(out)) == 2
+
+
+def test_row_order_is_a_windowed_sort_by_length_that_keeps_every_launch_range():
+    """hag_export_row_order: a permutation per list, sorted by length inside windows of 2048 rows that never cross
+    from the graph nodes into a level or from a level into the next; absent where neighbouring rows already match."""
+    w = synth.workload(6, scale=0.08)
+    g = w.graph
+    h = hb.Hag.build(g.row_ptr, g.col_idx, w.capacity)
+    a = h.arrays()
+    n, k = g.n, int(a["num_agg"])
+    assert int(a["num_levels"]) >= 3
+    level_ptr = np.asarray(a["level_ptr"], dtype=np.int64)
+    t_bounds = np.concatenate([[0, n], n + level_ptr[1:]])
+    csr_t_ptr = np.zeros(n + 1, np.int64)
+    np.add.at(csr_t_ptr, g.col_idx.astype(np.int64) + 1, 1)
+    csr_t_ptr = np.cumsum(csr_t_ptr)
+    lists = {0: (a["res_ptr"], 0, [0, n]), 1: (a["t_ptr"], 0, t_bounds), 2: (g.row_ptr, 0, [0, n]), 3: (csr_t_ptr, 0, [0, n])}
+    for cut_f, cut_b in ((1, 2), (0, 0)):
+        h.set_cuts(cut_f, cut_b)
+        p = h.pass_rows(0)      # (the expansion lists themselves are checked elsewhere; here their row ranges)
+        for which, first_expected in ((4, n + int(level_ptr[cut_f])), (5, n + int(level_ptr[cut_b]))):
+            first, order = h.row_order(which)
+            assert first == first_expected
+            if order.size:
+                assert np.array_equal(np.sort(order), first + np.arange(order.size))
+    seen_sorted = 0
+    for which, (ptr, first_expected, bounds) in lists.items():
+        first, order = h.row_order(which)
+        assert first == first_expected
+        lens = np.diff(np.asarray(ptr, dtype=np.int64))
+        if order.size == 0:
+            # only where pairs of neighbouring rows lose less than 8 % of the rounds of four loads
+            r = (lens + 3) // 4
+            if r.size % 2:
+                r = np.concatenate([r, [0]])
+            assert 2 * r.reshape(-1, 2).max(1).sum() < 1.08 * max(r.sum(), 1)
+            continue
+        seen_sorted += 1
+        assert order.size == lens.size
+        assert np.array_equal(np.sort(order), np.arange(order.size))          # a permutation
+        for b0, b1 in zip(bounds[:-1], bounds[1:]):
+            for w0 in range(int(b0), int(b1), 2048):
+                w1 = min(w0 + 2048, int(b1))
+                win = order[w0:w1]
+                assert win.min() >= w0 and win.max() < w1                      # the window maps onto itself
+                assert np.all(np.diff(lens[win]) <= 0)                         # longest first
+                same = np.diff(lens[win]) == 0
+                assert np.all(np.diff(win)[same] > 0)                          # equal lengths keep their order
+    assert seen_sorted >= 2
+    lib = hb.load_library()
+    assert lib.hag_export_row_order(h._h, 6, ctypes.byref(ctypes.c_int32()), ctypes.byref(ctypes.c_int64()), ctypes.byref(ctypes.c_void_p())) == 2

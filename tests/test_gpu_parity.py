@@ -50,7 +50,8 @@ def _check_all_paths(g, hag, x, gr, reduce, dtype, rows=None):
     a, t = O.direct_forward(g.row_ptr, g.col_idx, x.astype(np.float64), reduce, rows=rows)
     gx, tg = O.direct_backward(g.row_ptr, g.col_idx, gr.astype(np.float64), reduce, rows=rows)
     sel = slice(None) if rows is None else rows
-    for single_launch in (True, False):          # one launch per pass, then a launch per level (the default)
+    # the aggregation nodes in one launch and the graph nodes in a second; one launch per pass; a launch per level (default)
+    for single_launch in (2, 1, 0):
         hag.set_schedule(single_launch)
         for name, fwd, bwd in (("hag", hag.aggregate_fwd, hag.aggregate_bwd), ("csr", hag.csr_fwd, hag.csr_bwd)):
             out = _host(fwd(xd, reduce))[sel]
@@ -79,7 +80,7 @@ def _case(name):
     return _built[name]
 
 
-@pytest.mark.parametrize("name", list(CASES))
+@pytest.mark.parametrize("name", [c for c in CASES if c != "clique-union-70k"])
 @pytest.mark.parametrize("reduce", ["sum", "mean", "gcn"])
 def test_workload_shapes_match_oracle(name, reduce):
     w, h = _case(name)
@@ -88,6 +89,35 @@ def test_workload_shapes_match_oracle(name, reduce):
     gr = synth.upstream_grad(w.seed, g.n, w.d, w.feat_dist, w.dtype)
     assert h.info()["num_agg"] > 0
     _check_all_paths(g, h, x, gr, reduce, w.dtype)
+
+
+CASES["clique-union-70k"] = lambda: synth.workload(6, scale=0.7)
+
+
+@pytest.mark.parametrize("dtype,d,reduce", [("f32", 16, "sum"), ("f32", 32, "mean"), ("f32", 64, "gcn"), ("f32", 40, "mean"),
+                                             ("f32", 64, "sum"), ("bf16", 64, "sum"), ("bf16", 32, "mean"), ("bf16", 128, "gcn"),
+                                             ("bf16", 24, "sum")])
+def test_several_rows_per_warp_kernels_match_oracle(dtype, d, reduce):
+    """Rows of 256 bytes or less in launches large enough to fill the machine go to the kernels in which every group of
+    lanes walks a row of its own, in the windowed by-length order: 70 000 rows of very mixed lengths, hub rows cut
+    into segments among them, every lane-group width, dead lanes (d = 40, 24), factors per source (mean backward) and
+    the own-row term (gcn)."""
+    w, h = _case("clique-union-70k")
+    g = w.graph
+    assert g.n >= 8 * 4096 and int(np.diff(g.row_ptr).max()) > 256
+    assert h.row_order(0)[1].size == g.n and h.row_order(2)[1].size == g.n        # both passes take the sorted order
+    x = synth.features(91, g.n, d, "normal", dtype)
+    gr = synth.upstream_grad(91, g.n, d, "normal", dtype)
+    _check_all_paths(g, h, x, gr, reduce, dtype)
+    if reduce == "sum" and dtype == "f32":        # and exactly, on integers (fp32 holds every partial sum)
+        xi = synth.features(92, g.n, d, "int", dtype)
+        a, _ = O.direct_forward(g.row_ptr, g.col_idx, xi.astype(np.float64), "sum")
+        b, _ = O.direct_backward(g.row_ptr, g.col_idx, xi.astype(np.float64), "sum")
+        xd = _dev(xi, dtype)
+        h.set_schedule(False)
+        for fwd, bwd in ((h.aggregate_fwd, h.aggregate_bwd), (h.csr_fwd, h.csr_bwd)):
+            assert np.array_equal(_host(fwd(xd, "sum")).astype(np.float64), a)
+            assert np.array_equal(_host(bwd(xd, "sum")).astype(np.float64), b)
 
 
 @pytest.mark.parametrize("name", ["cfg1", "cfg2-small", "cfg4-small", "cfg5-small"])
@@ -124,7 +154,7 @@ def test_integer_features_are_bit_exact_for_sum(name):
         xd = _dev(x, dtype)
         if dtype == "bf16" and max(np.abs(a).max(), np.abs(gx).max()) > 256:
             continue  # bf16 output cannot hold the integers exactly
-        for single_launch in (True, False):
+        for single_launch in (2, 1, 0):
             h.set_schedule(single_launch)
             for fwd, bwd in ((h.aggregate_fwd, h.aggregate_bwd), (h.csr_fwd, h.csr_bwd)):
                 assert np.array_equal(_host(fwd(xd, "sum")), a)
@@ -256,7 +286,7 @@ def test_random_graphs_every_path_exact_on_integers(seed):
         h = hb.Hag.build(g.row_ptr, g.col_idx, cap, min_redundancy=min_r)
         L = h.info()["num_levels"]
         h.set_cuts(int(rng.integers(0, L + 1)), int(rng.integers(0, L + 1))).to_device(0)
-    for single_launch in (True, False):
+    for single_launch in (2, 1, 0):
         h.set_schedule(single_launch)
         assert np.array_equal(_host(h.aggregate_fwd(xd, "sum")), a)
         assert np.array_equal(_host(h.csr_fwd(xd, "sum")), a)
@@ -280,7 +310,7 @@ def test_every_cut_gives_the_same_values_on_the_device():
     assert L >= 4
     for cut in range(L + 1):
         h = hb.Hag.build(g.row_ptr, g.col_idx, w.capacity).set_cuts(cut, L - cut).to_device(0)
-        for single_launch in (True, False):
+        for single_launch in (2, 1, 0):
             h.set_schedule(single_launch)
             assert np.array_equal(_host(h.aggregate_fwd(xd, "sum")), a), (cut, single_launch)
             assert np.array_equal(_host(h.aggregate_bwd(xd, "sum")), b), (cut, single_launch)
@@ -298,6 +328,10 @@ def test_single_launch_is_one_kernel_and_its_bounded_wait_gives_up_cleanly():
     assert h.last_launch_count == 1
     h.set_schedule(False)
     assert torch.allclose(h.aggregate_fwd(x, "sum"), want, rtol=1e-4, atol=1e-4) and h.last_launch_count >= 2
+    h.set_schedule(2)          # the aggregation nodes (10+ levels) in one launch, the graph nodes in a second
+    assert torch.allclose(h.aggregate_fwd(x, "sum"), want, rtol=1e-4, atol=1e-4) and h.last_launch_count == 2
+    h.aggregate_bwd(x, "sum")
+    assert h.last_launch_count == 2
     h.set_schedule(True)
     lib = hb.load_library()
     assert h.device_status() == 0
@@ -309,7 +343,7 @@ def test_single_launch_is_one_kernel_and_its_bounded_wait_gives_up_cleanly():
     # ... and the handle stays usable
     assert torch.equal(h.aggregate_fwd(x, "sum"), want)
     assert h.device_status() == 0
-    assert lib.hag_device_status(None) == 1 and lib.hag_set_schedule(h._h, 2) == 2
+    assert lib.hag_device_status(None) == 1 and lib.hag_set_schedule(h._h, 3) == 2
     h.set_schedule(False)
 
 
