@@ -130,11 +130,12 @@ auto resident_kernel() {
     else return hagk::gather_sum_persistent_kernel<T, LPR, U, SS, MINB, SELF>;
 }
 
-template <typename T, int LPR, int U, bool SS, int MINB, bool SEGS, bool SELF>
+template <typename T, int LPR, int U, bool SS, int MINB, bool SEGS, bool SELF, int ITEMS>
 auto sub_kernel() {
-    if constexpr (SEGS) return hagk::gather_sum_sub_long_kernel<T, LPR, U, SS, MINB, SELF>;
-    else return hagk::gather_sum_sub_kernel<T, LPR, U, SS, MINB, SELF>;
+    if constexpr (SEGS) return hagk::gather_sum_sub_long_kernel<T, LPR, U, SS, MINB, SELF, ITEMS>;
+    else return hagk::gather_sum_sub_kernel<T, LPR, U, SS, MINB, SELF, ITEMS>;
 }
+constexpr int64_t kSubTwoGroupsRows = 262144;     // launches of this many rows give a warp two groups of rows
 
 // A launch that cannot give every resident warp a group of rows is bound by the latency of one row, which is shorter
 // with the whole warp on it.
@@ -149,10 +150,21 @@ cudaError_t launch_gather_shape(const hagk::GatherArgs &ga, const hagk::SegArgs 
     if constexpr (LPR < 32) {
         if (use_sub_rows(LPR, ga.row_count)) {
             constexpr int G = 32 / LPR;
-            const int64_t sub_items = (int64_t(ga.row_count) + G - 1) / G + (SEGS ? sg.seg_count : 0);
+            const int64_t groups = (int64_t(ga.row_count) + G - 1) / G;
+            const int items = ga.row_count >= kSubTwoGroupsRows ? 2 : 1;
+            const int64_t sub_items = (groups + items - 1) / items + (SEGS ? sg.seg_count : 0);
             const unsigned sub_grid = unsigned((sub_items + hagk::kWarps - 1) / hagk::kWarps);
-            if constexpr (sizeof(T) == 4) return launch_pdl(sub_kernel<T, LPR, 4, SS, SS ? 8 : 10, SEGS, SELF>(), sub_grid, a, s);
-            else return launch_pdl(sub_kernel<T, LPR, 2, SS, 8, SEGS, SELF>(), sub_grid, a, s);
+            // sweep on B200 (loads in flight per lane x CTAs per SM; cfg 2 / cfg 4 / clique-union step in ms): 4 x 10: 0.118 /
+            // 0.685 / 0.198; 8 x 8: 0.105 / 0.674 / 0.185; 8 x 9: 0.106 / 0.661 / 0.185; 16 x 5: 0.111 / 0.793 / 0.201;
+            // 2 x 16: 0.150 / 0.680 / 0.234.  A group walks its row alone, so loads in flight count for more here than
+            // in gather_row, where G groups share a row.
+            if constexpr (sizeof(T) == 4) {
+                if (items == 2) return launch_pdl(sub_kernel<T, LPR, 8, SS, SS ? 8 : 9, SEGS, SELF, 2>(), sub_grid, a, s);
+                return launch_pdl(sub_kernel<T, LPR, 8, SS, SS ? 8 : 9, SEGS, SELF, 1>(), sub_grid, a, s);
+            } else {
+                if (items == 2) return launch_pdl(sub_kernel<T, LPR, 2, SS, 8, SEGS, SELF, 2>(), sub_grid, a, s);
+                return launch_pdl(sub_kernel<T, LPR, 2, SS, 8, SEGS, SELF, 1>(), sub_grid, a, s);
+            }
         }
     }
     if constexpr (sizeof(T) == 4) {
@@ -270,6 +282,7 @@ cudaError_t launch_fused(const hag *h, const fused_table &t, hagk::GatherArgs a,
     k.ahat = ahat;
     k.err_host = h->d.err_dev;
     k.spin_limit = h->spin_limit;
+    k.static_order = head_only ? 1 : 0;
     const int lpr = lanes_per_row(n_chunks);
     const bool ss = a.src_scale != nullptr, self = !head_only && (a.out_is_f32 & 2) != 0;
 #define HAG_FUSED_CASE(L)                                                                                          \

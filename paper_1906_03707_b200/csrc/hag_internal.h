@@ -61,7 +61,7 @@ constexpr int kFusedMaxPhases = 56;       // deeper hierarchies run level by lev
 constexpr int64_t kFusedRowsForFullGrabs = 320000;   // phases with fewer rows are handed out two rows, below a quarter of it one row, per grab
 constexpr int kFusedCtlWords = 64;        // per launch: [0] next row, [1] finished warps, [2] error, [4 + p] finished rows of phase p
 constexpr int kFusedCtlSlots = 16;        // ring: consecutive launches (overlapping under programmatic dependent launch) take turns
-constexpr int kFusedSpinLimit = 1 << 21;  // polls of a waiting warp before it gives up (about a second)
+constexpr int kFusedSpinLimit = 1 << 20;  // polls of a waiting warp, a microsecond apart, before it gives up (about a second)
 
 struct fused_table {
     bool ok = false;                 // false: no row list (too many phases, or no rows); the id list is built all the same

@@ -572,7 +572,7 @@ __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_long_kernel(c
 // flight.  The groups of a warp run in lock step for as long as the longest of their rows lasts.
 // Order of additions of a row: per batch of LPR ids the tree sums of U rows at a time into `part`, batches into the
 // accumulator (two-level, as in gather_row).
-template <typename T, int LPR, int UNROLL, bool SRC_SCALE, bool HAS_SEGS, bool SELF>
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, bool HAS_SEGS, bool SELF, int ITEMS>
 __device__ __forceinline__ void gather_sum_sub_body(const KernelArgs<HAS_SEGS> &k) {
     static_assert(LPR < 32, "one row per warp is gather_row's job");
     const GatherArgs &a = k.a;
@@ -592,26 +592,55 @@ __device__ __forceinline__ void gather_sum_sub_body(const KernelArgs<HAS_SEGS> &
         item -= k.sg.seg_count;
     }
     const int slice = lane / LPR, gl = lane % LPR;
-    const int32_t r_local = item * G + slice;
+    // ITEMS groups of G rows per warp, one after the other: their row numbers, pointers and first ids are fetched
+    // together, so the order -> pointers -> ids chain of latencies is paid once per warp, not once per group.
+    // Measured on B200 with two groups: -3 % on 500 000 rows (cfg 4), +12 % and +36 % on 100 000 and 50 000 rows
+    // (half as many warps to fill the machine with): the host asks for two only on the largest launches.
+    item *= ITEMS;
     if (item * G >= a.row_count) return;
-    bool have = r_local < a.row_count;
-    int32_t row = a.row_begin + (have ? r_local : 0);
-    if (a.order) row = __ldg(a.order + row);
-    int32_t b = 0, e = 0;
-    if (have) {
-        b = __ldg(a.row_ptr + row);
-        e = __ldg(a.row_ptr + row + 1);
+    bool have_[ITEMS];
+    int32_t row_[ITEMS], b_[ITEMS], e_[ITEMS], mine_[ITEMS];
+    float mine_s_[ITEMS], dscale_[ITEMS];
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+        const int32_t r_local = (item + i) * G + slice;
+        have_[i] = r_local < a.row_count;
+        row_[i] = a.row_begin + (have_[i] ? r_local : 0);
     }
-    if constexpr (HAS_SEGS) {
-        if (e - b > k.sg.long_row) { have = false; e = b; }      // a long row: its segments are items of their own
+    if (a.order) {
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i) row_[i] = __ldg(a.order + row_[i]);
     }
-    int32_t mine = (b + gl < e) ? __ldg(a.idx + b + gl) : -1;
-    float mine_s = 1.0f;
-    if constexpr (SRC_SCALE) mine_s = (mine >= 0 && mine < a.n_prim) ? __ldg(a.src_scale + mine) : 1.0f;
-    const float dscale = (have && a.dst_scale && row < a.n_prim) ? __ldg(a.dst_scale + row) : 1.0f;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+        b_[i] = e_[i] = 0;
+        if (have_[i]) {
+            b_[i] = __ldg(a.row_ptr + row_[i]);
+            e_[i] = __ldg(a.row_ptr + row_[i] + 1);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+        if constexpr (HAS_SEGS) {
+            if (e_[i] - b_[i] > k.sg.long_row) { have_[i] = false; e_[i] = b_[i]; }      // a long row: its segments are items of their own
+        }
+        mine_[i] = (b_[i] + gl < e_[i]) ? __ldg(a.idx + b_[i] + gl) : -1;
+        mine_s_[i] = 1.0f;
+        if constexpr (SRC_SCALE) mine_s_[i] = (mine_[i] >= 0 && mine_[i] < a.n_prim) ? __ldg(a.src_scale + mine_[i]) : 1.0f;
+        dscale_[i] = (have_[i] && a.dst_scale && row_[i] < a.n_prim) ? __ldg(a.dst_scale + row_[i]) : 1.0f;
+    }
+    pdl_wait();        // structure arrays are static; features may come from the previous kernel
+    static_assert(ITEMS == 1 || ITEMS == 2, "the loop below selects between two sets of registers");
+#pragma unroll 1        // one copy of the loop body: two would not fit the register budget
+    for (int it = 0; it < ITEMS; ++it) {
+    if ((item + it) * G >= a.row_count) break;
+    const bool have = it ? have_[ITEMS - 1] : have_[0];
+    const int32_t row = it ? row_[ITEMS - 1] : row_[0], b = it ? b_[ITEMS - 1] : b_[0], e = it ? e_[ITEMS - 1] : e_[0];
+    int32_t mine = it ? mine_[ITEMS - 1] : mine_[0];
+    float mine_s = it ? mine_s_[ITEMS - 1] : mine_s_[0];
+    const float dscale = it ? dscale_[ITEMS - 1] : dscale_[0];
     const int32_t len = e - b;
     const int32_t max_len = __reduce_max_sync(FULL, len);
-    pdl_wait();        // structure arrays are static; features may come from the previous kernel
     const int n_chunks = a.D / E;
     const bool live = gl < n_chunks;
     const Tables<T> tab(a.prim, a.sec, a.n_prim, a.D, live ? gl : 0);
@@ -690,15 +719,16 @@ __device__ __forceinline__ void gather_sum_sub_body(const KernelArgs<HAS_SEGS> &
         for (int j = 0; j < E; ++j) acc[j] *= dscale;
         store_chunk<T>(a.out, a.out_is_f32 & 1, a.D, row - a.out_row_offset, gl, acc);
     }
+    }
 }
 
-template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS, bool SELF>
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS, bool SELF, int ITEMS>
 __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_sub_kernel(const KernelArgs<false> k) {
-    gather_sum_sub_body<T, LPR, UNROLL, SRC_SCALE, false, SELF>(k);
+    gather_sum_sub_body<T, LPR, UNROLL, SRC_SCALE, false, SELF, ITEMS>(k);
 }
-template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS, bool SELF>
+template <typename T, int LPR, int UNROLL, bool SRC_SCALE, int MIN_BLOCKS, bool SELF, int ITEMS>
 __global__ void __launch_bounds__(kThreads, MIN_BLOCKS) gather_sum_sub_long_kernel(const __grid_constant__ KernelArgs<true> k) {
-    gather_sum_sub_body<T, LPR, UNROLL, SRC_SCALE, true, SELF>(k);
+    gather_sum_sub_body<T, LPR, UNROLL, SRC_SCALE, true, SELF, ITEMS>(k);
 }
 
 // The same, with resident warps that take items four at a time from a shared
@@ -819,6 +849,11 @@ struct FusedArgs {
     float *ahat;               // = a.sec
     unsigned int *err_host;    // mapped host word, set when a wait ran out
     int32_t spin_limit;
+    int32_t static_order;      // 0: warps take the next four rows from the shared counter (balances a long last phase);
+                               // 1: warp w takes rows 4 w .. 4 w + 3, then the four W warps further on, and so on: no
+                               // shared counter, for lists of many short phases, where one atomic per row on a single
+                               // address costs more than the rows.  Needs every warp of the grid resident (as the
+                               // launch guarantees: no more CTAs than fit), like any wait between warps.
 };
 
 // Every lane polls (one address: one request per poll) and the exits are taken on warp votes, so the
@@ -834,7 +869,9 @@ __device__ __forceinline__ void fused_wait(const FusedArgs &k, int phase, int la
         asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(done) : "memory");
         if (__all_sync(FULL, v >= need)) { ok = true; break; }
         if (__any_sync(FULL, *failed != 0u)) break;     // somebody gave up already: do not add a second of waiting per row
-        __nanosleep(it < 32 ? 40 : 400);
+        // thousands of warps may wait for the same word, which is also the word the finishing warps add to: back off
+        // quickly, so that the polls do not stand in the way of what they wait for
+        __nanosleep(it < 2 ? 100 : (it < 6 ? 400 : 1000));
     }
     if (!ok && lane == 0) {
         k.ctl[kCtlError] = 1u;
@@ -853,9 +890,12 @@ __device__ __forceinline__ void fused_body(const FusedArgs &k) {
     constexpr unsigned FULL = 0xffffffffu;
     const int lane = threadIdx.x & 31;
     const int32_t count = k.n_items;
+    const int32_t stride = k.static_order ? int32_t(gridDim.x) * kWarps * CH : 0;
+    int32_t next_static = (int32_t(blockIdx.x) * kWarps + int32_t(threadIdx.x >> 5)) * CH;
     auto grab = [&]() -> int32_t {          // meaningful in lane 0
-        int32_t v = 0;
-        if (lane == 0) v = int32_t(atomicAdd(k.ctl + kCtlNext, unsigned(CH)));
+        int32_t v = next_static;
+        if (stride) next_static = min(next_static + stride, count);      // (count: nothing left; never overflows)
+        else if (lane == 0) v = int32_t(atomicAdd(k.ctl + kCtlNext, unsigned(CH)));
         return v;
     };
     // the four rows of a grab in ONE register per lane: lane 4 w + i holds word w (b, e, row, phases) of row i

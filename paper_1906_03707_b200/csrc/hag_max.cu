@@ -47,6 +47,7 @@ struct MaxArgs {
     void *out;
     int32_t out_is_f32;
     int32_t out_row_offset;
+    const int32_t *order;     // several-rows-per-warp kernels: the row taking the place of absolute row r, or null
 };
 
 struct PairMaxArgs {
@@ -90,20 +91,13 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {      // ex
     return *reinterpret_cast<const uint32_t *>(&r);
 }
 
+// max over the entries [b, e) of one row by the whole warp (`first`: the row's first 32 ids, one per lane).
 template <typename T, int LPR>
-__global__ void __launch_bounds__(kThreads, MaxShape<T>::kFwdBlocks) gather_max_kernel(const MaxArgs a) {
-    hagk::pdl_launch_dependents();
+__device__ __forceinline__ void max_row(const MaxArgs &a, int32_t row, int32_t b, int32_t e, int32_t first, int lane) {
     constexpr int E = Chunk<T>::kElems;
     constexpr int G = 32 / LPR;
     constexpr int U = MaxShape<T>::kFwdLoads < LPR ? MaxShape<T>::kFwdLoads : LPR;
     constexpr unsigned FULL = 0xffffffffu;
-    const int lane = threadIdx.x & 31;
-    const int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
-    if (r_local >= a.row_count) return;
-    const int32_t row = a.row_begin + r_local;
-    const int32_t b = __ldg(a.row_ptr + row), e = __ldg(a.row_ptr + row + 1);
-    const int32_t first = (b + lane < e) ? __ldg(a.idx + b + lane) : -1;
-    hagk::pdl_wait();
     const int slice = lane / LPR, gl = lane % LPR;
     const int n_chunks = a.D / E;
     const float ninf = __int_as_float(0xff800000);      // -infinity: the neutral element of max
@@ -225,6 +219,107 @@ __global__ void __launch_bounds__(kThreads, MaxShape<T>::kFwdBlocks) gather_max_
     }
 }
 
+template <typename T, int LPR>
+__global__ void __launch_bounds__(kThreads, MaxShape<T>::kFwdBlocks) gather_max_kernel(const MaxArgs a) {
+    hagk::pdl_launch_dependents();
+    const int lane = threadIdx.x & 31;
+    const int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (r_local >= a.row_count) return;
+    const int32_t row = a.row_begin + r_local;
+    const int32_t b = __ldg(a.row_ptr + row), e = __ldg(a.row_ptr + row + 1);
+    const int32_t first = (b + lane < e) ? __ldg(a.idx + b + lane) : -1;
+    hagk::pdl_wait();
+    max_row<T, LPR>(a, row, b, e, first, lane);
+}
+
+// Several rows per warp (feature rows of 256 bytes or less), as for the sums: every group of LPR lanes walks a row of its
+// own, taken in the list's by-length order, in lock step with the other groups; no value crosses lanes.  Rows are not
+// cut into segments here, so a row of more than kMaxSubLong entries is left out of the lock step and walked by the
+// whole warp afterwards.
+constexpr int32_t kMaxSubLong = 128;
+
+template <typename T, int LPR>
+__global__ void __launch_bounds__(kThreads, sizeof(T) == 4 ? 9 : 8) gather_max_sub_kernel(const MaxArgs a) {
+    static_assert(LPR < 32, "one row per warp is gather_max_kernel's job");
+    hagk::pdl_launch_dependents();
+    constexpr int E = Chunk<T>::kElems;
+    constexpr int G = 32 / LPR;
+    constexpr int U = sizeof(T) == 4 ? 8 : 2;      // fp32: 8 loads x 9 CTAs from a sweep (-7 % against 4 x 10 on cfg 4); bf16 rows are
+                                                   // widened to fp32 in flight, 8 registers each
+    constexpr unsigned FULL = 0xffffffffu;
+    const int lane = threadIdx.x & 31;
+    const int item = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (item * G >= a.row_count) return;
+    const int slice = lane / LPR, gl = lane % LPR;
+    const int32_t r_local = item * G + slice;
+    const bool have = r_local < a.row_count;
+    int32_t row = a.row_begin + (have ? r_local : 0);
+    if (a.order) row = __ldg(a.order + row);
+    int32_t b = 0, e = 0;
+    if (have) {
+        b = __ldg(a.row_ptr + row);
+        e = __ldg(a.row_ptr + row + 1);
+    }
+    const bool is_long = e - b > kMaxSubLong;
+    const int32_t len = is_long ? 0 : e - b;
+    int32_t mine = (gl < len) ? __ldg(a.idx + b + gl) : -1;
+    const int32_t max_len = __reduce_max_sync(FULL, len);
+    hagk::pdl_wait();
+    const int n_chunks = a.D / E;
+    const bool live = gl < n_chunks;
+    const float ninf = __int_as_float(0xff800000);
+    const Tables<T> tab(a.val_prim, a.val_sec, a.n_prim, a.D, live ? gl : 0);
+    float acc[E];
+#pragma unroll
+    for (int j = 0; j < E; ++j) acc[j] = ninf;
+    for (int32_t off = 0; off < max_len; off += LPR) {
+        const int32_t cur = mine;
+        const int32_t nb = off + LPR + gl;
+        mine = (nb < len) ? __ldg(a.idx + b + nb) : -1;
+        const int32_t cnt = len - off, max_cnt = max_len - off;
+#pragma unroll
+        for (int kk = 0; kk < LPR; kk += U) {
+            if (kk < max_cnt) {
+                float v[U][E];
+                if (__all_sync(FULL, kk + U <= cnt)) {
+#pragma unroll
+                    for (int u = 0; u < U; ++u) tab.load(__shfl_sync(FULL, cur, kk + u, LPR), v[u]);
+                } else {
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        const int32_t id = __shfl_sync(FULL, cur, kk + u, LPR);
+                        if (id >= 0 && live) {
+                            tab.load(id, v[u]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < E; ++j) v[u][j] = ninf;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+#pragma unroll
+                    for (int j = 0; j < E; ++j) acc[j] = fmaxf(acc[j], v[u][j]);
+            }
+        }
+    }
+    if (have && live && !is_long) {
+        if (e == b) {                 // empty neighbourhood: zero row
+#pragma unroll
+            for (int j = 0; j < E; ++j) acc[j] = 0.0f;
+        }
+        hagk::store_chunk<T>(a.out, a.out_is_f32, a.D, row - a.out_row_offset, gl, acc);
+    }
+    // the long rows among this warp's rows, one after the other, by the whole warp
+    unsigned todo = __ballot_sync(FULL, is_long && gl == 0);
+    while (todo) {
+        const int src = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const int32_t lrow = __shfl_sync(FULL, row, src), lb = __shfl_sync(FULL, b, src), le = __shfl_sync(FULL, e, src);
+        max_row<T, LPR>(a, lrow, lb, le, (lb + lane < le) ? __ldg(a.idx + lb + lane) : -1, lane);
+    }
+}
+
 // a-hat_w = max(a-hat_in0, a-hat_in1) for one level; one lane group per aggregation node.
 template <typename T, int LPR>
 __global__ void __launch_bounds__(kThreads) pair_max_kernel(const PairMaxArgs p) {
@@ -264,19 +359,11 @@ __device__ __forceinline__ void add_where_equal_bf16x8(float *acc, const uint4 &
 
 // grad_s[k] = sum over the destinations t of row s with max_t[k] == value_s[k] of grad_t[k].
 template <typename T, int LPR>
-__global__ void __launch_bounds__(kThreads, MaxShape<T>::bwd_blocks(LPR)) gather_maxgrad_kernel(const MaxArgs a) {
-    hagk::pdl_launch_dependents();
+__device__ __forceinline__ void maxgrad_row(const MaxArgs &a, int32_t row, int32_t b, int32_t e, int32_t first, int lane) {
     constexpr int E = Chunk<T>::kElems;
     constexpr int G = 32 / LPR;
     constexpr int U = MaxShape<T>::kBwdEntries < LPR ? MaxShape<T>::kBwdEntries : LPR;
     constexpr unsigned FULL = 0xffffffffu;
-    const int lane = threadIdx.x & 31;
-    const int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
-    if (r_local >= a.row_count) return;
-    const int32_t row = a.row_begin + r_local;
-    const int32_t b = __ldg(a.row_ptr + row), e = __ldg(a.row_ptr + row + 1);
-    const int32_t first = (b + lane < e) ? __ldg(a.idx + b + lane) : -1;
-    hagk::pdl_wait();
     const int slice = lane / LPR, gl = lane % LPR;
     const int n_chunks = a.D / E;
     for (int c0 = 0; c0 < n_chunks; c0 += LPR) {
@@ -409,6 +496,110 @@ __global__ void __launch_bounds__(kThreads, MaxShape<T>::bwd_blocks(LPR)) gather
     }
 }
 
+template <typename T, int LPR>
+__global__ void __launch_bounds__(kThreads, MaxShape<T>::bwd_blocks(LPR)) gather_maxgrad_kernel(const MaxArgs a) {
+    hagk::pdl_launch_dependents();
+    const int lane = threadIdx.x & 31;
+    const int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (r_local >= a.row_count) return;
+    const int32_t row = a.row_begin + r_local;
+    const int32_t b = __ldg(a.row_ptr + row), e = __ldg(a.row_ptr + row + 1);
+    const int32_t first = (b + lane < e) ? __ldg(a.idx + b + lane) : -1;
+    hagk::pdl_wait();
+    maxgrad_row<T, LPR>(a, row, b, e, first, lane);
+}
+
+// The backward form of gather_max_sub_kernel: a row per group of LPR lanes, two entries (a maximum row and a gradient
+// row each) in flight per lane; sums per batch of LPR ids, then batches.
+template <typename T, int LPR>
+__global__ void __launch_bounds__(kThreads, sizeof(T) == 4 ? 8 : 6) gather_maxgrad_sub_kernel(const MaxArgs a) {
+    static_assert(LPR < 32, "one row per warp is gather_maxgrad_kernel's job");
+    hagk::pdl_launch_dependents();
+    constexpr int E = Chunk<T>::kElems;
+    constexpr int G = 32 / LPR;
+    constexpr int U = sizeof(T) == 4 ? 4 : 2;      // entries (a maximum row and a gradient row each) in flight; fp32: 4 x 8 CTAs
+                                                   // from a sweep (-2 to -12 % against 2 x 10)
+    constexpr unsigned FULL = 0xffffffffu;
+    const int lane = threadIdx.x & 31;
+    const int item = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (item * G >= a.row_count) return;
+    const int slice = lane / LPR, gl = lane % LPR;
+    const int32_t r_local = item * G + slice;
+    const bool have = r_local < a.row_count;
+    int32_t row = a.row_begin + (have ? r_local : 0);
+    if (a.order) row = __ldg(a.order + row);
+    int32_t b = 0, e = 0;
+    if (have) {
+        b = __ldg(a.row_ptr + row);
+        e = __ldg(a.row_ptr + row + 1);
+    }
+    const bool is_long = e - b > kMaxSubLong;
+    const int32_t len = is_long ? 0 : e - b;
+    int32_t mine = (gl < len) ? __ldg(a.idx + b + gl) : -1;
+    const int32_t max_len = __reduce_max_sync(FULL, len);
+    hagk::pdl_wait();
+    const int n_chunks = a.D / E;
+    const bool live = gl < n_chunks;
+    const Tables<T> vals(a.val_prim, a.val_sec, a.n_prim, a.D, live ? gl : 0);
+    const Tables<T> grads(a.grad_prim, a.grad_sec, a.n_prim, a.D, live ? gl : 0);
+    float own[E], acc[E];
+    {
+        const Tables<T> self(a.own_prim, a.own_sec, a.n_prim, a.D, live ? gl : 0);
+        self.load(row, own);
+    }
+#pragma unroll
+    for (int j = 0; j < E; ++j) acc[j] = 0.0f;
+    for (int32_t off = 0; off < max_len; off += LPR) {
+        const int32_t cur = mine;
+        const int32_t nb = off + LPR + gl;
+        mine = (nb < len) ? __ldg(a.idx + b + nb) : -1;
+        const int32_t cnt = len - off, max_cnt = max_len - off;
+        float part[E];
+#pragma unroll
+        for (int j = 0; j < E; ++j) part[j] = 0.0f;
+#pragma unroll
+        for (int kk = 0; kk < LPR; kk += U) {
+            if (kk < max_cnt) {
+                float tv[U][E], tg[U][E];
+                if (__all_sync(FULL, kk + U <= cnt)) {
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        const int32_t id = __shfl_sync(FULL, cur, kk + u, LPR);
+                        vals.load(id, tv[u]);
+                        grads.load(id, tg[u]);
+                    }
+                } else {
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        const int32_t id = __shfl_sync(FULL, cur, kk + u, LPR);
+                        if (id >= 0 && live) {
+                            vals.load(id, tv[u]);
+                            grads.load(id, tg[u]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < E; ++j) { tv[u][j] = own[j]; tg[u][j] = 0.0f; }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+#pragma unroll
+                    for (int j = 0; j < E; ++j) part[j] += (tv[u][j] == own[j]) ? tg[u][j] : 0.0f;
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < E; ++j) acc[j] += part[j];
+    }
+    if (have && live && !is_long) hagk::store_chunk<T>(a.out, a.out_is_f32, a.D, row - a.out_row_offset, gl, acc);
+    unsigned todo = __ballot_sync(FULL, is_long && gl == 0);
+    while (todo) {
+        const int src = __ffs(todo) - 1;
+        todo &= todo - 1;
+        const int32_t lrow = __shfl_sync(FULL, row, src), lb = __shfl_sync(FULL, b, src), le = __shfl_sync(FULL, e, src);
+        maxgrad_row<T, LPR>(a, lrow, lb, le, (lb + lane < le) ? __ldg(a.idx + lb + lane) : -1, lane);
+    }
+}
+
 using DeviceScope = hagl::DeviceGuard;
 using hagl::aligned16;
 
@@ -419,14 +610,30 @@ cudaError_t launch(void (*kernel)(Args), int64_t warps, const Args &args, cudaSt
 
 inline int lanes_for(int n_chunks) { return hagl::lanes_per_row(n_chunks); }
 
+// Launches large enough to give every resident warp a group of rows take several rows per warp (as the sums do).
+constexpr int64_t kSubMinWarps = 4096;
+
+template <typename T, int LPR>
+cudaError_t launch_rows_lpr(bool grad, const MaxArgs &a, cudaStream_t s) {
+    if constexpr (LPR < 32) {
+        constexpr int G = 32 / LPR;
+        if (a.row_count >= kSubMinWarps * G) {
+            const int64_t items = (int64_t(a.row_count) + G - 1) / G;
+            return grad ? launch(gather_maxgrad_sub_kernel<T, LPR>, items, a, s) : launch(gather_max_sub_kernel<T, LPR>, items, a, s);
+        }
+    }
+    return grad ? launch(gather_maxgrad_kernel<T, LPR>, a.row_count, a, s) : launch(gather_max_kernel<T, LPR>, a.row_count, a, s);
+}
+
 template <typename T>
-cudaError_t launch_rows(bool grad, const MaxArgs &a, cudaStream_t s) {
+cudaError_t launch_rows(bool grad, MaxArgs a, const seg_set &set, cudaStream_t s) {
     if (a.row_count <= 0) return cudaSuccess;
+    a.order = set.d_order ? set.d_order - set.order_first_row : nullptr;
     switch (lanes_for(a.D / Chunk<T>::kElems)) {
-        case 4: return grad ? launch(gather_maxgrad_kernel<T, 4>, a.row_count, a, s) : launch(gather_max_kernel<T, 4>, a.row_count, a, s);
-        case 8: return grad ? launch(gather_maxgrad_kernel<T, 8>, a.row_count, a, s) : launch(gather_max_kernel<T, 8>, a.row_count, a, s);
-        case 16: return grad ? launch(gather_maxgrad_kernel<T, 16>, a.row_count, a, s) : launch(gather_max_kernel<T, 16>, a.row_count, a, s);
-        default: return grad ? launch(gather_maxgrad_kernel<T, 32>, a.row_count, a, s) : launch(gather_max_kernel<T, 32>, a.row_count, a, s);
+        case 4: return launch_rows_lpr<T, 4>(grad, a, s);
+        case 8: return launch_rows_lpr<T, 8>(grad, a, s);
+        case 16: return launch_rows_lpr<T, 16>(grad, a, s);
+        default: return launch_rows_lpr<T, 32>(grad, a, s);
     }
 }
 
@@ -481,7 +688,7 @@ hag_status max_fwd(hag *h, bool use_hag, int32_t D, const void *z, void *out, fl
             t.out = ahat;
             t.out_is_f32 = 1;
             t.out_row_offset = h->n;
-            if (launch_rows<T>(false, t, s) != cudaSuccess) return HAG_ERR_CUDA;
+            if (launch_rows<T>(false, t, h->seg_ftail, s) != cudaSuccess) return HAG_ERR_CUDA;
             ++launches;
         }
         a.val_sec = ahat;
@@ -493,7 +700,7 @@ hag_status max_fwd(hag *h, bool use_hag, int32_t D, const void *z, void *out, fl
     a.row_count = h->n;
     a.out = out;
     if (h->n > 0) {
-        if (launch_rows<T>(false, a, s) != cudaSuccess) return HAG_ERR_CUDA;
+        if (launch_rows<T>(false, a, use_hag ? h->seg_res : h->seg_csr, s) != cudaSuccess) return HAG_ERR_CUDA;
         ++launches;
     }
     h->last_launches = launches;
@@ -526,7 +733,7 @@ hag_status max_bwd(hag *h, bool use_hag, int32_t D, const void *z, const void *o
             t.out = ghat;
             t.out_is_f32 = 1;
             t.out_row_offset = h->n;
-            if (launch_rows<T>(true, t, s) != cudaSuccess) return HAG_ERR_CUDA;
+            if (launch_rows<T>(true, t, h->seg_btail, s) != cudaSuccess) return HAG_ERR_CUDA;
             ++launches;
         }
         for (int32_t l = h->bwd_cut; l >= 1; --l) {
@@ -539,7 +746,7 @@ hag_status max_bwd(hag *h, bool use_hag, int32_t D, const void *z, const void *o
             lv.out_is_f32 = 1;
             lv.out_row_offset = h->n;
             if (lv.row_count <= 0) continue;
-            if (launch_rows<T>(true, lv, s) != cudaSuccess) return HAG_ERR_CUDA;
+            if (launch_rows<T>(true, lv, h->seg_t, s) != cudaSuccess) return HAG_ERR_CUDA;
             ++launches;
         }
     }
@@ -549,7 +756,7 @@ hag_status max_bwd(hag *h, bool use_hag, int32_t D, const void *z, const void *o
     a.row_count = h->n;
     a.out = gz;
     if (h->n > 0) {
-        if (launch_rows<T>(true, a, s) != cudaSuccess) return HAG_ERR_CUDA;
+        if (launch_rows<T>(true, a, use_hag ? h->seg_t : h->seg_csr_t, s) != cudaSuccess) return HAG_ERR_CUDA;
         ++launches;
     }
     h->last_launches = launches;

@@ -139,6 +139,24 @@ def test_argument_errors():
     torch.cuda.synchronize()
 
 
+@pytest.mark.parametrize("dtype,d,ties", [("f32", 16, False), ("f32", 32, True), ("f32", 40, False), ("f32", 64, False),
+                                           ("bf16", 32, False), ("bf16", 64, True), ("bf16", 128, False)])
+def test_several_rows_per_warp_kernels(dtype, d, ties):
+    """Launches of 4096 x (groups per warp) rows or more take a row per group of lanes, in the list's by-length order;
+    rows of more than 128 entries among them are walked by the whole warp afterwards: the 70 000-row clique-union graph
+    (rows up to several hundred entries), every group width, dead lanes (d = 40), ties with integer gradients."""
+    w = synth.workload(6, scale=0.7)
+    g = w.graph
+    assert g.n >= 8 * 4096 and int(np.diff(g.row_ptr).max()) > 128
+    if ties:
+        z = np.clip(synth.features(3, g.n, d, "int", dtype), -1, 1).astype(np.float32)
+        gr = synth.features(4, g.n, d, "int", dtype)
+        # fp32 holds every integer sum exactly; a bf16 result is rounded, so that case keeps the tolerance
+        _check(g, w.capacity, d, dtype, seed=6, z=z, gr=gr, exact_grad=(dtype == "f32"))
+    else:
+        _check(g, w.capacity, d, dtype, seed=d)
+
+
 @pytest.mark.parametrize("index", [2, 4])
 def test_full_size_workloads(index):
     """The 50 000-node clustered workload and the batch of 5 000 small graphs at full size, fp32, D = 64:

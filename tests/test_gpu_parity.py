@@ -120,6 +120,20 @@ def test_several_rows_per_warp_kernels_match_oracle(dtype, d, reduce):
             assert np.array_equal(_host(bwd(xd, "sum")).astype(np.float64), b)
 
 
+@pytest.mark.parametrize("dtype,d,reduce", [("f32", 16, "mean"), ("f32", 32, "sum"), ("bf16", 64, "gcn"), ("bf16", 16, "sum")])
+def test_largest_launches_give_a_warp_two_groups_of_rows(dtype, d, reduce):
+    """From 262 144 rows on, a warp of the several-rows-per-warp kernels takes two groups of rows one after the other
+    (their pointers and first ids fetched together): 300 000 rows, 8 / 4 / 2 rows per group, both storage types."""
+    if "er-300k" not in _built:
+        g = synth.config4_graph(seed=77, n_graphs=6000, graph_size=50, p=0.3)
+        _built["er-300k"] = (g, hb.Hag.build(g.row_ptr, g.col_idx, g.n // 4).to_device(0))
+    g, h = _built["er-300k"]
+    assert g.n >= 262144
+    x = synth.features(55, g.n, d, "uniform", dtype)
+    gr = synth.upstream_grad(55, g.n, d, "uniform", dtype)
+    _check_all_paths(g, h, x, gr, reduce, dtype)
+
+
 @pytest.mark.parametrize("name", ["cfg1", "cfg2-small", "cfg4-small", "cfg5-small"])
 def test_structure_on_device_run_equals_oracle_structure(name):
     w, h = _case(name)
