@@ -46,6 +46,12 @@ L2_FLUSH_BYTES = 256 << 20
 NCU_FWD_GATHER = {
     "cfg3": {"dram_bytes": 719.8e6 + 115.6e6, "lts_throughput_pct": 73.2,
              "note": "profiles/gather_sum_persistent_cfg3.md: ncu --set full on this workload at full size"},
+    "cfg4": {"dram_bytes": 244.1e6 + 105.2e6, "lts_throughput_pct": 62.8,
+             "note": "profiles/gather_sum_sub_cfg4.md: ncu --set full on this workload at full size"},
+    "cfg2": {"dram_bytes": 23.6e6 + 0.2e6, "lts_throughput_pct": 45.8,
+             "note": "profiles/gather_sum_sub_cfg2.md: ncu --set full on this workload at full size"},
+    "clique-union": {"dram_bytes": 34.6e6 + 2.4e6, "lts_throughput_pct": 45.2,
+                     "note": "profiles/gather_sum_sub_clique_union.md: ncu --set full on this workload at full size"},
 }
 
 
@@ -586,6 +592,10 @@ def main():
             "plain_csr_ms_per_step": mi["csr_ms"], "speedup_hag_vs_plain": mi["ratio"], "steps": steps_i,
             "launches_per_step": mi["launches"] / steps_i, "hag": ri.hag_block(),
             "dtype": "f32" if wi.dtype == "f32" else "f32 accumulate, bf16 storage"})
+        if wi.name in NCU_FWD_GATHER:       # the ncu capture of this shape's largest launch: which roof it sits under
+            ni = NCU_FWD_GATHER[wi.name]
+            per_config[-1]["largest_launch_ncu"] = {"l2_frac": ni["lts_throughput_pct"] / 100.0, "dram_bytes": ni["dram_bytes"],
+                                                    "bound": "l2", "note": ni["note"]}
         ri.close()
         del ri
         torch.cuda.empty_cache()
