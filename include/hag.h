@@ -428,6 +428,23 @@ hag_status hag_export_pass(const hag_t *h, int32_t pass, hag_pass_view *out);
  * rebuilds lists 4 and 5.  Errors: NULL, ARG (list outside 0..5). */
 hag_status hag_export_row_order(const hag_t *h, int32_t list, int32_t *first_row, int64_t *count, const int32_t **order);
 
+/* Device-side check of the uploaded structure: small kernels read every index array on the device and test each
+ * pointer (first one 0, none stepping back, last one the list's length) and each id (inside the range of rows its
+ * list may name: graph nodes and aggregation nodes for the HAG's lists, graph nodes for the input graph, the levels
+ * up to the cut for the forward expansion, a permutation's own range for the row orders).  The aggregation kernels
+ * trust these arrays (hag_build validated the graph on the host before anything was derived from it), so this is
+ * the call that notices an upload or a device memory that went wrong, without a gather kernel ever being handed a
+ * bad index.  *failed_lists (may be NULL): bit 0 input pairs, 1 residual rows, 2 transposed HAG, 3 input graph, 4 its
+ * transpose, 5 / 6 forward / backward expansion, 7 row orders.  Allocates one word, synchronises the stream.
+ * Returns HAG_OK, or HAG_ERR_GRAPH if any bit is set.  Errors: NULL, NOT_ON_DEVICE, OOM_DEVICE, CUDA. */
+hag_status hag_device_validate(hag_t *h, uint32_t *failed_lists, void *cuda_stream);
+
+/* Test hook: the two predicates of hag_device_validate evaluated on the host: bit 0 = id lies in [lo, hi), bit 1 =
+ * pointer number i of a list of `rows` rows is acceptable (cur == first if i == 0, else cur >= prev; cur == last if
+ * i == rows). */
+int32_t hag_test_range_predicates(int32_t id, int32_t lo, int32_t hi, int64_t i, int64_t rows, int32_t prev, int32_t cur,
+                                  int32_t first, int32_t last);
+
 /* Test hook (process-wide): makes one of the library's next allocation attempts fail as if memory had run out,
  * so that callers can exercise their handling of HAG_ERR_OOM_HOST / HAG_ERR_OOM_DEVICE.  kind 0: host memory
  * (the checked points are the start of the search, of the layout and of every array upload), 1: device memory

@@ -26,7 +26,7 @@ HAG_F32, HAG_BF16 = 0, 1
  HAG_ERR_ALIGN, HAG_ERR_WORKSPACE, HAG_ERR_TIMEOUT, HAG_ERR_NOT_ON_DEVICE, HAG_ERR_TOO_LARGE) = range(13)
 
 EXPORTED_SYMBOLS = [
-    "hag_build", "hag_build_ex", "hag_build_threads", "hag_truncate", "hag_import", "hag_export_row_order", "hag_set_cuts", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes", "csr_workspace_bytes",
+    "hag_build", "hag_build_ex", "hag_build_threads", "hag_truncate", "hag_import", "hag_export_row_order", "hag_device_validate", "hag_test_range_predicates", "hag_set_cuts", "hag_destroy", "hag_get_info", "hag_export", "hag_to_device", "hag_workspace_bytes", "csr_workspace_bytes",
     "hag_aggregate_fwd", "hag_aggregate_bwd", "csr_aggregate_fwd", "csr_aggregate_bwd",
     "hag_aggregate_host", "hag_aggregate_fwd_static", "hag_graph_pool_fwd", "hag_graph_pool_bwd",
     "hag_max_workspace_bytes", "hag_max_fwd", "hag_max_bwd", "csr_max_fwd", "csr_max_bwd", "hag_profile_enable", "hag_profile_read", "hag_last_launch_count", "hag_status_str",
@@ -92,6 +92,10 @@ def load_library():
     lib.hag_truncate.restype = ctypes.c_int
     lib.hag_export_row_order.argtypes = [vp, i32, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(vp)]
     lib.hag_export_row_order.restype = ctypes.c_int
+    lib.hag_device_validate.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
+    lib.hag_device_validate.restype = ctypes.c_int
+    lib.hag_test_range_predicates.argtypes = [i32, i32, i32, ctypes.c_int64, ctypes.c_int64, i32, i32, i32, i32]
+    lib.hag_test_range_predicates.restype = i32
     lib.hag_import.argtypes = [i32, vp, vp, i32, vp, ctypes.POINTER(vp)]
     lib.hag_import.restype = ctypes.c_int
     lib.hag_set_cuts.argtypes = [vp, i32, i32]
@@ -293,6 +297,15 @@ class Hag:
         launch and the graph nodes in a second."""
         _check(load_library().hag_set_schedule(self._h, int(schedule)), "hag_set_schedule")
         return self
+
+    def device_validate(self, stream=None) -> int:
+        """``hag_device_validate``: 0 if every uploaded index array passes the device-side range checks, else the mask of
+        failed lists (raises for any other error)."""
+        mask = ctypes.c_uint32(0)
+        st = load_library().hag_device_validate(self._h, ctypes.byref(mask), stream)
+        if st not in (0, 3):
+            _check(st, "hag_device_validate")
+        return int(mask.value)
 
     def device_status(self) -> int:
         """``hag_device_status``: 0, or HAG_ERR_TIMEOUT if a device-side wait gave up (call after synchronising)."""

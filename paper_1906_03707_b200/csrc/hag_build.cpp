@@ -1039,6 +1039,11 @@ extern "C" hag_status hag_export_row_order(const hag_t *h, int32_t list, int32_t
     return HAG_OK;
 }
 
+extern "C" int32_t hag_test_range_predicates(int32_t id, int32_t lo, int32_t hi, int64_t i, int64_t rows, int32_t prev, int32_t cur,
+                                              int32_t first, int32_t last) {
+    return (hag_id_in_range(id, lo, hi) ? 1 : 0) | (hag_ptr_ok(i, rows, prev, cur, first, last) ? 2 : 0);
+}
+
 extern "C" const char *hag_status_str(hag_status s) {
     switch (s) {
         case HAG_OK: return "ok";

@@ -759,6 +759,76 @@ extern "C" hag_status hag_aggregate_host(hag_t *h, int backward, int use_hag, ha
 
 extern "C" int32_t hag_last_launch_count(const hag_t *h) { return h ? h->last_launches : 0; }
 
+// ---- device-side check of the uploaded structure (a diagnostic: no gather kernel is involved) ----------------------
+namespace {
+__global__ void check_ids_kernel(const int32_t *ids, int64_t count, int32_t lo, int32_t hi, unsigned int bit, unsigned int *err) {
+    for (int64_t i = blockIdx.x * int64_t(blockDim.x) + threadIdx.x; i < count; i += int64_t(gridDim.x) * blockDim.x)
+        if (!hag_id_in_range(ids[i], lo, hi)) {
+            atomicOr(err, bit);
+            return;
+        }
+}
+__global__ void check_ptr_kernel(const int32_t *ptr, int64_t rows, int32_t first, int32_t last, unsigned int bit, unsigned int *err) {
+    for (int64_t i = blockIdx.x * int64_t(blockDim.x) + threadIdx.x; i <= rows; i += int64_t(gridDim.x) * blockDim.x)
+        if (!hag_ptr_ok(i, rows, i ? ptr[i - 1] : 0, ptr[i], first, last)) {
+            atomicOr(err, bit);
+            return;
+        }
+}
+}  // namespace
+
+extern "C" hag_status hag_device_validate(hag_t *h, uint32_t *failed_lists, void *cuda_stream) {
+    if (!h) return HAG_ERR_NULL;
+    if (failed_lists) *failed_lists = 0;
+    if (h->device < 0) return HAG_ERR_NOT_ON_DEVICE;
+    hagl::DeviceGuard scope(h->device);
+    if (!scope.ok) { cudaGetLastError(); return HAG_ERR_CUDA; }
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    unsigned int *err = nullptr;
+    if (cudaMalloc(reinterpret_cast<void **>(&err), sizeof(unsigned int)) != cudaSuccess) { cudaGetLastError(); return HAG_ERR_OOM_DEVICE; }
+    bool ok = cudaMemsetAsync(err, 0, sizeof(unsigned int), s) == cudaSuccess;
+    const hag_device_arrays &d = h->d;
+    const int32_t n = h->n, k = h->num_agg;
+    auto grid_for = [](int64_t count) { return unsigned(std::max<int64_t>(1, std::min<int64_t>((count + 255) / 256, 1184))); };
+    auto ids = [&](const int32_t *p, int64_t count, int32_t lo, int32_t hi, int list) {
+        if (!ok || count <= 0 || !p) return;
+        check_ids_kernel<<<grid_for(count), 256, 0, s>>>(p, count, lo, hi, 1u << list, err);
+        ok = cudaGetLastError() == cudaSuccess;
+    };
+    auto ptrs = [&](const int32_t *p, int64_t rows, int64_t last, int list) {
+        if (!ok || !p) return;
+        check_ptr_kernel<<<grid_for(rows + 1), 256, 0, s>>>(p, rows, 0, int32_t(last), 1u << list, err);
+        ok = cudaGetLastError() == cudaSuccess;
+    };
+    const int64_t f_rows = int64_t(h->ftail_ptr.size()) - 1, b_rows = int64_t(h->btail_ptr.size()) - 1;
+    ids(d.agg_in, 2 * int64_t(k), 0, n + k, 0);
+    ptrs(d.res_ptr, n, h->e_res, 1);
+    ids(d.res_idx, h->e_res, 0, n + k, 1);
+    ptrs(d.t_ptr, int64_t(n) + k, h->e_hat, 2);
+    ids(d.t_idx, h->e_hat, 0, n + k, 2);
+    ptrs(d.csr_ptr, n, h->e, 3);
+    ids(d.csr_idx, h->e, 0, n, 3);
+    ptrs(d.csr_t_ptr, n, h->e, 4);
+    ids(d.csr_t_idx, h->e, 0, n, 4);
+    if (f_rows > 0) {       // sources of an expanded node: the layer input and the levels up to the forward cut
+        ptrs(d.ftail_ptr, f_rows, int64_t(h->ftail_idx.size()), 5);
+        ids(d.ftail_idx, int64_t(h->ftail_idx.size()), 0, n + int32_t(h->level_ptr[h->fwd_cut]), 5);
+    }
+    if (b_rows > 0) {       // destinations of an expanded node: graph nodes only
+        ptrs(d.btail_ptr, b_rows, int64_t(h->btail_idx.size()), 6);
+        ids(d.btail_idx, int64_t(h->btail_idx.size()), 0, n, 6);
+    }
+    for (const seg_set *set : {&h->seg_res, &h->seg_t, &h->seg_csr, &h->seg_csr_t, &h->seg_ftail, &h->seg_btail})
+        ids(set->d_order, int64_t(set->order.size()), set->order_first_row, set->order_first_row + int32_t(set->order.size()), 7);
+    unsigned int host = 0;
+    ok = ok && cudaMemcpyAsync(&host, err, sizeof(unsigned int), cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+         cudaStreamSynchronize(s) == cudaSuccess;
+    cudaFree(err);
+    if (!ok) { cudaGetLastError(); return HAG_ERR_CUDA; }
+    if (failed_lists) *failed_lists = host;
+    return host ? HAG_ERR_GRAPH : HAG_OK;
+}
+
 extern "C" hag_status hag_set_schedule(hag_t *h, int32_t schedule) {
     if (!h) return HAG_ERR_NULL;
     if (schedule < 0 || schedule > 2) return HAG_ERR_ARG;

@@ -8,6 +8,18 @@
 
 #include "hag.h"
 
+// Predicates of the device-side structure check (hag_device_validate), shared by its kernels and by the host test hook.
+#if defined(__CUDACC__)
+#define HAG_HOST_DEVICE __host__ __device__
+#else
+#define HAG_HOST_DEVICE
+#endif
+HAG_HOST_DEVICE inline bool hag_id_in_range(int32_t id, int32_t lo, int32_t hi) { return id >= lo && id < hi; }
+// pointer i of a CSR-like list: the first is `first`, none steps back, the last is `last`
+HAG_HOST_DEVICE inline bool hag_ptr_ok(int64_t i, int64_t rows, int32_t prev, int32_t cur, int32_t first, int32_t last) {
+    return (i == 0 ? cur == first : cur >= prev) && (i < rows || cur == last);
+}
+
 // Segments of the long rows of one CSR-like table (see hag_kernels.cuh): host copy and device copy.
 struct seg_table {
     std::vector<int32_t> segs;    // 4 per segment: row id, first entry, end entry, slot

@@ -506,3 +506,33 @@ def test_row_order_is_a_windowed_sort_by_length_that_keeps_every_launch_range():
     assert seen_sorted >= 2
     lib = hb.load_library()
     assert lib.hag_export_row_order(h._h, 6, ctypes.byref(ctypes.c_int32()), ctypes.byref(ctypes.c_int64()), ctypes.byref(ctypes.c_void_p())) == 2
+
+
+def test_range_predicates_of_the_device_side_check_on_the_host():
+    """hag_device_validate's kernels apply two predicates; here they run on the host (the GPU test only ever validates
+    good structures: no kernel is handed a bad index to see the check fire)."""
+    lib = hb.load_library()
+    pred = lib.hag_test_range_predicates
+
+    def id_ok(i, lo, hi):
+        return bool(pred(i, lo, hi, 0, 1, 0, 0, 0, 0) & 1)
+
+    def ptr_ok(i, rows, prev, cur, first, last):
+        return bool(pred(0, 0, 1, i, rows, prev, cur, first, last) & 2)
+
+    assert id_ok(0, 0, 1) and id_ok(9, 0, 10) and id_ok(5, 5, 6)
+    assert not id_ok(10, 0, 10) and not id_ok(-1, 0, 10) and not id_ok(4, 5, 6) and not id_ok(0, 0, 0)
+    assert not id_ok(2 ** 31 - 1, 0, 1000) and not id_ok(-2 ** 31, 0, 1000)
+    # a list of 3 rows with pointers 0, 2, 2, 7
+    good = [0, 2, 2, 7]
+    assert all(ptr_ok(i, 3, good[i - 1] if i else 0, good[i], 0, 7) for i in range(4))
+    assert not ptr_ok(0, 3, 0, 1, 0, 7)            # does not start at the list's beginning
+    assert not ptr_ok(2, 3, 2, 1, 0, 7)            # steps back
+    assert not ptr_ok(3, 3, 2, 6, 0, 7)            # does not end at the list's length
+    assert ptr_ok(3, 3, 7, 7, 0, 7) and ptr_ok(0, 0, 0, 0, 0, 0)
+    # without a device there is nothing to check
+    g = synth.config1_graph()
+    h = hb.Hag.build(g.row_ptr, g.col_idx, g.n // 4)
+    mask = ctypes.c_uint32(5)
+    assert lib.hag_device_validate(h._h, ctypes.byref(mask), None) == hb.HAG_ERR_NOT_ON_DEVICE and mask.value == 0
+    assert lib.hag_device_validate(None, None, None) == 1

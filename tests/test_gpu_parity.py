@@ -361,6 +361,26 @@ def test_single_launch_is_one_kernel_and_its_bounded_wait_gives_up_cleanly():
     h.set_schedule(False)
 
 
+def test_device_side_structure_check_passes_on_every_uploaded_structure():
+    """hag_device_validate reads every uploaded index array on the device and range-checks it: deep hierarchy with
+    both expansion lists and row orders, forced cuts, capacity 0, an empty graph."""
+    for name in ("cfg1", "cfg4-small", "clique-union-small", "clique-union-70k"):
+        w, h = _case(name)
+        assert h.device_validate() == 0, name
+    g = synth.workload(6, scale=0.03).graph
+    L = hb.Hag.build(g.row_ptr, g.col_idx, g.n // 4).info()["num_levels"]
+    for cuts in ((0, 0), (L, L), (1, L - 1)):
+        h = hb.Hag.build(g.row_ptr, g.col_idx, g.n // 4).set_cuts(*cuts).to_device(0)
+        assert h.device_validate(torch.cuda.current_stream().cuda_stream) == 0, cuts
+        h.close()
+    h = hb.Hag.build(g.row_ptr, g.col_idx, 0).to_device(0)
+    assert h.device_validate() == 0
+    h.close()
+    h = hb.Hag.build(np.zeros(1, np.int64), np.zeros(0, np.int32), 4).to_device(0)
+    assert h.device_validate() == 0
+    h.close()
+
+
 def test_empty_graph_launches_nothing():
     h = hb.Hag.build(np.zeros(1, np.int64), np.zeros(0, np.int32), 4).to_device(0)
     x = torch.empty((0, 64), device="cuda")
