@@ -44,7 +44,7 @@ L2_FLUSH_BYTES = 256 << 20
 # pass over the HAG, at the workload's full size): dram__bytes_read.sum + dram__bytes_write.sum per launch, and
 # lts__throughput (percent of the L2's peak) of that launch.
 NCU_FWD_GATHER = {
-    "cfg3": {"dram_bytes": 719.8e6 + 115.6e6, "lts_throughput_pct": 73.2,
+    "cfg3": {"dram_bytes": 599.9e6 + 114.4e6, "lts_throughput_pct": 79.2,
              "note": "profiles/gather_sum_persistent_cfg3.md: ncu --set full on this workload at full size"},
     "cfg4": {"dram_bytes": 244.1e6 + 105.2e6, "lts_throughput_pct": 62.8,
              "note": "profiles/gather_sum_sub_cfg4.md: ncu --set full on this workload at full size"},

@@ -169,7 +169,9 @@ cudaError_t launch_gather_shape(const hagk::GatherArgs &ga, const hagk::SegArgs 
     }
     if constexpr (sizeof(T) == 4) {
         if (ga.resident) {
-            if constexpr (LPR == 32) return launch_persistent(resident_kernel<T, LPR, 8, SS, 8, SEGS, SELF>(), a, items, sm_count, s);
+            // 512-byte rows and wider: 16 loads in flight per lane x 5 CTAs per SM (sweep on B200, cfg 3 step in ms: 8 x 8 2.44,
+            // 8 x 7 2.41, 16 x 4 2.39, 16 x 5 2.33, 16 x 6 2.48 (spills), 32 x 3 2.46, 4 x 12 2.71, no resident warps 2.82)
+            if constexpr (LPR == 32) return launch_persistent(resident_kernel<T, LPR, 16, SS, 5, SEGS, SELF>(), a, items, sm_count, s);
             return launch_persistent(resident_kernel<T, LPR, 4, SS, 8, SEGS, SELF>(), a, items, sm_count, s);
         }
         // the variant with per-source factors needs the registers of 8 CTAs per SM, or it spills
