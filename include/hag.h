@@ -422,8 +422,12 @@ hag_status hag_export_pass(const hag_t *h, int32_t pass, hag_pass_view *out);
  * (Algorithm 1 line 4), 3 its transpose, 4 / 5 the expansion lists of the forward / backward cut.  order[i] is the
  * row taking the place of row first_row + i: a permutation that sorts the rows by length (longest first) within
  * windows of 2048 rows, the windows never crossing from the graph nodes into a level or from one level into the next,
- * so every launch's rows map onto themselves.  count = 0 (order NULL): the rows are taken as they are (pairs of
- * neighbouring rows already lose less than 8 % of the lock-step rounds).  No value depends on the order: each row is
+ * so every launch's rows map onto themselves.  Aggregation nodes are numbered in the order of the search, not of the
+ * graph; a level or an expansion list of 8192 of their rows or more is therefore first put in the order of the rows'
+ * first entries (rows that read the same neighbourhood side by side: what one brings into the L2 the next find
+ * there; the one-row-per-warp kernel uses the order for these launches too), then cut into the windows.
+ * count = 0 (order NULL): the rows are taken as they are (pairs of neighbouring rows already lose less than 8 % of
+ * the lock-step rounds, and no segment qualifies for the order of first entries).  No value depends on the order: each row is
  * summed by one group in the row's own order of entries.  The array lives as long as the handle; hag_set_cuts
  * rebuilds lists 4 and 5.  Errors: NULL, ARG (list outside 0..5). */
 hag_status hag_export_row_order(const hag_t *h, int32_t list, int32_t *first_row, int64_t *count, const int32_t **order);

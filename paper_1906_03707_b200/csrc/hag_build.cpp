@@ -481,7 +481,13 @@ void build_segments(hag *h) {
     };
     // the row order of the several-rows-per-warp kernels (see seg_set); `bounds`: ascending local row indices where
     // launches begin (0 and rows included)
-    auto order = [](seg_set &set, const std::vector<int64_t> &ptr, int64_t rows, int32_t first_row_id, const std::vector<int64_t> &bounds) {
+    // `near_from`: from this segment of `bounds` on the rows are aggregation nodes, whose ids follow the order of the
+    // search, not of the graph: those segments are first put in the order of their first entry (rows that read the same
+    // neighbourhood side by side, so that what one row brings into the L2 the next ones find there), then sorted by
+    // length within the windows.  Segments of fewer than kOrderNearRows rows stay as they are (their launches are bound
+    // by latency, and the order costs a dependent load).
+    auto order = [](seg_set &set, const std::vector<int64_t> &ptr, const std::vector<int32_t> &idx, int64_t rows, int32_t first_row_id,
+                    const std::vector<int64_t> &bounds, size_t near_from) {
         set.order.clear();
         set.order_first_row = first_row_id;
         if (rows < 2) return;
@@ -492,17 +498,28 @@ void build_segments(hag *h) {
             own += a + b;
             paired += 2 * std::max(a, b);
         }
-        if (double(paired) < kOrderMinWaste * double(std::max<int64_t>(own, 1))) return;
+        bool any_near = false;
+        for (size_t i = near_from; i + 1 < bounds.size(); ++i) any_near = any_near || bounds[i + 1] - bounds[i] >= kOrderNearRows;
+        const bool by_length = double(paired) >= kOrderMinWaste * double(std::max<int64_t>(own, 1));
+        if (!by_length && !any_near) return;
         set.order.resize(size_t(rows));
         for (int64_t r = 0; r < rows; ++r) set.order[size_t(r)] = int32_t(first_row_id + r);
-        for (size_t i = 0; i + 1 < bounds.size(); ++i)
+        auto len_of = [&](int32_t x) { return ptr[x - first_row_id + 1] - ptr[x - first_row_id]; };
+        auto key_of = [&](int32_t x) {
+            const int64_t r = x - first_row_id;
+            return ptr[r] < ptr[r + 1] ? idx[size_t(ptr[r])] : std::numeric_limits<int32_t>::max();
+        };
+        for (size_t i = 0; i + 1 < bounds.size(); ++i) {
+            const bool near = i >= near_from && bounds[i + 1] - bounds[i] >= kOrderNearRows;
+            if (near)
+                std::stable_sort(set.order.begin() + bounds[i], set.order.begin() + bounds[i + 1],
+                                 [&](int32_t x, int32_t y) { return key_of(x) < key_of(y); });
+            if (!by_length && !near) continue;
             for (int64_t w0 = bounds[i]; w0 < bounds[i + 1]; w0 += kOrderWindow) {
                 const int64_t w1 = std::min<int64_t>(w0 + kOrderWindow, bounds[i + 1]);
-                std::stable_sort(set.order.begin() + w0, set.order.begin() + w1, [&](int32_t x, int32_t y) {
-                    const int64_t lx = ptr[x - first_row_id + 1] - ptr[x - first_row_id], ly = ptr[y - first_row_id + 1] - ptr[y - first_row_id];
-                    return lx > ly;
-                });
+                std::stable_sort(set.order.begin() + w0, set.order.begin() + w1, [&](int32_t x, int32_t y) { return len_of(x) > len_of(y); });
             }
+        }
     };
     std::vector<int64_t> t_bounds{0, n};
     for (size_t l = 1; l < h->level_ptr.size(); ++l) t_bounds.push_back(n + h->level_ptr[l]);
@@ -513,12 +530,13 @@ void build_segments(hag *h) {
     build(h->seg_csr_t, h->csr_t_ptr, n, 0);
     build(h->seg_ftail, h->ftail_ptr, f_rows, int32_t(n + h->level_ptr[h->fwd_cut]));
     build(h->seg_btail, h->btail_ptr, b_rows, int32_t(n + h->level_ptr[h->bwd_cut]));
-    order(h->seg_res, h->res_ptr, n, 0, {0, n});
-    order(h->seg_t, h->t_ptr, int64_t(n) + k, 0, t_bounds);
-    order(h->seg_csr, h->csr_ptr, n, 0, {0, n});
-    order(h->seg_csr_t, h->csr_t_ptr, n, 0, {0, n});
-    order(h->seg_ftail, h->ftail_ptr, f_rows, int32_t(n + h->level_ptr[h->fwd_cut]), {0, std::max<int64_t>(f_rows, 0)});
-    order(h->seg_btail, h->btail_ptr, b_rows, int32_t(n + h->level_ptr[h->bwd_cut]), {0, std::max<int64_t>(b_rows, 0)});
+    constexpr size_t kNone = size_t(1) << 30;
+    order(h->seg_res, h->res_ptr, h->res_idx, n, 0, {0, n}, kNone);
+    order(h->seg_t, h->t_ptr, h->t_idx, int64_t(n) + k, 0, t_bounds, 1);
+    order(h->seg_csr, h->csr_ptr, h->csr_idx, n, 0, {0, n}, kNone);
+    order(h->seg_csr_t, h->csr_t_ptr, h->csr_t_idx, n, 0, {0, n}, kNone);
+    order(h->seg_ftail, h->ftail_ptr, h->ftail_idx, f_rows, int32_t(n + h->level_ptr[h->fwd_cut]), {0, std::max<int64_t>(f_rows, 0)}, 0);
+    order(h->seg_btail, h->btail_ptr, h->btail_idx, b_rows, int32_t(n + h->level_ptr[h->bwd_cut]), {0, std::max<int64_t>(b_rows, 0)}, 0);
     h->max_segs_hag = std::max(std::max(h->seg_res.max_count(), h->seg_t.max_count()),
                                std::max(h->seg_ftail.max_count(), h->seg_btail.max_count()));
     h->max_segs_csr = std::max(h->seg_csr.max_count(), h->seg_csr_t.max_count());

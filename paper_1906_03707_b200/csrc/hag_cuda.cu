@@ -202,7 +202,10 @@ cudaError_t launch_gather(const hag *h, hagk::GatherArgs a, const seg_set &set, 
     const bool sub = use_sub_rows(lpr, a.row_count);
     // a lane group walks its row alone: nothing longer than 256 entries stays whole there
     const int gran = sub ? std::min(seg_gran_for_rows(a.row_count), 1) : seg_gran_for_rows(a.row_count);
-    a.order = (sub && set.d_order) ? set.d_order - set.order_first_row : nullptr;
+    // the row order: always for the several-rows-per-warp kernels; for the one-row-per-warp kernel on launches of
+    // aggregation-node rows large enough for it to matter (the resident-warp kernels take consecutive rows)
+    const bool near_rows = a.row_begin >= h->n && a.row_count >= kOrderNearRows && !(a.resident && sizeof(T) == 4);
+    a.order = (set.d_order && (sub || near_rows)) ? set.d_order - set.order_first_row : nullptr;
     const seg_table &table = set.g[gran];
     hagk::SegArgs sg{};
     sg.long_row = kSegLongRow[gran];

@@ -45,6 +45,7 @@ inline int seg_gran_for_rows(int64_t rows) { return rows < 8192 ? 0 : (rows < 65
 // rows as they are lose less than kOrderMinWaste of the lock-step rounds.
 constexpr int32_t kOrderWindow = 2048;
 constexpr double kOrderMinWaste = 1.08;
+constexpr int64_t kOrderNearRows = 8192;     // launches of aggregation-node rows from this size on are put in the order of their first entry
 
 struct seg_set {
     seg_table g[kSegGrans];

@@ -59,8 +59,9 @@ struct GatherArgs {
     int32_t out_is_f32;
     int32_t D;
     int32_t resident;         // host-side choice of the launch form; the kernels ignore it
-    const int32_t *order;     // several-rows-per-warp kernels only: the row that takes the place of absolute row r
-                              // (rows of like length side by side), or null for the rows as they are
+    const int32_t *order;     // the row that takes the place of absolute row r (rows of like length side by side for the
+                              // several-rows-per-warp kernels; aggregation-node rows that read the same neighbourhood
+                              // side by side), or null for the rows as they are; the resident-warp kernels ignore it
 };
 
 // Long rows (more than long_row entries) are not walked by one warp: they are cut into segments that
@@ -542,7 +543,8 @@ __device__ __forceinline__ void gather_sum_body(const KernelArgs<HAS_SEGS> &k) {
         r_local -= k.sg.seg_count;
     }
     if (r_local >= a.row_count) return;
-    const int32_t row = a.row_begin + r_local;
+    int32_t row = a.row_begin + r_local;
+    if (a.order) row = __ldg(a.order + row);       // aggregation-node rows in the order of their neighbourhoods
     const int32_t b = __ldg(a.row_ptr + row), e = __ldg(a.row_ptr + row + 1);
     if constexpr (HAS_SEGS) {
         if (e - b > k.sg.long_row) return;

@@ -228,7 +228,8 @@ __global__ void __launch_bounds__(kThreads, MaxShape<T>::fwd_blocks(LPR)) gather
     const int lane = threadIdx.x & 31;
     const int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
     if (r_local >= a.row_count) return;
-    const int32_t row = a.row_begin + r_local;
+    int32_t row = a.row_begin + r_local;
+    if (a.order) row = __ldg(a.order + row);
     const int32_t b = __ldg(a.row_ptr + row), e = __ldg(a.row_ptr + row + 1);
     const int32_t first = (b + lane < e) ? __ldg(a.idx + b + lane) : -1;
     hagk::pdl_wait();
@@ -505,7 +506,8 @@ __global__ void __launch_bounds__(kThreads, MaxShape<T>::bwd_blocks(LPR)) gather
     const int lane = threadIdx.x & 31;
     const int r_local = blockIdx.x * kWarps + (threadIdx.x >> 5);
     if (r_local >= a.row_count) return;
-    const int32_t row = a.row_begin + r_local;
+    int32_t row = a.row_begin + r_local;
+    if (a.order) row = __ldg(a.order + row);
     const int32_t b = __ldg(a.row_ptr + row), e = __ldg(a.row_ptr + row + 1);
     const int32_t first = (b + lane < e) ? __ldg(a.idx + b + lane) : -1;
     hagk::pdl_wait();
@@ -629,10 +631,14 @@ cudaError_t launch_rows_lpr(bool grad, const MaxArgs &a, cudaStream_t s) {
 }
 
 template <typename T>
-cudaError_t launch_rows(bool grad, MaxArgs a, const seg_set &set, cudaStream_t s) {
+cudaError_t launch_rows(bool grad, MaxArgs a, const seg_set &set, bool agg_rows, cudaStream_t s) {
     if (a.row_count <= 0) return cudaSuccess;
-    a.order = set.d_order ? set.d_order - set.order_first_row : nullptr;
-    switch (lanes_for(a.D / Chunk<T>::kElems)) {
+    const int lpr = lanes_for(a.D / Chunk<T>::kElems);
+    // the row order: for the several-rows-per-warp kernels, and for launches of aggregation-node rows large enough for
+    // the order of their neighbourhoods to matter
+    const bool sub = lpr < 32 && a.row_count >= kSubMinWarps * (32 / lpr);
+    a.order = (set.d_order && (sub || (agg_rows && a.row_count >= kOrderNearRows))) ? set.d_order - set.order_first_row : nullptr;
+    switch (lpr) {
         case 4: return launch_rows_lpr<T, 4>(grad, a, s);
         case 8: return launch_rows_lpr<T, 8>(grad, a, s);
         case 16: return launch_rows_lpr<T, 16>(grad, a, s);
@@ -691,7 +697,7 @@ hag_status max_fwd(hag *h, bool use_hag, int32_t D, const void *z, void *out, fl
             t.out = ahat;
             t.out_is_f32 = 1;
             t.out_row_offset = h->n;
-            if (launch_rows<T>(false, t, h->seg_ftail, s) != cudaSuccess) return HAG_ERR_CUDA;
+            if (launch_rows<T>(false, t, h->seg_ftail, true, s) != cudaSuccess) return HAG_ERR_CUDA;
             ++launches;
         }
         a.val_sec = ahat;
@@ -703,7 +709,7 @@ hag_status max_fwd(hag *h, bool use_hag, int32_t D, const void *z, void *out, fl
     a.row_count = h->n;
     a.out = out;
     if (h->n > 0) {
-        if (launch_rows<T>(false, a, use_hag ? h->seg_res : h->seg_csr, s) != cudaSuccess) return HAG_ERR_CUDA;
+        if (launch_rows<T>(false, a, use_hag ? h->seg_res : h->seg_csr, false, s) != cudaSuccess) return HAG_ERR_CUDA;
         ++launches;
     }
     h->last_launches = launches;
@@ -736,7 +742,7 @@ hag_status max_bwd(hag *h, bool use_hag, int32_t D, const void *z, const void *o
             t.out = ghat;
             t.out_is_f32 = 1;
             t.out_row_offset = h->n;
-            if (launch_rows<T>(true, t, h->seg_btail, s) != cudaSuccess) return HAG_ERR_CUDA;
+            if (launch_rows<T>(true, t, h->seg_btail, true, s) != cudaSuccess) return HAG_ERR_CUDA;
             ++launches;
         }
         for (int32_t l = h->bwd_cut; l >= 1; --l) {
@@ -749,7 +755,7 @@ hag_status max_bwd(hag *h, bool use_hag, int32_t D, const void *z, const void *o
             lv.out_is_f32 = 1;
             lv.out_row_offset = h->n;
             if (lv.row_count <= 0) continue;
-            if (launch_rows<T>(true, lv, h->seg_t, s) != cudaSuccess) return HAG_ERR_CUDA;
+            if (launch_rows<T>(true, lv, h->seg_t, true, s) != cudaSuccess) return HAG_ERR_CUDA;
             ++launches;
         }
     }
@@ -759,7 +765,7 @@ hag_status max_bwd(hag *h, bool use_hag, int32_t D, const void *z, const void *o
     a.row_count = h->n;
     a.out = gz;
     if (h->n > 0) {
-        if (launch_rows<T>(true, a, use_hag ? h->seg_t : h->seg_csr_t, s) != cudaSuccess) return HAG_ERR_CUDA;
+        if (launch_rows<T>(true, a, use_hag ? h->seg_t : h->seg_csr_t, false, s) != cudaSuccess) return HAG_ERR_CUDA;
         ++launches;
     }
     h->last_launches = launches;

@@ -536,3 +536,42 @@ def test_range_predicates_of_the_device_side_check_on_the_host():
     mask = ctypes.c_uint32(5)
     assert lib.hag_device_validate(h._h, ctypes.byref(mask), None) == hb.HAG_ERR_NOT_ON_DEVICE and mask.value == 0
     assert lib.hag_device_validate(None, None, None) == 1
+
+
+def test_large_aggregation_node_segments_follow_their_neighbourhoods():
+    """Segments of 8192 aggregation-node rows or more (a level of the transposed HAG, an expansion list) are put in
+    the order of their first entry before the windows are sorted by length: a permutation of the segment, windows
+    sorted by length, and every window's first entries at or above those of the window before."""
+    g = synth.config4_graph(seed=9, n_graphs=400, graph_size=100)
+    h = hb.Hag.build(g.row_ptr, g.col_idx, g.n // 4)
+    a = h.arrays()
+    n, k = g.n, int(a["num_agg"])
+    level_ptr = np.asarray(a["level_ptr"], dtype=np.int64)
+    assert level_ptr[1] >= 8192
+
+    def check_segment(order, first, ptr, idx, s0, s1):
+        seg = order[s0:s1]
+        assert np.array_equal(np.sort(seg), first + np.arange(s0, s1))                 # the segment maps onto itself
+        lens = np.diff(ptr)
+        key = np.where(lens > 0, idx[np.minimum(ptr[:-1], len(idx) - 1)], np.iinfo(np.int32).max)
+        prev_max = -1
+        for w0 in range(s0, s1, 2048):
+            win = order[w0:min(w0 + 2048, s1)] - first
+            assert np.all(np.diff(lens[win]) <= 0)                                     # longest first inside a window
+            assert key[win].min() >= prev_max                                          # windows ascend in their first entries
+            prev_max = key[win].max()
+        moved = np.flatnonzero(seg != first + np.arange(s0, s1))
+        assert moved.size > 0
+
+    t_ptr, t_idx = np.asarray(a["t_ptr"], dtype=np.int64), np.asarray(a["t_idx"])
+    first, order = h.row_order(1)
+    assert first == 0 and order.size == n + k
+    check_segment(order, 0, t_ptr, t_idx, n, n + int(level_ptr[1]))
+    for cut_f, cut_b in ((0, 0),):
+        h.set_cuts(cut_f, cut_b)
+        v = h.arrays()
+        for which, ptr_key, idx_key in ((4, "ftail_ptr", "ftail_idx"), (5, "btail_ptr", "btail_idx")):
+            first, order = h.row_order(which)
+            ptr, idx = np.asarray(v[ptr_key], dtype=np.int64), np.asarray(v[idx_key])
+            assert first == n and order.size == k == ptr.size - 1
+            check_segment(order, n, ptr, idx, 0, k)
