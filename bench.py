@@ -46,7 +46,7 @@ L2_FLUSH_BYTES = 256 << 20
 NCU_FWD_GATHER = {
     "cfg3": {"dram_bytes": 599.9e6 + 114.4e6, "lts_throughput_pct": 79.2,
              "note": "profiles/gather_sum_persistent_cfg3.md: ncu --set full on this workload at full size"},
-    "cfg4": {"dram_bytes": 244.1e6 + 105.2e6, "lts_throughput_pct": 62.8,
+    "cfg4": {"dram_bytes": 244.1e6 + 105.1e6, "lts_throughput_pct": 63.5,
              "note": "profiles/gather_sum_sub_cfg4.md: ncu --set full on this workload at full size"},
     "cfg2": {"dram_bytes": 23.6e6 + 0.2e6, "lts_throughput_pct": 45.8,
              "note": "profiles/gather_sum_sub_cfg2.md: ncu --set full on this workload at full size"},
