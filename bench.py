@@ -48,7 +48,7 @@ NCU_FWD_GATHER = {
              "note": "profiles/gather_sum_persistent_cfg3.md: ncu --set full on this workload at full size"},
     "cfg4": {"dram_bytes": 244.1e6 + 105.1e6, "lts_throughput_pct": 63.5,
              "note": "profiles/gather_sum_sub_cfg4.md: ncu --set full on this workload at full size"},
-    "cfg5": {"dram_bytes": 2103.9e6 + 513.4e6, "lts_throughput_pct": 61.2,
+    "cfg5": {"dram_bytes": 2109.6e6 + 514.7e6, "lts_throughput_pct": 64.5,
              "note": "profiles/gather_sum_bf16_cfg5.md: ncu --set full on this workload at full size"},
     "cfg2": {"dram_bytes": 23.6e6 + 0.2e6, "lts_throughput_pct": 45.8,
              "note": "profiles/gather_sum_sub_cfg2.md: ncu --set full on this workload at full size"},

@@ -140,6 +140,16 @@ __device__ __forceinline__ void add_rows(float *a, const float *b) {
 template <bool SCALED>
 __device__ __forceinline__ void add_bf16x8(float *acc, const uint4 &r, float factor) {
     const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+    if constexpr (!SCALED) {
+        // sm_100 adds a bf16 value to an fp32 one in one instruction (add.f32.bf16: the bf16 operand is widened exactly,
+        // the sum rounded to nearest, i.e. the bits of widening first and adding then): 8 instructions per 16 bytes
+        // instead of 8 shifts or masks and 4 packed adds
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.rn.f32.bf16 %0, lo, %0;\n\tadd.rn.f32.bf16 %1, hi, %1;\n\t}"
+                : "+f"(acc[2 * i]), "+f"(acc[2 * i + 1])
+                : "r"(w[i]));
+    } else {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const float2 x = make_float2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xffff0000u));
@@ -147,6 +157,7 @@ __device__ __forceinline__ void add_bf16x8(float *acc, const uint4 &r, float fac
         const float2 s = SCALED ? __ffma2_rn(x, make_float2(factor, factor), a) : __fadd2_rn(a, x);
         acc[2 * i] = s.x;
         acc[2 * i + 1] = s.y;
+    }
     }
 }
 
